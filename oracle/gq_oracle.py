@@ -1,0 +1,141 @@
+"""CPU fp64 oracle for the guided layer objective (GuidedQuant, Section 3.2).
+
+TEST INFRASTRUCTURE ONLY: imported by ``tests/``, by ``__graft_entry__.smoke``
+and by the ``cpu_baseline`` / ``--impl reference`` legs of ``bench.py``.  The
+product package never imports it and it never imports the product's CUDA path.
+
+Two independent statements of the same definitions live here:
+
+* ``impl="c"`` -- ``gq_oracle.c``: entry-by-entry fp64 loops (the oracle of
+  record; fast enough for token prefixes of the large layers);
+* ``impl="numpy"`` -- the definitions written with numpy fp64 library
+  primitives (``einsum`` / ``@``), used to cross-check the C loops and for
+  tiny cases.
+
+Array conventions (identical to the C-ABI library so the same buffers serve
+both sides): ``grad`` and ``X`` are ``uint16`` arrays holding bf16 bit patterns,
+row = token; ``s`` is ``[g, n]``; ``H`` is ``[g, d_in, d_in]``; ``W``/``W_hat``
+are fp32 ``[d_out, d_in]`` with row ``j`` = output channel ``j`` (the paper's
+column ``w_j``, Section 2).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gq_oracle.c")
+_LIB = os.path.join(_HERE, "libgq_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile ``gq_oracle.c`` with gcc (OpenMP) next to its source."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", tmp, _SRC])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _c():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i64, i32, dbl, vp = ctypes.c_int64, ctypes.c_int32, ctypes.c_double, ctypes.c_void_p
+        lib.gq_oracle_saliency.argtypes = [vp, i64, i64, i64, i32, dbl, vp, i64]
+        lib.gq_oracle_hessian_accumulate.argtypes = [vp, i64, i64, i64, vp, i64, i32, vp]
+        lib.gq_oracle_objective.argtypes = [vp, vp, i64, i64, vp, i32, vp]
+        for f in (lib.gq_oracle_saliency, lib.gq_oracle_hessian_accumulate, lib.gq_oracle_objective,
+                  lib.gq_oracle_threads):
+            f.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def threads() -> int:
+    return int(_c().gq_oracle_threads())
+
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Widen bf16 bit patterns (uint16) to fp64 exactly."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def f64_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round fp64/fp32 values to bf16 (nearest, ties to even); for building test inputs."""
+    f = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    rounded = (f + 0x7FFF + ((f >> 16) & 1)) >> 16
+    return rounded.astype(np.uint16)
+
+
+def _ptr(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def saliency(grad_bits: np.ndarray, g: int, grad_scale: float = 1.0, impl: str = "c") -> np.ndarray:
+    """Algorithm 1 line 2: ``s[k, i] = mean_{j in J_k} (grad_scale * grad[i, j])**2``."""
+    grad_bits = np.ascontiguousarray(grad_bits, dtype=np.uint16)
+    n, d_out = grad_bits.shape
+    if g < 1 or d_out % g:
+        raise ValueError("d_out must be divisible by g")
+    if impl == "numpy":
+        gr = bf16_bits_to_f64(grad_bits) * float(grad_scale)
+        return np.ascontiguousarray((gr * gr).reshape(n, g, d_out // g).mean(axis=2).T)
+    s = np.zeros((g, n), dtype=np.float64)
+    rc = _c().gq_oracle_saliency(_ptr(grad_bits), n, d_out, d_out, g, float(grad_scale), _ptr(s), n)
+    if rc:
+        raise RuntimeError("gq_oracle_saliency rc=%d" % rc)
+    return s
+
+
+def hessian(x_bits: np.ndarray, s: np.ndarray, H: np.ndarray | None = None, impl: str = "c") -> np.ndarray:
+    """Algorithm 1 line 4: ``H[k] (+)= X^T Diag(s[k]) X`` (full matrices, no 1/n).
+
+    Passing ``H`` accumulates into it (streaming over token chunks)."""
+    x_bits = np.ascontiguousarray(x_bits, dtype=np.uint16)
+    s = np.ascontiguousarray(s, dtype=np.float64)
+    n, d_in = x_bits.shape
+    g = s.shape[0]
+    if s.shape[1] != n:
+        raise ValueError("s must be [g, n]")
+    if H is None:
+        H = np.zeros((g, d_in, d_in), dtype=np.float64)
+    assert H.shape == (g, d_in, d_in) and H.dtype == np.float64 and H.flags.c_contiguous
+    if impl == "numpy":
+        x = bf16_bits_to_f64(x_bits)
+        for k in range(g):
+            H[k] += (x * s[k][:, None]).T @ x
+        return H
+    rc = _c().gq_oracle_hessian_accumulate(_ptr(x_bits), n, d_in, d_in, _ptr(s), n, g, _ptr(H))
+    if rc:
+        raise RuntimeError("gq_oracle_hessian_accumulate rc=%d" % rc)
+    return H
+
+
+def objective(W: np.ndarray, W_hat: np.ndarray, H: np.ndarray, impl: str = "c") -> np.ndarray:
+    """Eq. 7: ``loss[k] = sum_{j in J_k} (w_j - what_j)^T H[k] (w_j - what_j)``; ``loss[g]`` = total."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    W_hat = np.ascontiguousarray(W_hat, dtype=np.float32)
+    H = np.ascontiguousarray(H, dtype=np.float64)
+    d_out, d_in = W.shape
+    g = H.shape[0]
+    if W_hat.shape != W.shape or H.shape != (g, d_in, d_in) or d_out % g:
+        raise ValueError("shape mismatch")
+    loss = np.zeros(g + 1, dtype=np.float64)
+    if impl == "numpy":
+        m = d_out // g
+        delta = W.astype(np.float64) - W_hat.astype(np.float64)
+        for k in range(g):
+            dk = delta[k * m:(k + 1) * m]
+            loss[k] = np.einsum("ja,ab,jb->", dk, H[k], dk, optimize=True)
+        loss[g] = loss[:g].sum()
+        return loss
+    rc = _c().gq_oracle_objective(_ptr(W), _ptr(W_hat), d_in, d_out, _ptr(H), g, _ptr(loss))
+    if rc:
+        raise RuntimeError("gq_oracle_objective rc=%d" % rc)
+    return loss
