@@ -1,0 +1,164 @@
+/*
+ * libgq -- construction of GuidedQuant's end-loss-guided layer objective on one B200 (sm_100a).
+ *
+ * For one linear layer with input activations X (n tokens x d_in), end-loss gradients of the
+ * layer output dl/dZ (n x d_out) and weights W, the library computes
+ *
+ *   J_k   = { m k, ..., m (k+1) - 1 },  m = d_out / g          (Algorithm 1, line 1)
+ *   s_k   = 1/|J_k| * sum_{j in J_k} (dl/dz_j)^2                (Algorithm 1, line 2)
+ *   H_k   = X^T Diag(s_k) X                                     (Algorithm 1, line 4; Section 3.2)
+ *   loss  = sum_k sum_{j in J_k} (w_j - what_j)^T H_k (w_j - what_j)          (Eq. 7)
+ *
+ * Conventions shared by every call
+ *   - Plain C ABI.  Unless a parameter is documented as HOST memory, every pointer is a DEVICE
+ *     pointer owned by the caller; the library never allocates or frees device memory and never
+ *     keeps a pointer after the call returns.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls only
+ *     enqueue work; they do not synchronise the host.  Results are in device memory and are
+ *     ordered after the call on `stream`.
+ *   - Return value: GQ_OK or a negative gq_status.  Invalid arguments are detected on the host
+ *     before anything is launched; nothing is written in that case.
+ *   - Problems that can only be seen on the device (a pipeline wait that ran out of its time
+ *     budget) are recorded in a per-device status word that gq_check() reads.
+ *   - Tokens are rows: X is [n, ld_x] and dl/dZ is [n, ld_grad], both bf16, row-major.
+ *     Weights are [d_out, d_in] row-major fp32, i.e. row j is the paper's column w_j (Section 2).
+ */
+#ifndef GQ_H_
+#define GQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum gq_status {
+    GQ_OK = 0,
+    GQ_ERR_INVALID_ARG = -1,       /* null pointer, negative size, g < 1, d_out % g != 0, bad flags  */
+    GQ_ERR_ALIGNMENT = -2,         /* pointer or leading dimension not aligned as documented          */
+    GQ_ERR_UNSUPPORTED_SHAPE = -3, /* size outside what the kernels index (see each call)             */
+    GQ_ERR_WORKSPACE = -4,         /* workspace missing or smaller than the *_workspace_bytes() value */
+    GQ_ERR_CUDA = -5,              /* a CUDA runtime/driver call failed: see gq_last_cuda_error()     */
+    GQ_ERR_TIMEOUT = -6            /* a device-side wait gave up (reported by gq_check)               */
+} gq_status;
+
+/* Library version, major * 10000 + minor * 100 + patch. */
+int gq_version(void);
+
+/* Static, human readable name of a status code (never NULL). */
+const char *gq_status_string(int32_t status);
+
+/* The cudaError_t value of the most recent failing CUDA call made by this library on the
+ * calling thread (0 if none). */
+int32_t gq_last_cuda_error(void);
+
+/*
+ * Saliency: Algorithm 1, line 2, with the gradient scaling of Section 3.2 applied to the gradient
+ * before it is squared:
+ *     s[k * ld_s + i] = (grad_scale^2 / m) * sum_{j = m k}^{m (k+1) - 1} grad[i * ld_grad + j]^2
+ *
+ *   grad        bf16 [n, ld_grad], 16-byte aligned, ld_grad >= d_out, ld_grad % 8 == 0
+ *   n           tokens in this call, >= 0 (0 is a no-op)
+ *   d_out, g    d_out % g == 0 and (d_out / g) % 8 == 0, 1 <= g <= 1024
+ *   grad_scale  finite; the paper uses 1e3, tests use 1
+ *   s           fp32 [g, ld_s] (group-major so that each s_k is contiguous), ld_s >= n
+ * Squares and sums are fp32.  The result does not depend on the launch shape.
+ */
+int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad, int32_t g,
+                    float grad_scale, float *s, int64_t ld_s, void *stream);
+
+/*
+ * Guided Hessian, one token chunk: Algorithm 1, line 4, streamed,
+ *     H[k][a][b] += sum_{i < n} s[k * ld_s + i] * X[i * ld_x + a] * X[i * ld_x + b]
+ * for every group k and every a <= b (the upper triangle including the diagonal).  No 1/n factor.
+ *
+ *   X          bf16 [n, ld_x], 16-byte aligned, ld_x >= d_in, ld_x % 8 == 0
+ *   n          tokens in this chunk, 0 <= n <= the n_max the workspace was sized for
+ *   d_in       d_in % 8 == 0, 8 <= d_in <= 65536
+ *   s          fp32 [g, ld_s], s >= 0 (as produced by gq_saliency), ld_s >= n
+ *   H          fp32 [g, d_in, d_in] row-major, 16-byte aligned.  The caller zeroes it before the
+ *              first chunk and keeps it resident between chunks.  After any number of calls only
+ *              entries with a <= b are defined; entries below the diagonal hold unspecified finite
+ *              values until gq_hessian_finalize() is called.
+ *   flags      must be 0
+ *   workspace  device scratch of at least gq_hessian_workspace_bytes(n_max, d_in, g, flags)
+ *              bytes, 1024-byte aligned; contents need not be preserved between calls.
+ * Arithmetic: rows of X are multiplied by s_k in fp32 and rounded to bf16 once; products are
+ * accumulated in fp32 on the tensor cores; each call adds its fp32 tile sums to H.  Every element
+ * of H has a single writer, so results are bit-reproducible run to run.
+ */
+int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld_x, const float *s,
+                              int64_t ld_s, int32_t g, float *H, uint32_t flags, void *workspace,
+                              size_t workspace_bytes, void *stream);
+
+/* Scratch bytes gq_hessian_accumulate needs for chunks of up to n_max tokens (0 on bad arguments). */
+size_t gq_hessian_workspace_bytes(int64_t n_max, int64_t d_in, int32_t g, uint32_t flags);
+
+/*
+ * Completes H after the last chunk: copies the upper triangle onto the lower one,
+ * H[k][b][a] = H[k][a][b] for a < b, so that every H_k is a full, exactly symmetric matrix
+ * (H_k is symmetric by definition: Section 3.2).  Idempotent.
+ */
+int32_t gq_hessian_finalize(float *H, int64_t d_in, int32_t g, void *stream);
+
+/*
+ * Objective, Eq. 7:
+ *     loss_out[k] = sum_{j in J_k} (w_j - what_j)^T H_k (w_j - what_j),  k < g
+ *     loss_out[g] = sum_k loss_out[k]
+ *
+ *   W, W_hat   fp32 [d_out, d_in] row-major, 16-byte aligned (row j = output channel j)
+ *   H          fp32 [g, d_in, d_in] as left by gq_hessian_accumulate or gq_hessian_finalize:
+ *              only entries with a <= b are read
+ *   loss_out   fp64 [g + 1] in device memory
+ *   workspace  device scratch of at least gq_objective_workspace_bytes(d_in, d_out, g) bytes,
+ *              1024-byte aligned
+ * Same shape rules as above (d_in % 8 == 0, d_out % g == 0, (d_out / g) % 8 == 0).
+ * Arithmetic: delta = W - W_hat in fp32, split into two bf16 terms (delta = hi + lo to ~2^-17);
+ * the Gram matrices Delta_k^T Delta_k are formed on the tensor cores with fp32 accumulation and
+ * contracted with H_k in the same kernel; partial sums are reduced in fp64 in a fixed order.
+ */
+int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d_out, const float *H,
+                     int32_t g, double *loss_out, void *workspace, size_t workspace_bytes,
+                     void *stream);
+
+size_t gq_objective_workspace_bytes(int64_t d_in, int64_t d_out, int32_t g);
+
+/*
+ * The whole path for one layer with HOST inputs and outputs (Algorithm 1 lines 1, 2, 4 and Eq. 7):
+ * streams X and dl/dZ from host memory in chunks of `chunk` tokens, builds s and H on the device,
+ * finalizes H, evaluates the objective and copies the results back.
+ *
+ *   X_host, grad_host   HOST bf16 [n, d_in] / [n, d_out], densely packed (pinned memory makes
+ *                       the copies asynchronous; pageable memory also works)
+ *   W_host, W_hat_host  HOST fp32 [d_out, d_in]
+ *   loss_host           HOST fp64 [g + 1], written before the call returns
+ *   H_host              HOST fp32 [g, d_in, d_in] or NULL to skip copying H back
+ *   arena, arena_bytes  DEVICE scratch of at least gq_layer_host_arena_bytes(...) bytes,
+ *                       1024-byte aligned; it holds the chunk buffers, s, H and the workspaces
+ * The call synchronises `stream` before returning (it is the only call that does) and also
+ * returns device-side errors (as gq_check would).
+ */
+int32_t gq_layer_objective_host(const void *X_host, const void *grad_host, int64_t n, int64_t chunk,
+                                int64_t d_in, int64_t d_out, int32_t g, float grad_scale,
+                                const float *W_host, const float *W_hat_host, double *loss_host,
+                                float *H_host, void *arena, size_t arena_bytes, void *stream);
+
+size_t gq_layer_host_arena_bytes(int64_t chunk, int64_t d_in, int64_t d_out, int32_t g);
+
+/*
+ * Synchronises `stream`, then returns and clears the first device-side error recorded on the
+ * current device since the last gq_check (GQ_OK if none).  A pipeline wait inside a kernel that
+ * exceeds its time budget (2 s by default; environment variable GQ_WAIT_BUDGET_MS) makes the
+ * kernel stop early, leave its outputs incomplete and record GQ_ERR_TIMEOUT here.
+ * If `detail` is not NULL it receives 4 words: {status, site id, block index, work-unit index}.
+ */
+int32_t gq_check(void *stream, uint32_t *detail /* HOST, may be NULL */);
+
+/* Number of kernels this library has launched from the calling process (for bookkeeping). */
+uint64_t gq_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GQ_H_ */

@@ -40,6 +40,7 @@ int gq_oracle_saliency(const uint16_t *grad, int64_t n, int64_t d_out, int64_t l
     if (g < 1 || d_out < 1 || d_out % g != 0 || ld_grad < d_out || ld_s < n) return -1;
     const int64_t m = d_out / g;
     for (int32_t k = 0; k < g; ++k) {
+#pragma omp parallel for schedule(static)
         for (int64_t i = 0; i < n; ++i) {
             double acc = 0.0;
             for (int64_t j = m * k; j < m * (k + 1); ++j) {

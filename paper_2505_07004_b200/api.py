@@ -1,0 +1,231 @@
+"""ctypes binding of the C-ABI library ``libgq.so`` (declared in ``include/gq.h``).
+
+Argument marshalling only: every function here checks dtypes/devices, passes raw
+device pointers and the current CUDA stream to the entry point of the same name,
+and raises :class:`GQError` on a non-zero status.  PyTorch is used for device
+memory and streams; no arithmetic of the method runs in Python and there is no
+CPU fallback: if ``libgq.so`` is missing or no CUDA device is present the calls fail.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgq.so")
+_lib = None
+
+EXPORTS = (
+    "gq_version", "gq_status_string", "gq_last_cuda_error", "gq_saliency", "gq_hessian_accumulate",
+    "gq_hessian_workspace_bytes", "gq_hessian_finalize", "gq_objective", "gq_objective_workspace_bytes",
+    "gq_layer_objective_host", "gq_layer_host_arena_bytes", "gq_check", "gq_launch_count",
+)
+
+
+class GQError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        self.status = status
+        name = lib().gq_status_string(status).decode()
+        extra = ""
+        if name == "GQ_ERR_CUDA":
+            extra = " (cudaError %d)" % lib().gq_last_cuda_error()
+        super().__init__("%s failed: %s%s" % (fn, name, extra))
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the in-tree ``libgq.so``; fails loudly if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "libgq.so not found at %s: build it with `python -m paper_2505_07004_b200.build` "
+                "(there is no CPU fallback)" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        i64, i32, u32, f32, vp, sz = (ctypes.c_int64, ctypes.c_int32, ctypes.c_uint32, ctypes.c_float,
+                                      ctypes.c_void_p, ctypes.c_size_t)
+        L.gq_version.restype = ctypes.c_int
+        L.gq_status_string.restype = ctypes.c_char_p
+        L.gq_status_string.argtypes = [i32]
+        L.gq_last_cuda_error.restype = i32
+        L.gq_launch_count.restype = ctypes.c_uint64
+        L.gq_saliency.restype = i32
+        L.gq_saliency.argtypes = [vp, i64, i64, i64, i32, f32, vp, i64, vp]
+        L.gq_hessian_workspace_bytes.restype = sz
+        L.gq_hessian_workspace_bytes.argtypes = [i64, i64, i32, u32]
+        L.gq_hessian_accumulate.restype = i32
+        L.gq_hessian_accumulate.argtypes = [vp, i64, i64, i64, vp, i64, i32, vp, u32, vp, sz, vp]
+        L.gq_hessian_finalize.restype = i32
+        L.gq_hessian_finalize.argtypes = [vp, i64, i32, vp]
+        L.gq_objective_workspace_bytes.restype = sz
+        L.gq_objective_workspace_bytes.argtypes = [i64, i64, i32]
+        L.gq_objective.restype = i32
+        L.gq_objective.argtypes = [vp, vp, i64, i64, vp, i32, vp, vp, sz, vp]
+        L.gq_layer_host_arena_bytes.restype = sz
+        L.gq_layer_host_arena_bytes.argtypes = [i64, i64, i64, i32]
+        L.gq_layer_objective_host.restype = i32
+        L.gq_layer_objective_host.argtypes = [vp, vp, i64, i64, i64, i64, i32, f32, vp, vp, vp, vp, vp, sz, vp]
+        L.gq_check.restype = i32
+        L.gq_check.argtypes = [vp, vp]
+        _lib = L
+    return _lib
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    st = stream if stream is not None else torch.cuda.current_stream()
+    return int(st.cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
+    if not t.is_cuda:
+        raise ValueError("%s must be a CUDA tensor" % name)
+    if t.dtype != dtype:
+        raise ValueError("%s must be %s" % (name, dtype))
+    return t
+
+
+def _rows(t: torch.Tensor, name: str):
+    """(n, width, leading dimension) of a 2-D tensor whose last dimension is contiguous."""
+    if t.dim() != 2 or (t.shape[1] > 1 and t.stride(1) != 1):
+        raise ValueError("%s must be 2-D with a contiguous last dimension" % name)
+    return t.shape[0], t.shape[1], (t.stride(0) if t.shape[0] > 1 else max(t.shape[1], t.stride(0)))
+
+
+def alloc_workspace(nbytes: int, device) -> torch.Tensor:
+    """Device scratch of ``nbytes`` bytes whose base is 1024-byte aligned."""
+    buf = torch.empty(int(nbytes) + 1024, dtype=torch.uint8, device=device)
+    off = (-buf.data_ptr()) % 1024
+    return buf[off:off + int(nbytes)]
+
+
+def gq_version() -> int:
+    return int(lib().gq_version())
+
+
+def gq_launch_count() -> int:
+    return int(lib().gq_launch_count())
+
+
+def gq_saliency(grad: torch.Tensor, g: int, grad_scale: float = 1.0, s: Optional[torch.Tensor] = None,
+                stream=None) -> torch.Tensor:
+    """``s[k, i] = grad_scale**2 / m * sum_{j in J_k} grad[i, j]**2`` (Algorithm 1, line 2)."""
+    _dev(grad, torch.bfloat16, "grad")
+    n, d_out, ld = _rows(grad, "grad")
+    if s is None:
+        s = torch.empty((g, n), dtype=torch.float32, device=grad.device)
+    _dev(s, torch.float32, "s")
+    _, s_n, ld_s = _rows(s, "s")
+    if s.shape[0] != g or s_n < n:
+        raise ValueError("s must be [g, >= n]")
+    rc = lib().gq_saliency(grad.data_ptr(), n, d_out, ld, g, float(grad_scale), s.data_ptr(), ld_s,
+                           _stream_ptr(stream))
+    if rc:
+        raise GQError("gq_saliency", rc)
+    return s
+
+
+def gq_hessian_workspace_bytes(n_max: int, d_in: int, g: int, flags: int = 0) -> int:
+    return int(lib().gq_hessian_workspace_bytes(n_max, d_in, g, flags))
+
+
+def gq_hessian_accumulate(X: torch.Tensor, s: torch.Tensor, H: torch.Tensor, workspace: torch.Tensor,
+                          flags: int = 0, stream=None) -> torch.Tensor:
+    """``H[k] += X^T Diag(s[k]) X`` on the upper triangle (Algorithm 1, line 4), one token chunk."""
+    _dev(X, torch.bfloat16, "X")
+    _dev(s, torch.float32, "s")
+    _dev(H, torch.float32, "H")
+    n, d_in, ld_x = _rows(X, "X")
+    g, s_n, ld_s = _rows(s, "s")
+    if s_n < n:
+        raise ValueError("s must be [g, >= n]")
+    s_n = n
+    if tuple(H.shape) != (g, d_in, d_in) or not H.is_contiguous():
+        raise ValueError("H must be a contiguous [g, d_in, d_in] tensor")
+    rc = lib().gq_hessian_accumulate(X.data_ptr(), n, d_in, ld_x, s.data_ptr(), ld_s, g, H.data_ptr(), flags,
+                                     workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                     _stream_ptr(stream))
+    if rc:
+        raise GQError("gq_hessian_accumulate", rc)
+    return H
+
+
+def gq_hessian_finalize(H: torch.Tensor, stream=None) -> torch.Tensor:
+    """Mirror the upper triangle of every ``H[k]`` onto the lower one."""
+    _dev(H, torch.float32, "H")
+    if H.dim() != 3 or H.shape[1] != H.shape[2] or not H.is_contiguous():
+        raise ValueError("H must be a contiguous [g, d_in, d_in] tensor")
+    rc = lib().gq_hessian_finalize(H.data_ptr(), H.shape[1], H.shape[0], _stream_ptr(stream))
+    if rc:
+        raise GQError("gq_hessian_finalize", rc)
+    return H
+
+
+def gq_objective_workspace_bytes(d_in: int, d_out: int, g: int) -> int:
+    return int(lib().gq_objective_workspace_bytes(d_in, d_out, g))
+
+
+def gq_objective(W: torch.Tensor, W_hat: torch.Tensor, H: torch.Tensor, workspace: torch.Tensor,
+                 loss: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Eq. 7: returns fp64 ``[g + 1]`` = per-group losses followed by their total (device tensor)."""
+    _dev(W, torch.float32, "W")
+    _dev(W_hat, torch.float32, "W_hat")
+    _dev(H, torch.float32, "H")
+    if W.dim() != 2 or W.shape != W_hat.shape or not W.is_contiguous() or not W_hat.is_contiguous():
+        raise ValueError("W and W_hat must be contiguous [d_out, d_in]")
+    d_out, d_in = W.shape
+    g = H.shape[0]
+    if tuple(H.shape) != (g, d_in, d_in) or not H.is_contiguous():
+        raise ValueError("H must be a contiguous [g, d_in, d_in] tensor")
+    if loss is None:
+        loss = torch.empty(g + 1, dtype=torch.float64, device=W.device)
+    _dev(loss, torch.float64, "loss")
+    rc = lib().gq_objective(W.data_ptr(), W_hat.data_ptr(), d_in, d_out, H.data_ptr(), g, loss.data_ptr(),
+                            workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc:
+        raise GQError("gq_objective", rc)
+    return loss
+
+
+def gq_layer_host_arena_bytes(chunk: int, d_in: int, d_out: int, g: int) -> int:
+    return int(lib().gq_layer_host_arena_bytes(chunk, d_in, d_out, g))
+
+
+def gq_layer_objective_host(X_host: torch.Tensor, grad_host: torch.Tensor, chunk: int, g: int, grad_scale: float,
+                            W_host: torch.Tensor, W_hat_host: torch.Tensor, arena: torch.Tensor,
+                            loss_host: Optional[torch.Tensor] = None, H_host: Optional[torch.Tensor] = None,
+                            stream=None) -> torch.Tensor:
+    """Whole path from HOST tensors (ideally pinned): returns the host fp64 ``[g + 1]`` losses."""
+    for t, dt, nm in ((X_host, torch.bfloat16, "X_host"), (grad_host, torch.bfloat16, "grad_host"),
+                      (W_host, torch.float32, "W_host"), (W_hat_host, torch.float32, "W_hat_host")):
+        if t.is_cuda or t.dtype != dt or not t.is_contiguous():
+            raise ValueError("%s must be a contiguous host tensor of dtype %s" % (nm, dt))
+    n, d_in = X_host.shape
+    d_out = grad_host.shape[1]
+    if grad_host.shape[0] != n or tuple(W_host.shape) != (d_out, d_in) or W_hat_host.shape != W_host.shape:
+        raise ValueError("shape mismatch")
+    if loss_host is None:
+        loss_host = torch.empty(g + 1, dtype=torch.float64)
+    if H_host is not None and (H_host.is_cuda or H_host.dtype != torch.float32 or not H_host.is_contiguous()
+                               or tuple(H_host.shape) != (g, d_in, d_in)):
+        raise ValueError("H_host must be a contiguous host fp32 [g, d_in, d_in] tensor")
+    if not arena.is_cuda:
+        raise ValueError("arena must be device memory")
+    rc = lib().gq_layer_objective_host(X_host.data_ptr(), grad_host.data_ptr(), n, chunk, d_in, d_out, g,
+                                       float(grad_scale), W_host.data_ptr(), W_hat_host.data_ptr(),
+                                       loss_host.data_ptr(), H_host.data_ptr() if H_host is not None else None,
+                                       arena.data_ptr(), arena.numel() * arena.element_size(), _stream_ptr(stream))
+    if rc:
+        raise GQError("gq_layer_objective_host", rc)
+    return loss_host
+
+
+def gq_check(stream=None):
+    """Synchronises the stream and raises :class:`GQError` if a kernel recorded a device-side error."""
+    detail = (ctypes.c_uint32 * 4)()
+    rc = lib().gq_check(_stream_ptr(stream), detail)
+    if rc:
+        err = GQError("gq_check", rc)
+        err.detail = tuple(int(v) for v in detail)
+        raise err

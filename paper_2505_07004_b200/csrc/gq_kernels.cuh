@@ -1,0 +1,180 @@
+// Bandwidth-bound kernels of libgq: saliency reduction, row scaling, mirror, weight-error split,
+// final fp64 reduction.  All use 128-bit accesses and grid-stride loops over a grid sized from the
+// SM count.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace gq {
+
+__device__ __forceinline__ void bf16x8_to_float(const uint4 &v, float (&f)[8])
+{
+    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&v);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const float2 t = __bfloat1622float2(h[e]);
+        f[2 * e] = t.x;
+        f[2 * e + 1] = t.y;
+    }
+}
+
+__device__ __forceinline__ uint4 float_to_bf16x8(const float (&f)[8])
+{
+    uint4 v;
+    __nv_bfloat162 *h = reinterpret_cast<__nv_bfloat162 *>(&v);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) h[e] = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
+    return v;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Algorithm 1 line 2.  One warp per (token, group) segment of m = d_out / g gradients:
+//   s[k][i] = (grad_scale^2 / m) * sum_j grad[i][m k + j]^2.
+// A lane reads 16 bytes (8 bf16) per step, four steps are kept in flight; the lane-to-element
+// assignment and the butterfly reduction are fixed, so the result does not depend on the grid.
+__global__ void __launch_bounds__(256)
+saliency_kernel(const __nv_bfloat16 *__restrict__ grad, long long n, int m, long long ld_grad, int g, float coef,
+                float *__restrict__ s, long long ld_s)
+{
+    const int lane = threadIdx.x & 31;
+    const long long warp0 = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    const long long nwarps = (static_cast<long long>(gridDim.x) * blockDim.x) >> 5;
+    const long long segments = n * g;
+    const int vecs = m >> 3;                             // 16-byte vectors per segment
+    for (long long seg = warp0; seg < segments; seg += nwarps) {
+        const long long i = seg / g;
+        const int k = static_cast<int>(seg - i * g);
+        const uint4 *src = reinterpret_cast<const uint4 *>(grad + i * ld_grad + static_cast<long long>(k) * m);
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        int v = lane;
+        for (; v + 96 < vecs; v += 128) {
+            uint4 x[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) x[t] = __ldcs(src + v + 32 * t);
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                float f[8];
+                bf16x8_to_float(x[t], f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[t] = fmaf(f[e], f[e], acc[t]);
+            }
+        }
+        for (int t = 0; v < vecs; v += 32, ++t) {
+            float f[8];
+            bf16x8_to_float(__ldcs(src + v), f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[t & 3] = fmaf(f[e], f[e], acc[t & 3]);
+        }
+        float sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+        if (lane == 0) s[static_cast<long long>(k) * ld_s + i] = sum * coef;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Row scaling for Algorithm 1 line 4:  Y[k][i][a] = bf16( s[k][i] * X[i][a] ), so that
+// H_k = X^T Diag(s_k) X = X^T Y_k.  One thread handles 8 features of one token for all groups.
+__global__ void __launch_bounds__(256)
+scale_rows_kernel(const __nv_bfloat16 *__restrict__ X, long long n, int d, long long ld_x, const float *__restrict__ s,
+                  long long ld_s, int g, __nv_bfloat16 *__restrict__ Y)
+{
+    const int vec_per_row = d >> 3;
+    const long long total = n * vec_per_row;
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    const long long group_stride = n * static_cast<long long>(d);
+    for (long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total; idx += stride) {
+        const long long i = idx / vec_per_row;
+        const int a = static_cast<int>(idx - i * vec_per_row) << 3;
+        float x[8];
+        bf16x8_to_float(__ldg(reinterpret_cast<const uint4 *>(X + i * ld_x + a)), x);
+        for (int k = 0; k < g; ++k) {
+            const float sk = __ldg(s + static_cast<long long>(k) * ld_s + i);
+            float y[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) y[e] = sk * x[e];
+            *reinterpret_cast<uint4 *>(Y + k * group_stride + i * d + a) = float_to_bf16x8(y);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// H[k][b][a] = H[k][a][b] for a < b (H_k is symmetric by definition, Section 3.2).
+// blockIdx.x / .y = 32 x 32 block column / row, blockIdx.z = group; blocks below the diagonal exit.
+__global__ void __launch_bounds__(256)
+mirror_kernel(float *__restrict__ H, int d)
+{
+    const int bj = blockIdx.x, bi = blockIdx.y;
+    if (bi > bj) return;
+    __shared__ float tile[32][33];
+    float *Hk = H + static_cast<size_t>(blockIdx.z) * d * d;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;    // 32 x 8 threads
+#pragma unroll
+    for (int r = ty; r < 32; r += 8) {
+        const int a = bi * 32 + r, b = bj * 32 + tx;
+        tile[r][tx] = (a < d && b < d) ? Hk[static_cast<size_t>(a) * d + b] : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = ty; r < 32; r += 8) {
+        const int b = bj * 32 + r, a = bi * 32 + tx;          // write H[b][a] = tile[a - bi*32][b - bj*32]
+        if (a < d && b < d && a < b) Hk[static_cast<size_t>(b) * d + a] = tile[tx][r];
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Weight error of Eq. 7, delta = W - W_hat in fp32, split into bf16 hi + bf16 lo
+// (hi = bf16(delta), lo = bf16(delta - hi)); |delta - hi - lo| <= 2^-17 |delta|.
+__global__ void __launch_bounds__(256)
+split_delta_kernel(const float *__restrict__ W, const float *__restrict__ What, long long count8,
+                   __nv_bfloat16 *__restrict__ hi, __nv_bfloat16 *__restrict__ lo)
+{
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; idx < count8; idx += stride) {
+        const float4 *w = reinterpret_cast<const float4 *>(W) + idx * 2;
+        const float4 *q = reinterpret_cast<const float4 *>(What) + idx * 2;
+        const float4 w0 = __ldcs(w), w1 = __ldcs(w + 1), q0 = __ldcs(q), q1 = __ldcs(q + 1);
+        const float dlt[8] = {w0.x - q0.x, w0.y - q0.y, w0.z - q0.z, w0.w - q0.w,
+                              w1.x - q1.x, w1.y - q1.y, w1.z - q1.z, w1.w - q1.w};
+        float h[8], l[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            h[e] = __bfloat162float(__float2bfloat16_rn(dlt[e]));
+            l[e] = dlt[e] - h[e];
+        }
+        reinterpret_cast<uint4 *>(hi)[idx] = float_to_bf16x8(h);
+        reinterpret_cast<uint4 *>(lo)[idx] = float_to_bf16x8(l);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// loss[k] = sum over the group's tile partials (fixed order), loss[g] = sum_k loss[k].  One block.
+// partials: [tile_slots][g][4].
+__global__ void __launch_bounds__(1024)
+reduce_partials_kernel(const double *__restrict__ partials, int tile_slots, int g, double *__restrict__ loss)
+{
+    __shared__ double red[1024];
+    double total = 0.0;
+    for (int k = 0; k < g; ++k) {
+        double acc = 0.0;
+        for (int idx = threadIdx.x; idx < tile_slots * 4; idx += blockDim.x) {
+            const int t = idx >> 2, q = idx & 3;
+            acc += partials[(static_cast<size_t>(t) * g + k) * 4 + q];
+        }
+        red[threadIdx.x] = acc;
+        __syncthreads();
+        for (int off = blockDim.x >> 1; off > 0; off >>= 1) {
+            if (static_cast<int>(threadIdx.x) < off) red[threadIdx.x] += red[threadIdx.x + off];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) {
+            loss[k] = red[0];
+            total += red[0];
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) loss[g] = total;
+}
+
+}  // namespace gq

@@ -1,0 +1,449 @@
+// libgq C-ABI (see include/gq.h): argument validation, tensor maps, launches.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "../../include/gq.h"
+#include "gq_gram.cuh"
+#include "gq_kernels.cuh"
+
+#define GQ_VERSION_NUMBER 100   /* 0.1.0 */
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+
+thread_local int32_t tl_last_cuda_error = 0;
+std::atomic<uint64_t> g_launches{0};
+
+// Per-device status word {status, site, block, unit}; written by kernels, read by gq_check().
+__device__ uint32_t g_status_word[4];
+
+struct DeviceInfo {
+    bool ready = false;
+    int sm_count = 0;
+    uint32_t *status_ptr = nullptr;
+};
+DeviceInfo g_dev[kMaxDevices];
+std::mutex g_dev_mutex;
+PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
+
+#define GQ_CUDA(call)                                   \
+    do {                                                \
+        cudaError_t e_ = (call);                        \
+        if (e_ != cudaSuccess) {                        \
+            tl_last_cuda_error = static_cast<int32_t>(e_); \
+            return GQ_ERR_CUDA;                         \
+        }                                               \
+    } while (0)
+
+inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int32_t device_info(DeviceInfo **out)
+{
+    int dev = 0;
+    GQ_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return GQ_ERR_UNSUPPORTED_SHAPE;
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    DeviceInfo &di = g_dev[dev];
+    if (!di.ready) {
+        GQ_CUDA(cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev));
+        void *sym = nullptr;
+        GQ_CUDA(cudaGetSymbolAddress(&sym, g_status_word));
+        di.status_ptr = static_cast<uint32_t *>(sym);
+        GQ_CUDA(cudaFuncSetAttribute(gq::gram_kernel<gq::EPI_ACCUM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     gq::GRAM_SMEM_BYTES));
+        GQ_CUDA(cudaFuncSetAttribute(gq::gram_kernel<gq::EPI_DOT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     gq::GRAM_SMEM_BYTES));
+        if (!g_encode) {
+            void *fn = nullptr;
+            cudaDriverEntryPointQueryResult qres;
+            GQ_CUDA(cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres));
+            if (qres != cudaDriverEntryPointSuccess || !fn) {
+                tl_last_cuda_error = static_cast<int32_t>(cudaErrorNotSupported);
+                return GQ_ERR_CUDA;
+            }
+            g_encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+        }
+        di.ready = true;
+    }
+    *out = &di;
+    return GQ_OK;
+}
+
+unsigned long long wait_budget_ns()
+{
+    static const unsigned long long v = [] {
+        const char *e = std::getenv("GQ_WAIT_BUDGET_MS");
+        long ms = e ? std::atol(e) : 2000;
+        if (ms < 1) ms = 1;
+        if (ms > 60000) ms = 60000;
+        return static_cast<unsigned long long>(ms) * 1000000ull;
+    }();
+    return v;
+}
+
+// bf16 tensor [groups][rows][features] (row stride ld, group stride gstride, in elements) as a TMA map
+// with 64-feature x 64-row boxes and the 128-byte swizzle.
+int32_t make_map(CUtensorMap *map, const void *base, int64_t features, int64_t rows, int64_t groups, int64_t ld,
+                 int64_t gstride)
+{
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(features), static_cast<cuuint64_t>(rows),
+                          static_cast<cuuint64_t>(groups)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(ld) * 2, static_cast<cuuint64_t>(gstride) * 2};
+    cuuint32_t box[3] = {gq::BOX_FEATURES, gq::TILE_K, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        tl_last_cuda_error = static_cast<int32_t>(cudaErrorInvalidValue);
+        return GQ_ERR_CUDA;
+    }
+    return GQ_OK;
+}
+
+int grid_for(long long work_items, int threads, int sm_count, int blocks_per_sm)
+{
+    long long blocks = (work_items + threads - 1) / threads;
+    const long long cap = static_cast<long long>(sm_count) * blocks_per_sm;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return static_cast<int>(blocks);
+}
+
+int tile_slots_for(int64_t d)
+{
+    const int64_t nj = (d + gq::TILE_N - 1) / gq::TILE_N;
+    return static_cast<int>(nj * nj + nj);
+}
+
+int32_t check_layer_shape(int64_t d_in, int64_t d_out, int32_t g, bool need_out)
+{
+    if (g < 1 || d_in < 1) return GQ_ERR_INVALID_ARG;
+    if (d_in % 8 != 0 || d_in < 8 || d_in > 65536 || g > 1024) return GQ_ERR_UNSUPPORTED_SHAPE;
+    if (need_out) {
+        if (d_out < 1 || d_out % g != 0) return GQ_ERR_INVALID_ARG;
+        if ((d_out / g) % 8 != 0 || d_out > (1ll << 24)) return GQ_ERR_UNSUPPORTED_SHAPE;
+    }
+    return GQ_OK;
+}
+
+size_t hessian_ws_bytes(int64_t n_max, int64_t d_in, int32_t g)
+{
+    return round_up(static_cast<size_t>(g) * static_cast<size_t>(n_max) * static_cast<size_t>(d_in) * 2, 1024);
+}
+
+struct ObjectiveLayout {
+    size_t hi_off, lo_off, partials_off, total;
+};
+ObjectiveLayout objective_layout(int64_t d_in, int64_t d_out, int32_t g)
+{
+    ObjectiveLayout L;
+    const size_t mat = round_up(static_cast<size_t>(d_in) * static_cast<size_t>(d_out) * 2, 1024);
+    L.hi_off = 0;
+    L.lo_off = mat;
+    L.partials_off = 2 * mat;
+    L.total = L.partials_off + round_up(static_cast<size_t>(tile_slots_for(d_in)) * g * 4 * sizeof(double), 1024);
+    return L;
+}
+
+}  // namespace
+
+extern "C" {
+
+int gq_version(void) { return GQ_VERSION_NUMBER; }
+
+const char *gq_status_string(int32_t status)
+{
+    switch (status) {
+    case GQ_OK: return "GQ_OK";
+    case GQ_ERR_INVALID_ARG: return "GQ_ERR_INVALID_ARG";
+    case GQ_ERR_ALIGNMENT: return "GQ_ERR_ALIGNMENT";
+    case GQ_ERR_UNSUPPORTED_SHAPE: return "GQ_ERR_UNSUPPORTED_SHAPE";
+    case GQ_ERR_WORKSPACE: return "GQ_ERR_WORKSPACE";
+    case GQ_ERR_CUDA: return "GQ_ERR_CUDA";
+    case GQ_ERR_TIMEOUT: return "GQ_ERR_TIMEOUT";
+    default: return "GQ_ERR_UNKNOWN";
+    }
+}
+
+int32_t gq_last_cuda_error(void) { return tl_last_cuda_error; }
+
+uint64_t gq_launch_count(void) { return g_launches.load(); }
+
+int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad, int32_t g, float grad_scale,
+                    float *s, int64_t ld_s, void *stream)
+{
+    if (!grad || !s || n < 0 || g < 1 || d_out < 1 || d_out % g != 0 || ld_grad < d_out || ld_s < n ||
+        !(grad_scale == grad_scale) || grad_scale - grad_scale != 0.0f)
+        return GQ_ERR_INVALID_ARG;
+    if ((d_out / g) % 8 != 0 || g > 1024 || d_out > (1ll << 24) || n > (1ll << 40)) return GQ_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned(grad, 16) || ld_grad % 8 != 0 || !aligned(s, 4)) return GQ_ERR_ALIGNMENT;
+    if (n == 0) return GQ_OK;
+    DeviceInfo *di;
+    if (int32_t rc = device_info(&di)) return rc;
+    const int m = static_cast<int>(d_out / g);
+    const float coef = grad_scale * grad_scale / static_cast<float>(m);
+    const int grid = grid_for(n * g * 32, 256, di->sm_count, 8);
+    gq::saliency_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const __nv_bfloat16 *>(grad), n, m, ld_grad, g, coef, s, ld_s);
+    g_launches.fetch_add(1);
+    GQ_CUDA(cudaGetLastError());
+    return GQ_OK;
+}
+
+size_t gq_hessian_workspace_bytes(int64_t n_max, int64_t d_in, int32_t g, uint32_t flags)
+{
+    if (flags != 0 || n_max < 0 || check_layer_shape(d_in, 0, g, false) != GQ_OK) return 0;
+    return hessian_ws_bytes(n_max, d_in, g);
+}
+
+int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld_x, const float *s, int64_t ld_s,
+                              int32_t g, float *H, uint32_t flags, void *workspace, size_t workspace_bytes,
+                              void *stream)
+{
+    if (!X || !s || !H || n < 0 || ld_x < d_in || ld_s < n || flags != 0) return GQ_ERR_INVALID_ARG;
+    if (int32_t rc = check_layer_shape(d_in, 0, g, false)) return rc;
+    if (n > (1ll << 31) - 64) return GQ_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned(X, 16) || ld_x % 8 != 0 || !aligned(H, 16) || !aligned(s, 4)) return GQ_ERR_ALIGNMENT;
+    if (n == 0) return GQ_OK;
+    if (!workspace || workspace_bytes < hessian_ws_bytes(n, d_in, g)) return GQ_ERR_WORKSPACE;
+    if (!aligned(workspace, 1024)) return GQ_ERR_ALIGNMENT;
+    DeviceInfo *di;
+    if (int32_t rc = device_info(&di)) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    __nv_bfloat16 *Y = static_cast<__nv_bfloat16 *>(workspace);
+
+    // Y_k = Diag(s_k) X rounded to bf16, so that H_k += X^T Y_k.
+    {
+        const int grid = grid_for(n * (d_in / 8), 256, di->sm_count, 8);
+        gq::scale_rows_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), n, static_cast<int>(d_in),
+                                                    ld_x, s, ld_s, g, Y);
+        g_launches.fetch_add(1);
+        GQ_CUDA(cudaGetLastError());
+    }
+    CUtensorMap mapX, mapY;
+    if (int32_t rc = make_map(&mapX, X, d_in, n, 1, ld_x, n * ld_x)) return rc;
+    if (int32_t rc = make_map(&mapY, Y, d_in, n, g, d_in, n * d_in)) return rc;
+    gq::GramParams p{};
+    p.d = static_cast<int>(d_in);
+    p.rows = static_cast<int>(n);
+    p.g = g;
+    p.n_terms = 1;
+    p.term_a[0] = 0;
+    p.term_b[0] = 1;
+    p.map_grouped[0] = 0;
+    p.map_grouped[1] = 1;
+    p.tile_slots = tile_slots_for(d_in);
+    p.units = p.tile_slots * g;
+    p.H = H;
+    p.partials = nullptr;
+    p.status = di->status_ptr;
+    p.wait_budget_ns = wait_budget_ns();
+    const int grid = p.units < di->sm_count ? p.units : di->sm_count;
+    gq::gram_kernel<gq::EPI_ACCUM><<<grid, gq::GRAM_THREADS, gq::GRAM_SMEM_BYTES, st>>>(mapX, mapY, p);
+    g_launches.fetch_add(1);
+    GQ_CUDA(cudaGetLastError());
+    return GQ_OK;
+}
+
+int32_t gq_hessian_finalize(float *H, int64_t d_in, int32_t g, void *stream)
+{
+    if (!H) return GQ_ERR_INVALID_ARG;
+    if (int32_t rc = check_layer_shape(d_in, 0, g, false)) return rc;
+    if (!aligned(H, 16)) return GQ_ERR_ALIGNMENT;
+    const unsigned nb = static_cast<unsigned>((d_in + 31) / 32);
+    dim3 grid(nb, nb, static_cast<unsigned>(g));
+    gq::mirror_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(H, static_cast<int>(d_in));
+    g_launches.fetch_add(1);
+    GQ_CUDA(cudaGetLastError());
+    return GQ_OK;
+}
+
+size_t gq_objective_workspace_bytes(int64_t d_in, int64_t d_out, int32_t g)
+{
+    if (check_layer_shape(d_in, d_out, g, true) != GQ_OK) return 0;
+    return objective_layout(d_in, d_out, g).total;
+}
+
+int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d_out, const float *H, int32_t g,
+                     double *loss_out, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!W || !W_hat || !H || !loss_out) return GQ_ERR_INVALID_ARG;
+    if (int32_t rc = check_layer_shape(d_in, d_out, g, true)) return rc;
+    if (!aligned(W, 16) || !aligned(W_hat, 16) || !aligned(H, 16) || !aligned(loss_out, 8)) return GQ_ERR_ALIGNMENT;
+    const ObjectiveLayout L = objective_layout(d_in, d_out, g);
+    if (!workspace || workspace_bytes < L.total) return GQ_ERR_WORKSPACE;
+    if (!aligned(workspace, 1024)) return GQ_ERR_ALIGNMENT;
+    DeviceInfo *di;
+    if (int32_t rc = device_info(&di)) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    __nv_bfloat16 *hi = reinterpret_cast<__nv_bfloat16 *>(ws + L.hi_off);
+    __nv_bfloat16 *lo = reinterpret_cast<__nv_bfloat16 *>(ws + L.lo_off);
+    double *partials = reinterpret_cast<double *>(ws + L.partials_off);
+    const int64_t m = d_out / g;
+    {
+        const long long count8 = d_in * d_out / 8;
+        const int grid = grid_for(count8, 256, di->sm_count, 8);
+        gq::split_delta_kernel<<<grid, 256, 0, st>>>(W, W_hat, count8, hi, lo);
+        g_launches.fetch_add(1);
+        GQ_CUDA(cudaGetLastError());
+    }
+    CUtensorMap mapHi, mapLo;
+    if (int32_t rc = make_map(&mapHi, hi, d_in, m, g, d_in, m * d_in)) return rc;
+    if (int32_t rc = make_map(&mapLo, lo, d_in, m, g, d_in, m * d_in)) return rc;
+    gq::GramParams p{};
+    p.d = static_cast<int>(d_in);
+    p.rows = static_cast<int>(m);
+    p.g = g;
+    p.n_terms = 3;                     // hi^T hi + hi^T lo + lo^T hi
+    p.term_a[0] = 0; p.term_b[0] = 0;
+    p.term_a[1] = 0; p.term_b[1] = 1;
+    p.term_a[2] = 1; p.term_b[2] = 0;
+    p.map_grouped[0] = 1;
+    p.map_grouped[1] = 1;
+    p.tile_slots = tile_slots_for(d_in);
+    p.units = p.tile_slots * g;
+    p.H = const_cast<float *>(H);
+    p.partials = partials;
+    p.status = di->status_ptr;
+    p.wait_budget_ns = wait_budget_ns();
+    const int grid = p.units < di->sm_count ? p.units : di->sm_count;
+    gq::gram_kernel<gq::EPI_DOT><<<grid, gq::GRAM_THREADS, gq::GRAM_SMEM_BYTES, st>>>(mapHi, mapLo, p);
+    g_launches.fetch_add(1);
+    GQ_CUDA(cudaGetLastError());
+    gq::reduce_partials_kernel<<<1, 1024, 0, st>>>(partials, p.tile_slots, g, loss_out);
+    g_launches.fetch_add(1);
+    GQ_CUDA(cudaGetLastError());
+    return GQ_OK;
+}
+
+int32_t gq_check(void *stream, uint32_t *detail)
+{
+    DeviceInfo *di;
+    if (int32_t rc = device_info(&di)) return rc;
+    GQ_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    uint32_t word[4] = {0, 0, 0, 0};
+    GQ_CUDA(cudaMemcpy(word, di->status_ptr, sizeof word, cudaMemcpyDeviceToHost));
+    if (detail) std::memcpy(detail, word, sizeof word);
+    if (word[0] == 0) return GQ_OK;
+    GQ_CUDA(cudaMemset(di->status_ptr, 0, sizeof word));
+    if (detail) detail[0] = static_cast<uint32_t>(GQ_ERR_TIMEOUT);
+    return word[0] == gq::STATUS_TIMEOUT ? GQ_ERR_TIMEOUT : GQ_ERR_CUDA;
+}
+
+size_t gq_layer_host_arena_bytes(int64_t chunk, int64_t d_in, int64_t d_out, int32_t g)
+{
+    if (chunk < 1 || check_layer_shape(d_in, d_out, g, true) != GQ_OK) return 0;
+    size_t total = 0;
+    total += 2 * round_up(static_cast<size_t>(chunk) * d_in * 2, 1024);      // X chunk, double buffered
+    total += 2 * round_up(static_cast<size_t>(chunk) * d_out * 2, 1024);     // grad chunk, double buffered
+    total += round_up(static_cast<size_t>(g) * chunk * 4, 1024);             // s
+    total += round_up(static_cast<size_t>(g) * d_in * d_in * 4, 1024);       // H
+    total += 2 * round_up(static_cast<size_t>(d_out) * d_in * 4, 1024);      // W, W_hat
+    total += 1024;                                                           // loss
+    total += hessian_ws_bytes(chunk, d_in, g);
+    total += objective_layout(d_in, d_out, g).total;
+    return total;
+}
+
+int32_t gq_layer_objective_host(const void *X_host, const void *grad_host, int64_t n, int64_t chunk, int64_t d_in,
+                                int64_t d_out, int32_t g, float grad_scale, const float *W_host,
+                                const float *W_hat_host, double *loss_host, float *H_host, void *arena,
+                                size_t arena_bytes, void *stream)
+{
+    if (!X_host || !grad_host || !W_host || !W_hat_host || !loss_host || n < 0 || chunk < 1)
+        return GQ_ERR_INVALID_ARG;
+    if (int32_t rc = check_layer_shape(d_in, d_out, g, true)) return rc;
+    const size_t need = gq_layer_host_arena_bytes(chunk, d_in, d_out, g);
+    if (!arena || arena_bytes < need) return GQ_ERR_WORKSPACE;
+    if (!aligned(arena, 1024)) return GQ_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    uint8_t *p = static_cast<uint8_t *>(arena);
+    auto take = [&p](size_t bytes) { uint8_t *q = p; p += round_up(bytes, 1024); return q; };
+    uint8_t *xbuf[2], *gbuf[2];
+    xbuf[0] = take(static_cast<size_t>(chunk) * d_in * 2);
+    xbuf[1] = take(static_cast<size_t>(chunk) * d_in * 2);
+    gbuf[0] = take(static_cast<size_t>(chunk) * d_out * 2);
+    gbuf[1] = take(static_cast<size_t>(chunk) * d_out * 2);
+    float *s = reinterpret_cast<float *>(take(static_cast<size_t>(g) * chunk * 4));
+    const size_t h_bytes = static_cast<size_t>(g) * d_in * d_in * 4;
+    float *H = reinterpret_cast<float *>(take(h_bytes));
+    const size_t w_bytes = static_cast<size_t>(d_out) * d_in * 4;
+    float *W = reinterpret_cast<float *>(take(w_bytes));
+    float *What = reinterpret_cast<float *>(take(w_bytes));
+    double *loss = reinterpret_cast<double *>(take(1024));
+    const size_t hws_bytes = hessian_ws_bytes(chunk, d_in, g);
+    void *hws = take(hws_bytes);
+    const size_t ows_bytes = objective_layout(d_in, d_out, g).total;
+    void *ows = take(ows_bytes);
+
+    // Copies run on a second stream so that chunk c+1 is in flight while chunk c is processed.
+    cudaStream_t copy_st = nullptr;
+    cudaEvent_t copied[2] = {nullptr, nullptr}, consumed[2] = {nullptr, nullptr}, start = nullptr;
+    int32_t rc = GQ_OK;
+    auto fail = [&rc](cudaError_t e) {
+        if (e != cudaSuccess && rc == GQ_OK) { tl_last_cuda_error = static_cast<int32_t>(e); rc = GQ_ERR_CUDA; }
+        return e != cudaSuccess;
+    };
+    fail(cudaStreamCreateWithFlags(&copy_st, cudaStreamNonBlocking));
+    for (int b = 0; b < 2 && rc == GQ_OK; ++b) {
+        fail(cudaEventCreateWithFlags(&copied[b], cudaEventDisableTiming));
+        fail(cudaEventCreateWithFlags(&consumed[b], cudaEventDisableTiming));
+    }
+    if (rc == GQ_OK) fail(cudaEventCreateWithFlags(&start, cudaEventDisableTiming));
+    if (rc == GQ_OK) {
+        fail(cudaEventRecord(start, st));              // the copy stream starts after prior work on `stream`
+        fail(cudaStreamWaitEvent(copy_st, start, 0));
+        fail(cudaMemsetAsync(H, 0, h_bytes, st));
+        fail(cudaMemcpyAsync(W, W_host, w_bytes, cudaMemcpyHostToDevice, st));
+        fail(cudaMemcpyAsync(What, W_hat_host, w_bytes, cudaMemcpyHostToDevice, st));
+    }
+    const int64_t n_chunks = (n + chunk - 1) / chunk;
+    for (int64_t c = 0; c < n_chunks && rc == GQ_OK; ++c) {
+        const int b = static_cast<int>(c & 1);
+        const int64_t tok0 = c * chunk;
+        const int64_t nt = (n - tok0 < chunk) ? (n - tok0) : chunk;
+        if (c >= 2) fail(cudaStreamWaitEvent(copy_st, consumed[b], 0));
+        fail(cudaMemcpyAsync(xbuf[b], static_cast<const uint8_t *>(X_host) + static_cast<size_t>(tok0) * d_in * 2,
+                             static_cast<size_t>(nt) * d_in * 2, cudaMemcpyHostToDevice, copy_st));
+        fail(cudaMemcpyAsync(gbuf[b], static_cast<const uint8_t *>(grad_host) + static_cast<size_t>(tok0) * d_out * 2,
+                             static_cast<size_t>(nt) * d_out * 2, cudaMemcpyHostToDevice, copy_st));
+        fail(cudaEventRecord(copied[b], copy_st));
+        fail(cudaStreamWaitEvent(st, copied[b], 0));
+        if (rc != GQ_OK) break;
+        rc = gq_saliency(gbuf[b], nt, d_out, d_out, g, grad_scale, s, chunk, st);
+        if (rc == GQ_OK) rc = gq_hessian_accumulate(xbuf[b], nt, d_in, d_in, s, chunk, g, H, 0, hws, hws_bytes, st);
+        if (rc == GQ_OK) fail(cudaEventRecord(consumed[b], st));
+    }
+    if (rc == GQ_OK) rc = gq_hessian_finalize(H, d_in, g, st);
+    if (rc == GQ_OK) rc = gq_objective(W, What, d_in, d_out, H, g, loss, ows, ows_bytes, st);
+    if (rc == GQ_OK) {
+        fail(cudaMemcpyAsync(loss_host, loss, sizeof(double) * (g + 1), cudaMemcpyDeviceToHost, st));
+        if (H_host) fail(cudaMemcpyAsync(H_host, H, h_bytes, cudaMemcpyDeviceToHost, st));
+    }
+    // Always drain both streams before their events and the copy stream are destroyed.
+    if (copy_st) cudaStreamSynchronize(copy_st);
+    const int32_t chk = gq_check(stream, nullptr);
+    if (rc == GQ_OK) rc = chk;
+    for (int b = 0; b < 2; ++b) {
+        if (copied[b]) cudaEventDestroy(copied[b]);
+        if (consumed[b]) cudaEventDestroy(consumed[b]);
+    }
+    if (start) cudaEventDestroy(start);
+    if (copy_st) cudaStreamDestroy(copy_st);
+    return rc;
+}
+
+}  // extern "C"

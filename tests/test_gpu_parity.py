@@ -1,0 +1,329 @@
+"""GPU parity: libgq (through the C-ABI binding) against the CPU fp64 oracle, same seeded inputs.
+
+Tolerances (stated by the benchmark spec for this path):
+  saliency   |s - s_o| <= 1e-4 * |s_o| per element (plus a floor of 1e-4 * max|s_o| * 1e-6 for zeros)
+  Hessian    ||H_k - H_k_o||_F <= 5e-3 ||H_k_o||_F   and   max|H_k - H_k_o| <= 1e-2 max|H_k_o|
+  objective  |loss - loss_o| <= 1e-3 |loss_o|
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gq_oracle as orc
+from paper_2505_07004_b200 import api as libgq
+from paper_2505_07004_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+S_RTOL, H_FRO, H_MAX, L_RTOL = 1e-4, 5e-3, 1e-2, 1e-3
+
+
+@pytest.fixture(scope="module")
+def dev():
+    assert torch.cuda.is_available()
+    torch.cuda.set_device(0)
+    return torch.device("cuda:0")
+
+
+def check_s(s_gpu, s_ref):
+    s_gpu = s_gpu.detach().cpu().numpy().astype(np.float64)
+    floor = 1e-10 * np.abs(s_ref).max()
+    assert np.all(np.abs(s_gpu - s_ref) <= S_RTOL * np.abs(s_ref) + floor), \
+        "saliency max rel err %.3e" % (np.abs(s_gpu - s_ref) / (np.abs(s_ref) + floor)).max()
+
+
+def check_H(H_gpu, H_ref, upper_only=False):
+    H_gpu = H_gpu.detach().cpu().numpy().astype(np.float64)
+    for k in range(H_ref.shape[0]):
+        a, b = H_gpu[k], H_ref[k]
+        if upper_only:
+            a, b = np.triu(a), np.triu(b)
+        fro = np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300)
+        mx = np.abs(a - b).max() / max(np.abs(b).max(), 1e-300)
+        assert fro <= H_FRO and mx <= H_MAX, "group %d: rel Frobenius %.3e, max-elem %.3e" % (k, fro, mx)
+
+
+def check_loss(loss_gpu, loss_ref):
+    loss_gpu = loss_gpu.detach().cpu().numpy()
+    assert np.all(np.isfinite(loss_gpu))
+    scale = np.maximum(np.abs(loss_ref), 1e-300)
+    assert np.all(np.abs(loss_gpu - loss_ref) <= L_RTOL * scale), \
+        "objective rel err %s" % (np.abs(loss_gpu - loss_ref) / scale)
+
+
+def gpu_hessian(X_chunks, s_chunks, d_in, g, dev, finalize=True):
+    H = torch.zeros((g, d_in, d_in), dtype=torch.float32, device=dev)
+    n_max = max([x.shape[0] for x in X_chunks] + [1])
+    ws = libgq.alloc_workspace(libgq.gq_hessian_workspace_bytes(n_max, d_in, g), dev)
+    for x, s in zip(X_chunks, s_chunks):
+        libgq.gq_hessian_accumulate(x, s, H, ws)
+    if finalize:
+        libgq.gq_hessian_finalize(H)
+    libgq.gq_check()
+    return H
+
+
+# ------------------------------------------------------------------------------------------ saliency
+@pytest.mark.parametrize("n,d_out,g,pad,scale", [
+    (2048, 512, 4, 0, 1.0),       # tiny config
+    (1, 8, 1, 0, 1.0),            # one token, one vector
+    (333, 4096, 4, 0, 1.0),       # m = 1024: one full unrolled pass
+    (257, 11008, 16, 0, 1.0),     # m = 688: tail path only
+    (100, 2560, 2, 64, 1e3),      # m = 1280: unrolled pass + tail; padded rows; paper's scale
+    (65, 24, 3, 8, 1.0),          # m = 8
+])
+def test_saliency_parity(dev, n, d_out, g, pad, scale):
+    gen = torch.Generator(device=dev).manual_seed(n * 7 + d_out)
+    full = (torch.randn(n, d_out + pad, generator=gen, device=dev) * 1e-3).to(torch.bfloat16)
+    grad = full[:, :d_out]
+    s = libgq.gq_saliency(grad, g, scale)
+    libgq.gq_check()
+    s_ref = orc.saliency(synth.bf16_bits(grad.contiguous()), g, scale)
+    check_s(s, s_ref)
+
+
+def test_saliency_empty_and_errors(dev):
+    grad = torch.zeros((0, 64), dtype=torch.bfloat16, device=dev)
+    s = libgq.gq_saliency(grad, 2)
+    assert tuple(s.shape) == (2, 0)
+    grad = torch.zeros((4, 24), dtype=torch.bfloat16, device=dev)
+    with pytest.raises(libgq.GQError) as e:
+        libgq.gq_saliency(grad, 5)                      # 24 % 5 != 0
+    assert "GQ_ERR_INVALID_ARG" in str(e.value)
+    with pytest.raises(libgq.GQError) as e:
+        libgq.gq_saliency(grad, 6)                      # m = 4 is not a multiple of 8
+    assert "GQ_ERR_UNSUPPORTED_SHAPE" in str(e.value)
+    with pytest.raises(libgq.GQError) as e:
+        libgq.gq_saliency(grad, 1, float("nan"))
+    assert "GQ_ERR_INVALID_ARG" in str(e.value)
+
+
+# ------------------------------------------------------------------------------------------ Hessian
+@pytest.mark.parametrize("n,d_in,g,chunks", [
+    (2048, 256, 4, [2048]),                 # tiny config: one 128 x 256 tile per group
+    (677, 384, 2, [677]),                   # ragged K tail, d_in = 1.5 column blocks
+    (1, 8, 1, [1]),                         # smallest legal problem
+    (130, 520, 3, [64, 1, 65]),             # several chunks incl. a 1-token chunk; ragged tiles
+    (300, 1032, 2, [300]),                  # 5 column blocks, tail of 8 features
+    (96, 640, 5, [0, 96]),                  # an empty chunk is a no-op
+])
+def test_hessian_parity_small(dev, n, d_in, g, chunks):
+    gen = torch.Generator(device=dev).manual_seed(n + d_in)
+    feat = torch.exp(torch.randn(d_in, generator=gen, device=dev))
+    X = (torch.randn(n, d_in, generator=gen, device=dev) * feat).to(torch.bfloat16)
+    s = (torch.rand(g, n, generator=gen, device=dev) * torch.exp(torch.randn(1, n, generator=gen, device=dev)))
+    s = s.contiguous()
+    xs, ss, lo = [], [], 0
+    for c in chunks:
+        xs.append(X[lo:lo + c])
+        ss.append(s[:, lo:lo + c])
+        lo += c
+    assert lo == n
+    H = gpu_hessian(xs, ss, d_in, g, dev, finalize=False)
+    H_ref = orc.hessian(synth.bf16_bits(X), s.cpu().numpy().astype(np.float64))
+    check_H(H, H_ref, upper_only=True)
+    libgq.gq_hessian_finalize(H)
+    libgq.gq_check()
+    check_H(H, H_ref)
+    Hc = H.cpu()
+    assert torch.equal(Hc, Hc.transpose(1, 2)), "finalized H must be exactly symmetric"
+
+
+def test_hessian_unit_saliency_is_gram_and_deterministic(dev):
+    n, d_in = 500, 512
+    gen = torch.Generator(device=dev).manual_seed(3)
+    X = torch.randn(n, d_in, generator=gen, device=dev).to(torch.bfloat16)
+    s = torch.ones(1, n, device=dev)
+    H1 = gpu_hessian([X], [s], d_in, 1, dev)
+    H2 = gpu_hessian([X], [s], d_in, 1, dev)
+    assert torch.equal(H1, H2)
+    ref = X.double().T @ X.double()
+    rel = (H1[0].double() - ref).norm() / ref.norm()
+    assert rel.item() < 1e-5            # unit weights are exact in bf16: only fp32 accumulation error remains
+
+
+def test_hessian_errors(dev):
+    X = torch.zeros((16, 64), dtype=torch.bfloat16, device=dev)
+    s = torch.zeros((2, 16), dtype=torch.float32, device=dev)
+    H = torch.zeros((2, 64, 64), dtype=torch.float32, device=dev)
+    ws = libgq.alloc_workspace(libgq.gq_hessian_workspace_bytes(16, 64, 2), dev)
+    with pytest.raises(libgq.GQError) as e:
+        libgq.gq_hessian_accumulate(X, s, H, ws[:1024])
+    assert "GQ_ERR_WORKSPACE" in str(e.value)
+    with pytest.raises(libgq.GQError) as e:
+        libgq.gq_hessian_accumulate(X, s, H, ws, flags=1)
+    assert "GQ_ERR_INVALID_ARG" in str(e.value)
+    Xbad = torch.zeros((16, 68), dtype=torch.bfloat16, device=dev)
+    Hbad = torch.zeros((2, 68, 68), dtype=torch.float32, device=dev)
+    with pytest.raises(libgq.GQError) as e:
+        libgq.gq_hessian_accumulate(Xbad, s, Hbad, ws)
+    assert "GQ_ERR_UNSUPPORTED_SHAPE" in str(e.value)
+    assert libgq.gq_hessian_workspace_bytes(16, 68, 2) == 0
+    assert torch.count_nonzero(H).item() == 0            # nothing was written by the rejected calls
+
+
+# ------------------------------------------------------------------------------------------ objective
+@pytest.mark.parametrize("d_in,d_out,g", [(256, 512, 4), (384, 256, 2), (8, 8, 1), (520, 120, 3), (1032, 64, 1)])
+def test_objective_on_oracle_hessian(dev, d_in, d_out, g):
+    """Isolates Eq. 7: H comes from the oracle (rounded to fp32), only the objective runs on the GPU."""
+    rng = np.random.default_rng(d_in + d_out)
+    n = 200
+    xb = orc.f64_to_bf16_bits(rng.standard_normal((n, d_in)) * np.exp(rng.standard_normal(d_in)))
+    s = rng.random((g, n)) * np.exp(rng.standard_normal(n))
+    H32 = orc.hessian(xb, s).astype(np.float32)
+    W = (0.02 * rng.standard_normal((d_out, d_in))).astype(np.float32)
+    What = synth.uniform_grid_round(torch.from_numpy(W), 16).numpy()
+    loss_ref = orc.objective(W, What, H32.astype(np.float64))
+    Hd = torch.from_numpy(H32).to(dev)
+    ws = libgq.alloc_workspace(libgq.gq_objective_workspace_bytes(d_in, d_out, g), dev)
+    loss = libgq.gq_objective(torch.from_numpy(W).to(dev), torch.from_numpy(What).to(dev), Hd, ws)
+    libgq.gq_check()
+    check_loss(loss, loss_ref)
+    # only the upper triangle may be read: garbage below the diagonal must not change the result
+    Hd2 = Hd.clone()
+    tril = torch.tril(torch.ones(d_in, d_in, device=dev, dtype=torch.bool), diagonal=-1)
+    Hd2[:, tril] = 1e30
+    loss2 = libgq.gq_objective(torch.from_numpy(W).to(dev), torch.from_numpy(What).to(dev), Hd2, ws)
+    libgq.gq_check()
+    assert torch.equal(loss, loss2)
+
+
+def test_objective_zero_and_single_entry(dev):
+    d_in, d_out, g = 128, 16, 2
+    gen = torch.Generator(device=dev).manual_seed(5)
+    X = torch.randn(64, d_in, generator=gen, device=dev).to(torch.bfloat16)
+    s = torch.rand(g, 64, generator=gen, device=dev)
+    H = gpu_hessian([X], [s], d_in, g, dev)
+    W = torch.randn(d_out, d_in, generator=gen, device=dev)
+    ws = libgq.alloc_workspace(libgq.gq_objective_workspace_bytes(d_in, d_out, g), dev)
+    loss = libgq.gq_objective(W, W.clone(), H, ws)
+    libgq.gq_check()
+    assert torch.count_nonzero(loss).item() == 0
+    # a single perturbed weight with a value that bf16 cannot hold: the hi/lo split must recover it
+    What = W.clone()
+    What[11, 77] += 0.123456789
+    loss = libgq.gq_objective(W, What, H, ws)
+    libgq.gq_check()
+    delta = float(W[11, 77].double() - What[11, 77].double())
+    expect = delta * delta * float(H[1, 77, 77])
+    got = loss.cpu().numpy()
+    assert got[0] == 0.0
+    assert abs(got[1] - expect) <= 1e-4 * expect and abs(got[2] - expect) <= 1e-4 * expect
+
+
+# ------------------------------------------------------------------------------------------ whole path
+def run_layer(cfg, dev, n_tokens=None, grad_scale=1.0, seed=0):
+    syn = synth.LayerSynth(cfg, dev, seed=seed)
+    g = cfg.g
+    n = cfg.n if n_tokens is None else n_tokens
+    H = torch.zeros((g, cfg.d_in, cfg.d_in), dtype=torch.float32, device=dev)
+    ws = libgq.alloc_workspace(libgq.gq_hessian_workspace_bytes(cfg.chunk, cfg.d_in, g), dev)
+    xs, gs, ss = [], [], []
+    done, c = 0, 0
+    while done < n:
+        nt = min(cfg.chunk, n - done)
+        X, grad = syn.x_chunk(c, nt), syn.grad_chunk(c, nt)
+        s = libgq.gq_saliency(grad, g, grad_scale)
+        libgq.gq_hessian_accumulate(X, s, H, ws)
+        xs.append(X), gs.append(grad), ss.append(s)
+        done += nt
+        c += 1
+    libgq.gq_hessian_finalize(H)
+    W, What = syn.weights()
+    ows = libgq.alloc_workspace(libgq.gq_objective_workspace_bytes(cfg.d_in, cfg.d_out, g), dev)
+    loss = libgq.gq_objective(W, What, H, ows)
+    libgq.gq_check()
+    return xs, gs, ss, H, W, What, loss
+
+
+@pytest.mark.parametrize("grad_scale", [1.0, 1e3])
+def test_tiny_config_end_to_end(dev, grad_scale):
+    cfg = synth.CONFIGS["c0_tiny"]
+    xs, gs, ss, H, W, What, loss = run_layer(cfg, dev, grad_scale=grad_scale)
+    xb = np.concatenate([synth.bf16_bits(x) for x in xs])
+    gb = np.concatenate([synth.bf16_bits(x) for x in gs])
+    s_ref = orc.saliency(gb, cfg.g, grad_scale)
+    check_s(torch.cat(ss, dim=1), s_ref)
+    H_ref = orc.hessian(xb, s_ref)
+    check_H(H, H_ref)
+    check_loss(loss, orc.objective(W.cpu().numpy(), What.cpu().numpy(), H_ref))
+    # PSD up to rounding: the smallest eigenvalue is not below -1e-3 of the largest
+    for k in range(cfg.g):
+        ev = np.linalg.eigvalsh(H[k].cpu().numpy().astype(np.float64))
+        assert ev.min() >= -1e-3 * ev.max()
+
+
+@pytest.mark.parametrize("name,prefix", [("c1_7b_attn", 512), ("c2_7b_down", 128), ("c4_sweep", 160)])
+def test_large_shapes_token_prefix(dev, name, prefix):
+    """Full d_in / d_out of the large layers on a token prefix the oracle finishes in seconds."""
+    cfg = synth.CONFIGS[name]
+    for g in (cfg.groups if name == "c4_sweep" else cfg.groups[:1]):
+        c = synth.LayerConfig(cfg.name, prefix, min(cfg.chunk, 200), cfg.d_in, cfg.d_out, (g,), cfg.x_kind,
+                              cfg.outlier_frac, cfg.outlier_mult)
+        xs, gs, ss, H, W, What, loss = run_layer(c, dev)
+        xb = np.concatenate([synth.bf16_bits(x) for x in xs])
+        gb = np.concatenate([synth.bf16_bits(x) for x in gs])
+        s_ref = orc.saliency(gb, g)
+        check_s(torch.cat(ss, dim=1), s_ref)
+        H_ref = orc.hessian(xb, s_ref)
+        check_H(H, H_ref)
+        # objective through the token form (never forms the fp64 H product with all channels)
+        delta = (W.double() - What.double()).cpu().numpy()
+        z = orc.bf16_bits_to_f64(xb) @ delta.T                            # [n, d_out]
+        m = cfg.d_out // g
+        loss_ref = np.array([(s_ref[k][:, None] * z[:, k * m:(k + 1) * m] ** 2).sum() for k in range(g)])
+        check_loss(loss[:g], loss_ref)
+        check_loss(loss[g:], np.array([loss_ref.sum()]))
+        del H, xs, gs, ss
+        torch.cuda.empty_cache()
+
+
+def test_bench_workload_full_size_sampled(dev):
+    """Config 1 at full size (131072 tokens, 16 chunks), as bench.py runs it.
+
+    The oracle cannot form 4 x 4096^2 x 131072 products in seconds, so it is run exactly on a sampled
+    sub-problem: for 48 sampled input features F it computes H_k[F][:, F] from the columns X[:, F] alone,
+    which are the same entries of the full H_k; s is checked in full; the objective is checked with the
+    weight error restricted to the sampled features (W_hat = W elsewhere), which needs only those entries."""
+    cfg = synth.CONFIGS["c1_7b_attn"]
+    g = cfg.g
+    xs, gs, ss, H, W, What, loss = run_layer(cfg, dev)
+    rng = np.random.default_rng(0)
+    syn = synth.LayerSynth(cfg, dev, seed=0)
+    F = np.sort(np.concatenate([rng.choice(cfg.d_in, 40, replace=False),
+                                syn.outlier_features[:8].cpu().numpy()]))
+    F = np.unique(F)
+    Ft = torch.from_numpy(F).to(dev)
+    xb = np.concatenate([synth.bf16_bits(x[:, Ft].contiguous()) for x in xs])          # [n, |F|]
+    # saliency: the oracle on the whole gradient (one pass over 1 GB on the host)
+    s_ref = np.concatenate([orc.saliency(synth.bf16_bits(gc), g) for gc in gs], axis=1)
+    check_s(torch.cat(ss, dim=1), s_ref)
+    H_ref = orc.hessian(xb, s_ref)                                                     # [g, |F|, |F|]
+    H_sub = H[:, Ft][:, :, Ft]
+    check_H(H_sub, H_ref)
+    Hc = H[0].cpu()
+    assert torch.equal(Hc, Hc.T)
+    # objective: restrict to the sampled features by zeroing delta elsewhere (W_hat = W off F)
+    mask = torch.zeros(cfg.d_in, dtype=torch.bool, device=dev)
+    mask[Ft] = True
+    What_f = torch.where(mask[None, :], What, W)
+    ows = libgq.alloc_workspace(libgq.gq_objective_workspace_bytes(cfg.d_in, cfg.d_out, g), dev)
+    loss_f = libgq.gq_objective(W, What_f, H, ows)
+    libgq.gq_check()
+    loss_ref = orc.objective(W[:, Ft].contiguous().cpu().numpy(), What[:, Ft].contiguous().cpu().numpy(), H_ref)
+    check_loss(loss_f, loss_ref)
+    assert np.all(loss.cpu().numpy() > 0)
+
+
+# ------------------------------------------------------------------------------------------ host path
+def test_host_pipeline_matches_device_calls(dev):
+    cfg = synth.LayerConfig("host", 700, 256, 384, 256, (2,), "lognormal", 0.01, 20.0)
+    xs, gs, ss, H, W, What, loss = run_layer(cfg, dev)
+    X_host = torch.cat(xs).cpu().pin_memory()
+    grad_host = torch.cat(gs).cpu().pin_memory()
+    arena = libgq.alloc_workspace(libgq.gq_layer_host_arena_bytes(cfg.chunk, cfg.d_in, cfg.d_out, cfg.g), dev)
+    H_host = torch.empty((cfg.g, cfg.d_in, cfg.d_in), dtype=torch.float32).pin_memory()
+    loss_host = libgq.gq_layer_objective_host(X_host, grad_host, cfg.chunk, cfg.g, 1.0, W.cpu(), What.cpu(), arena,
+                                              H_host=H_host)
+    assert torch.equal(H_host, H.cpu())
+    assert torch.equal(loss_host, loss.cpu())
