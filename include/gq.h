@@ -59,7 +59,7 @@ int32_t gq_last_cuda_error(void);
  *     s[k * ld_s + i] = (grad_scale^2 / m) * sum_{j = m k}^{m (k+1) - 1} grad[i * ld_grad + j]^2
  *
  *   grad        bf16 [n, ld_grad], 16-byte aligned, ld_grad >= d_out, ld_grad % 8 == 0
- *   n           tokens in this call, >= 0 (0 is a no-op)
+ *   n           tokens in this call, >= 0 (0 is a no-op: sizes are still validated, pointers are not)
  *   d_out, g    d_out % g == 0 and (d_out / g) % 8 == 0, 1 <= g <= 1024
  *   grad_scale  finite; the paper uses 1e3, tests use 1
  *   s           fp32 [g, ld_s] (group-major so that each s_k is contiguous), ld_s >= n
@@ -74,7 +74,8 @@ int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad,
  * for every group k and every a <= b (the upper triangle including the diagonal).  No 1/n factor.
  *
  *   X          bf16 [n, ld_x], 16-byte aligned, ld_x >= d_in, ld_x % 8 == 0
- *   n          tokens in this chunk, 0 <= n <= the n_max the workspace was sized for
+ *   n          tokens in this chunk, 0 <= n <= the n_max the workspace was sized for (0 is a no-op:
+ *              sizes are still validated, pointers are not)
  *   d_in       d_in % 8 == 0, 8 <= d_in <= 65536
  *   s          fp32 [g, ld_s], s >= 0 (as produced by gq_saliency), ld_s >= n
  *   H          fp32 [g, d_in, d_in] row-major, 16-byte aligned.  The caller zeroes it before the

@@ -183,12 +183,14 @@ uint64_t gq_launch_count(void) { return g_launches.load(); }
 int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad, int32_t g, float grad_scale,
                     float *s, int64_t ld_s, void *stream)
 {
-    if (!grad || !s || n < 0 || g < 1 || d_out < 1 || d_out % g != 0 || ld_grad < d_out || ld_s < n ||
+    if (n < 0 || g < 1 || d_out < 1 || d_out % g != 0 || ld_grad < d_out || ld_s < n ||
         !(grad_scale == grad_scale) || grad_scale - grad_scale != 0.0f)
         return GQ_ERR_INVALID_ARG;
     if ((d_out / g) % 8 != 0 || g > 1024 || d_out > (1ll << 24) || n > (1ll << 40)) return GQ_ERR_UNSUPPORTED_SHAPE;
-    if (!aligned(grad, 16) || ld_grad % 8 != 0 || !aligned(s, 4)) return GQ_ERR_ALIGNMENT;
-    if (n == 0) return GQ_OK;
+    if (ld_grad % 8 != 0) return GQ_ERR_ALIGNMENT;
+    if (n == 0) return GQ_OK;              // nothing to read or write: pointers are not looked at
+    if (!grad || !s) return GQ_ERR_INVALID_ARG;
+    if (!aligned(grad, 16) || !aligned(s, 4)) return GQ_ERR_ALIGNMENT;
     DeviceInfo *di;
     if (int32_t rc = device_info(&di)) return rc;
     const int m = static_cast<int>(d_out / g);
@@ -211,11 +213,13 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
                               int32_t g, float *H, uint32_t flags, void *workspace, size_t workspace_bytes,
                               void *stream)
 {
-    if (!X || !s || !H || n < 0 || ld_x < d_in || ld_s < n || flags != 0) return GQ_ERR_INVALID_ARG;
+    if (n < 0 || ld_x < d_in || ld_s < n || flags != 0) return GQ_ERR_INVALID_ARG;
     if (int32_t rc = check_layer_shape(d_in, 0, g, false)) return rc;
     if (n > (1ll << 31) - 64) return GQ_ERR_UNSUPPORTED_SHAPE;
-    if (!aligned(X, 16) || ld_x % 8 != 0 || !aligned(H, 16) || !aligned(s, 4)) return GQ_ERR_ALIGNMENT;
-    if (n == 0) return GQ_OK;
+    if (ld_x % 8 != 0) return GQ_ERR_ALIGNMENT;
+    if (n == 0) return GQ_OK;              // an empty chunk adds nothing: pointers are not looked at
+    if (!X || !s || !H) return GQ_ERR_INVALID_ARG;
+    if (!aligned(X, 16) || !aligned(H, 16) || !aligned(s, 4)) return GQ_ERR_ALIGNMENT;
     if (!workspace || workspace_bytes < hessian_ws_bytes(n, d_in, g)) return GQ_ERR_WORKSPACE;
     if (!aligned(workspace, 1024)) return GQ_ERR_ALIGNMENT;
     DeviceInfo *di;
