@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the guided-objective hot path (saliency -> guided Hessians -> objective).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One "step" is one pass of the whole path over one synthetic layer: for every token chunk
+gq_saliency + gq_hessian_accumulate, then gq_hessian_finalize and gq_objective (H is zeroed at the
+start of the step).  The default workload is the Llama-2-7B attention-projection shape
+(131072 tokens in 16 chunks of 8192, d_in = d_out = 4096, g = 4).  All inputs are seeded and
+synthetic and stay resident in HBM for the device-timed number; the `e2e` number goes through
+gq_layer_objective_host with pinned host buffers (host->device copies inside the timed region).
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank processes its own layer
+(different seed): the path shards over layers with no data-path collective, so scaling is weak and the
+only communication is the barrier / max-reduction of the timing.
+
+`--impl reference` times the CPU fp64 oracle on the host cores on a bounded sample of the same
+workload (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2505_07004_b200 import synth
+
+METRIC = "guided_hessian_tokens_per_s"
+UNIT = "tokens/s"
+# DRAM bytes per launch of the dominant kernel from the committed ncu capture (profiles/), scaled to
+# one launch of the default workload; None until a capture exists for the current kernel.
+NCU_TRAFFIC_BYTES = {"c1_7b_attn": None}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "of measured (MEASURED_PEAKS.json)"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "source": "of fallback (earlier measurement on this pool)"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting"}
+
+    def __init__(self, device):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.max_mhz, self.ok = [], set(), None, False
+        self._stop_evt = threading.Event()
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if hasattr(uuid, "encode") else uuid)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception as e:  # NVML missing: clocks are reported as unknown
+            self.err = repr(e)
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    mask = int(self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop_evt.wait(0.05)
+
+    def finish(self):
+        self._stop_evt.set()
+        self.join(timeout=2.0)
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["nvml_unavailable"]}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def oracle_sample(cfg, g, tokens, channels_per_group, seed=0):
+    """One bounded pass of the oracle: saliency + Hessian on `tokens` tokens of chunk 0 and the objective
+    on `channels_per_group` channels of every group.  Returns (tokens/s equivalent, seconds, description)."""
+    from oracle import gq_oracle as orc
+    syn = synth.LayerSynth(cfg, "cpu", seed=seed)
+    xb = synth.bf16_bits(syn.x_chunk(0, tokens))
+    gb = synth.bf16_bits(syn.grad_chunk(0, tokens))
+    m = cfg.d_out // g
+    cpg = min(channels_per_group, m)
+    W, What = syn.weights()
+    rows = torch.cat([torch.arange(k * m, k * m + cpg) for k in range(g)])
+    Wn, Whn = W[rows].contiguous().numpy(), What[rows].contiguous().numpy()
+    t0 = time.perf_counter()
+    s = orc.saliency(gb, g, 1.0)
+    t1 = time.perf_counter()
+    H = orc.hessian(xb, s)
+    t2 = time.perf_counter()
+    orc.objective(Wn, Whn, H)
+    t3 = time.perf_counter()
+    # the objective is paid once per layer: amortise its full-layer cost over the layer's n tokens
+    t_obj_per_token = (t3 - t2) * (m / cpg) / cfg.n
+    seconds = (t1 - t0) + (t2 - t1) + t_obj_per_token * tokens
+    desc = ("fp64 oracle as is: saliency+Hessian on the first %d tokens of chunk 0 (%.2f s + %.2f s), objective on %d of "
+            "%d channels per group (%.2f s) scaled to all channels and amortised over n=%d tokens"
+            % (tokens, t1 - t0, t2 - t1, cpg, m, t3 - t2, cfg.n))
+    return tokens / seconds, (t3 - t0), desc
+
+
+def run_reference(args, cfg, g):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    from oracle import gq_oracle as orc
+    orc.build()
+    tokens, cpg = args.ref_tokens, args.ref_channels
+    for _ in range(args.warmup):
+        oracle_sample(cfg, g, tokens, cpg)
+    t0 = time.perf_counter()
+    vals = []
+    desc = ""
+    for _ in range(args.steps):
+        v, _, desc = oracle_sample(cfg, g, tokens, cpg)
+        vals.append(v)
+    wall = time.perf_counter() - t0
+    value = len(vals) / sum(1.0 / v for v in vals)          # harmonic mean = total tokens / total time
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * wall / max(1, args.steps),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "n": cfg.n, "chunk": cfg.chunk, "d_in": cfg.d_in, "d_out": cfg.d_out, "g": g},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.threads(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out), flush=True)
+
+
+def run_ours(args, cfg, g):
+    from paper_2505_07004_b200 import api as libgq
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: libgq has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    libgq.lib()
+    peaks = load_peaks()
+
+    # ---- resident synthetic layer (one per rank: the path shards over layers)
+    syn = synth.LayerSynth(cfg, dev, seed=rank)
+    n_chunks = cfg.n_chunks
+    xs = [syn.x_chunk(c) for c in range(n_chunks)]
+    gs = [syn.grad_chunk(c) for c in range(n_chunks)]
+    W, What = syn.weights()
+    H = torch.empty((g, cfg.d_in, cfg.d_in), dtype=torch.float32, device=dev)
+    s_buf = torch.empty((g, cfg.chunk), dtype=torch.float32, device=dev)
+    ws = libgq.alloc_workspace(libgq.gq_hessian_workspace_bytes(cfg.chunk, cfg.d_in, g), dev)
+    ows = libgq.alloc_workspace(libgq.gq_objective_workspace_bytes(cfg.d_in, cfg.d_out, g), dev)
+    loss = torch.empty(g + 1, dtype=torch.float64, device=dev)
+
+    def step():
+        H.zero_()
+        for c in range(n_chunks):
+            nt = xs[c].shape[0]
+            libgq.gq_saliency(gs[c], g, 1.0, s=s_buf[:, :nt])
+            libgq.gq_hessian_accumulate(xs[c], s_buf[:, :nt], H, ws)
+        libgq.gq_hessian_finalize(H)
+        libgq.gq_objective(W, What, H, ows, loss=loss)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    libgq.gq_check()
+
+    sampler = ClockSampler(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    launches0 = libgq.gq_launch_count()
+    libgq.gq_kernel_timing_enable(True)
+    sampler.start()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    clocks = sampler.finish()
+    ms_total = e0.elapsed_time(e1)
+    kern = libgq.gq_kernel_timing_read()
+    libgq.gq_kernel_timing_enable(False)
+    launches = libgq.gq_launch_count() - launches0
+    libgq.gq_check()
+    loss_host = loss.cpu().numpy()
+    if not np.all(np.isfinite(loss_host)) or loss_host[g] <= 0:
+        raise RuntimeError("objective is not finite/positive: %s" % loss_host)
+
+    # ---- end to end from pinned host memory through the host-buffer entry point
+    e2e_s, e2e_steps, h2d, d2h = float('nan'), 0, 0, 0
+    if not args.no_e2e:
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        Xh = torch.empty((cfg.n, cfg.d_in), dtype=torch.bfloat16).pin_memory()
+        Gh = torch.empty((cfg.n, cfg.d_out), dtype=torch.bfloat16).pin_memory()
+        off = 0
+        for c in range(n_chunks):
+            nt = xs[c].shape[0]
+            Xh[off:off + nt].copy_(xs[c])
+            Gh[off:off + nt].copy_(gs[c])
+            off += nt
+        Wh, Whh = W.cpu().pin_memory(), What.cpu().pin_memory()
+        loss_h = torch.empty(g + 1, dtype=torch.float64).pin_memory()
+        del xs, gs
+        torch.cuda.empty_cache()
+        arena = libgq.alloc_workspace(libgq.gq_layer_host_arena_bytes(cfg.chunk, cfg.d_in, cfg.d_out, g), dev)
+        libgq.gq_layer_objective_host(Xh, Gh, cfg.chunk, g, 1.0, Wh, Whh, arena, loss_host=loss_h)   # warm-up
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            libgq.gq_layer_objective_host(Xh, Gh, cfg.chunk, g, 1.0, Wh, Whh, arena, loss_host=loss_h)
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
+        if abs(loss_h[g].item() - loss_host[g]) > 1e-9 * abs(loss_host[g]):
+            raise RuntimeError("host-buffer path and device path disagree: %r vs %r" % (loss_h[g].item(), loss_host[g]))
+        h2d = Xh.numel() * 2 + Gh.numel() * 2 + Wh.numel() * 4 + Whh.numel() * 4
+        d2h = (g + 1) * 8
+
+    # ---- max over ranks
+    times = torch.tensor([ms_total, e2e_s * 1e3], dtype=torch.float64, device=dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms = float(times[0]), float(times[1])
+
+    if rank == 0:
+        tokens_per_step = cfg.n * world
+        value = tokens_per_step * args.steps / (ms_total * 1e-3)
+        e2e_value = tokens_per_step * e2e_steps / (e2e_ms * 1e-3) if e2e_steps else None
+        # dominant kernel: the tensor-core Gram kernel of gq_hessian_accumulate
+        ga_ms, ga_n = kern["gram_accum"]
+        flops_per_launch = float(g) * cfg.chunk * cfg.d_in * (cfg.d_in + 1)      # upper triangle, mul + add
+        achieved = flops_per_launch / (ga_ms / max(1, ga_n) * 1e-3) / 1e12 if ga_n else None
+        peak = peaks["bf16_tflops_sustained"]
+        kernel_ms = sum(v[0] for v in kern.values())
+        kernels = {k: {"launches": v[1], "ms_total": round(v[0], 4), "share": round(v[0] / kernel_ms, 4) if kernel_ms else None}
+                   for k, v in kern.items()}
+        sal_ms, sal_n = kern["saliency"]
+        sal_bytes = cfg.chunk * (2 * cfg.d_out + 4 * g)
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "n": cfg.n, "chunk": cfg.chunk, "d_in": cfg.d_in, "d_out": cfg.d_out, "g": g,
+                       "l2": "inputs (%.2f GB of X and grad per step, streamed once) are larger than L2; no flush"
+                             % ((cfg.n * (cfg.d_in + cfg.d_out) * 2) / 1e9),
+                       "parallelism": "one layer per GPU, no collective"},
+            "hessian_tflops_useful": (float(g) * cfg.n * cfg.d_in * (cfg.d_in + 1)) * world * args.steps / (ms_total * 1e-3) / 1e12,
+            "roofline": {"kernel": "gram_kernel<EPI_ACCUM> (gq_hessian_accumulate)", "bound": "tensor",
+                         "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                         "frac": (achieved / peak) if achieved else None,
+                         "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
+                         "peak_source": "bf16_tflops_sustained, " + peaks["source"],
+                         "frac_of_burst_peak": (achieved / peaks["bf16_tflops"]) if achieved else None,
+                         "flops_per_launch": flops_per_launch, "ms_per_launch": ga_ms / max(1, ga_n)},
+            "saliency_hbm": {"achieved_gbs": (sal_bytes / (sal_ms / max(1, sal_n) * 1e-3) / 1e9) if sal_n else None,
+                             "peak_gbs": peaks["hbm_gbs"]},
+            "kernels": kernels,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps, "api": "gq_layer_objective_host (pinned host buffers)"},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "loss_total": float(loss_host[g]),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            from oracle import gq_oracle as orc
+            orc.build()
+            v, secs, desc = oracle_sample(cfg, g, args.cpu_tokens, args.cpu_channels)
+            out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": orc.threads(), "kind": "oracle",
+                                   "sample": desc, "seconds": secs}
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c1_7b_attn", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--g", type=int, default=0, help="override the number of groups (sweep config)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-tokens", type=int, default=768)
+    ap.add_argument("--cpu-channels", type=int, default=128)
+    ap.add_argument("--ref-tokens", type=int, default=256)
+    ap.add_argument("--ref-channels", type=int, default=64)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--tokens", type=int, default=0, help="use only the first TOKENS tokens (profiling runs)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = synth.CONFIGS[args.workload]
+    if args.tokens:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, n=min(cfg.n, args.tokens))
+    g = args.g if args.g else cfg.g
+    if args.impl == "reference":
+        run_reference(args, cfg, g)
+    else:
+        run_ours(args, cfg, g)
+
+
+if __name__ == "__main__":
+    main()

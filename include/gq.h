@@ -159,6 +159,30 @@ int32_t gq_check(void *stream, uint32_t *detail /* HOST, may be NULL */);
 /* Number of kernels this library has launched from the calling process (for bookkeeping). */
 uint64_t gq_launch_count(void);
 
+/*
+ * Measurement aid (no counterpart in the paper).  The library's kernels, in launch order of a layer:
+ */
+enum gq_kernel_id {
+    GQ_KERNEL_SALIENCY = 0,    /* Algorithm 1 line 2                                    */
+    GQ_KERNEL_SCALE_ROWS = 1,  /* Diag(s_k) X, bf16                                      */
+    GQ_KERNEL_GRAM_ACCUM = 2,  /* tensor-core X^T (Diag(s_k) X), H += (Algorithm 1 l. 4) */
+    GQ_KERNEL_MIRROR = 3,      /* gq_hessian_finalize                                    */
+    GQ_KERNEL_SPLIT_DELTA = 4, /* W - W_hat -> bf16 hi/lo                                */
+    GQ_KERNEL_GRAM_DOT = 5,    /* tensor-core Delta_k^T Delta_k contracted with H_k (Eq. 7) */
+    GQ_KERNEL_REDUCE = 6,      /* fp64 reduction of the partial sums                     */
+    GQ_KERNEL_COUNT = 7
+};
+
+/*
+ * gq_kernel_timing_enable(1) makes every later launch record a CUDA event on its stream directly
+ * before and after the kernel; gq_kernel_timing_enable(0) stops that.  Either call discards what
+ * was recorded so far.  gq_kernel_timing_read() waits for the recorded events and writes, per
+ * gq_kernel_id, the summed device time in milliseconds and the number of launches into two HOST
+ * arrays of GQ_KERNEL_COUNT entries, then discards them.  Off by default.
+ */
+int32_t gq_kernel_timing_enable(int32_t enable);
+int32_t gq_kernel_timing_read(double *ms_sum, uint64_t *launches);
+
 #ifdef __cplusplus
 }
 #endif

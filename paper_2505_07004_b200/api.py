@@ -22,7 +22,9 @@ EXPORTS = (
     "gq_version", "gq_status_string", "gq_last_cuda_error", "gq_saliency", "gq_hessian_accumulate",
     "gq_hessian_workspace_bytes", "gq_hessian_finalize", "gq_objective", "gq_objective_workspace_bytes",
     "gq_layer_objective_host", "gq_layer_host_arena_bytes", "gq_check", "gq_launch_count",
+    "gq_kernel_timing_enable", "gq_kernel_timing_read",
 )
+KERNEL_NAMES = ("saliency", "scale_rows", "gram_accum", "mirror", "split_delta", "gram_dot", "reduce")
 
 
 class GQError(RuntimeError):
@@ -69,6 +71,10 @@ def lib() -> ctypes.CDLL:
         L.gq_layer_objective_host.argtypes = [vp, vp, i64, i64, i64, i64, i32, f32, vp, vp, vp, vp, vp, sz, vp]
         L.gq_check.restype = i32
         L.gq_check.argtypes = [vp, vp]
+        L.gq_kernel_timing_enable.restype = i32
+        L.gq_kernel_timing_enable.argtypes = [i32]
+        L.gq_kernel_timing_read.restype = i32
+        L.gq_kernel_timing_read.argtypes = [vp, vp]
         _lib = L
     return _lib
 
@@ -229,3 +235,19 @@ def gq_check(stream=None):
         err = GQError("gq_check", rc)
         err.detail = tuple(int(v) for v in detail)
         raise err
+
+
+def gq_kernel_timing_enable(enable: bool) -> None:
+    rc = lib().gq_kernel_timing_enable(1 if enable else 0)
+    if rc:
+        raise GQError("gq_kernel_timing_enable", rc)
+
+
+def gq_kernel_timing_read() -> dict:
+    """``{kernel name: (summed device ms, launches)}`` for the launches recorded since the last read."""
+    ms = (ctypes.c_double * len(KERNEL_NAMES))()
+    cnt = (ctypes.c_uint64 * len(KERNEL_NAMES))()
+    rc = lib().gq_kernel_timing_read(ms, cnt)
+    if rc:
+        raise GQError("gq_kernel_timing_read", rc)
+    return {name: (float(ms[i]), int(cnt[i])) for i, name in enumerate(KERNEL_NAMES)}

@@ -9,6 +9,8 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <utility>
+#include <vector>
 
 #include "../../include/gq.h"
 #include "gq_gram.cuh"
@@ -22,6 +24,37 @@ constexpr int kMaxDevices = 64;
 
 thread_local int32_t tl_last_cuda_error = 0;
 std::atomic<uint64_t> g_launches{0};
+
+// Optional per-kernel timing (gq_kernel_timing_*): a pair of events around every launch.
+std::atomic<int> g_timing_on{0};
+std::mutex g_timing_mutex;
+std::vector<std::pair<cudaEvent_t, cudaEvent_t>> g_timing_events[GQ_KERNEL_COUNT];
+
+struct LaunchScope {
+    int id;
+    cudaStream_t st;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    LaunchScope(int id_, cudaStream_t st_) : id(id_), st(st_)
+    {
+        g_launches.fetch_add(1);
+        if (g_timing_on.load(std::memory_order_relaxed)) {
+            if (cudaEventCreate(&e0) == cudaSuccess && cudaEventCreate(&e1) == cudaSuccess) {
+                cudaEventRecord(e0, st);
+            } else {
+                if (e0) cudaEventDestroy(e0);
+                e0 = e1 = nullptr;
+            }
+        }
+    }
+    ~LaunchScope()
+    {
+        if (e0) {
+            cudaEventRecord(e1, st);
+            std::lock_guard<std::mutex> lock(g_timing_mutex);
+            g_timing_events[id].emplace_back(e0, e1);
+        }
+    }
+};
 
 // Per-device status word {status, site, block, unit}; written by kernels, read by gq_check().
 __device__ uint32_t g_status_word[4];
@@ -196,9 +229,11 @@ int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad,
     const int m = static_cast<int>(d_out / g);
     const float coef = grad_scale * grad_scale / static_cast<float>(m);
     const int grid = grid_for(n * g * 32, 256, di->sm_count, 8);
-    gq::saliency_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const __nv_bfloat16 *>(grad), n, m, ld_grad, g, coef, s, ld_s);
-    g_launches.fetch_add(1);
+    {
+        LaunchScope scope(GQ_KERNEL_SALIENCY, static_cast<cudaStream_t>(stream));
+        gq::saliency_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+            static_cast<const __nv_bfloat16 *>(grad), n, m, ld_grad, g, coef, s, ld_s);
+    }
     GQ_CUDA(cudaGetLastError());
     return GQ_OK;
 }
@@ -230,9 +265,11 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
     // Y_k = Diag(s_k) X rounded to bf16, so that H_k += X^T Y_k.
     {
         const int grid = grid_for(n * (d_in / 8), 256, di->sm_count, 8);
-        gq::scale_rows_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), n, static_cast<int>(d_in),
-                                                    ld_x, s, ld_s, g, Y);
-        g_launches.fetch_add(1);
+        {
+            LaunchScope scope(GQ_KERNEL_SCALE_ROWS, st);
+            gq::scale_rows_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), n, static_cast<int>(d_in),
+                                                        ld_x, s, ld_s, g, Y);
+        }
         GQ_CUDA(cudaGetLastError());
     }
     CUtensorMap mapX, mapY;
@@ -254,8 +291,10 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
     p.status = di->status_ptr;
     p.wait_budget_ns = wait_budget_ns();
     const int grid = p.units < di->sm_count ? p.units : di->sm_count;
-    gq::gram_kernel<gq::EPI_ACCUM><<<grid, gq::GRAM_THREADS, gq::GRAM_SMEM_BYTES, st>>>(mapX, mapY, p);
-    g_launches.fetch_add(1);
+    {
+        LaunchScope scope(GQ_KERNEL_GRAM_ACCUM, st);
+        gq::gram_kernel<gq::EPI_ACCUM><<<grid, gq::GRAM_THREADS, gq::GRAM_SMEM_BYTES, st>>>(mapX, mapY, p);
+    }
     GQ_CUDA(cudaGetLastError());
     return GQ_OK;
 }
@@ -267,8 +306,10 @@ int32_t gq_hessian_finalize(float *H, int64_t d_in, int32_t g, void *stream)
     if (!aligned(H, 16)) return GQ_ERR_ALIGNMENT;
     const unsigned nb = static_cast<unsigned>((d_in + 31) / 32);
     dim3 grid(nb, nb, static_cast<unsigned>(g));
-    gq::mirror_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(H, static_cast<int>(d_in));
-    g_launches.fetch_add(1);
+    {
+        LaunchScope scope(GQ_KERNEL_MIRROR, static_cast<cudaStream_t>(stream));
+        gq::mirror_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(H, static_cast<int>(d_in));
+    }
     GQ_CUDA(cudaGetLastError());
     return GQ_OK;
 }
@@ -299,8 +340,10 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     {
         const long long count8 = d_in * d_out / 8;
         const int grid = grid_for(count8, 256, di->sm_count, 8);
-        gq::split_delta_kernel<<<grid, 256, 0, st>>>(W, W_hat, count8, hi, lo);
-        g_launches.fetch_add(1);
+        {
+            LaunchScope scope(GQ_KERNEL_SPLIT_DELTA, st);
+            gq::split_delta_kernel<<<grid, 256, 0, st>>>(W, W_hat, count8, hi, lo);
+        }
         GQ_CUDA(cudaGetLastError());
     }
     CUtensorMap mapHi, mapLo;
@@ -323,13 +366,60 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     p.status = di->status_ptr;
     p.wait_budget_ns = wait_budget_ns();
     const int grid = p.units < di->sm_count ? p.units : di->sm_count;
-    gq::gram_kernel<gq::EPI_DOT><<<grid, gq::GRAM_THREADS, gq::GRAM_SMEM_BYTES, st>>>(mapHi, mapLo, p);
-    g_launches.fetch_add(1);
+    {
+        LaunchScope scope(GQ_KERNEL_GRAM_DOT, st);
+        gq::gram_kernel<gq::EPI_DOT><<<grid, gq::GRAM_THREADS, gq::GRAM_SMEM_BYTES, st>>>(mapHi, mapLo, p);
+    }
     GQ_CUDA(cudaGetLastError());
-    gq::reduce_partials_kernel<<<1, 1024, 0, st>>>(partials, p.tile_slots, g, loss_out);
-    g_launches.fetch_add(1);
+    {
+        LaunchScope scope(GQ_KERNEL_REDUCE, st);
+        gq::reduce_partials_kernel<<<1, 1024, 0, st>>>(partials, p.tile_slots, g, loss_out);
+    }
     GQ_CUDA(cudaGetLastError());
     return GQ_OK;
+}
+
+int32_t gq_kernel_timing_enable(int32_t enable)
+{
+    std::lock_guard<std::mutex> lock(g_timing_mutex);
+    for (auto &v : g_timing_events) {
+        for (auto &pr : v) {
+            cudaEventDestroy(pr.first);
+            cudaEventDestroy(pr.second);
+        }
+        v.clear();
+    }
+    g_timing_on.store(enable ? 1 : 0);
+    return GQ_OK;
+}
+
+int32_t gq_kernel_timing_read(double *ms_sum, uint64_t *launches)
+{
+    if (!ms_sum || !launches) return GQ_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_timing_mutex);
+    int32_t rc = GQ_OK;
+    for (int id = 0; id < GQ_KERNEL_COUNT; ++id) {
+        double total = 0.0;
+        uint64_t count = 0;
+        for (auto &pr : g_timing_events[id]) {
+            float ms = 0.0f;
+            cudaError_t e = cudaEventSynchronize(pr.second);
+            if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, pr.first, pr.second);
+            if (e != cudaSuccess) {
+                tl_last_cuda_error = static_cast<int32_t>(e);
+                rc = GQ_ERR_CUDA;
+            } else {
+                total += ms;
+                ++count;
+            }
+            cudaEventDestroy(pr.first);
+            cudaEventDestroy(pr.second);
+        }
+        g_timing_events[id].clear();
+        ms_sum[id] = total;
+        launches[id] = count;
+    }
+    return rc;
 }
 
 int32_t gq_check(void *stream, uint32_t *detail)
