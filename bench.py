@@ -34,7 +34,7 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
-from paper_2505_07004_b200 import synth
+from paper_2505_07004_b200 import shard, synth
 
 METRIC = "guided_hessian_tokens_per_s"
 UNIT = "tokens/s"
@@ -92,7 +92,7 @@ class ClockSampler(threading.Thread):
                         self.reasons.add(name)
             except Exception:
                 pass
-            self._stop_evt.wait(0.05)
+            self._stop_evt.wait(0.02)
 
     def finish(self):
         self._stop_evt.set()
@@ -178,7 +178,7 @@ def run_ours(args, cfg, g):
     peaks = load_peaks()
 
     # ---- resident synthetic layer (one per rank: the path shards over layers)
-    syn = synth.LayerSynth(cfg, dev, seed=rank)
+    syn = synth.LayerSynth(cfg, dev, seed=shard.layer_seed_for_rank(0, rank))
     n_chunks = cfg.n_chunks
     xs = [syn.x_chunk(c) for c in range(n_chunks)]
     gs = [syn.grad_chunk(c) for c in range(n_chunks)]
@@ -259,16 +259,11 @@ def run_ours(args, cfg, g):
         d2h = (g + 1) * 8
 
     # ---- max over ranks
-    times = torch.tensor([ms_total, e2e_s * 1e3], dtype=torch.float64, device=dev)
-    if world > 1:
-        import torch.distributed as dist
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms = float(times[0]), float(times[1])
+    ms_total, e2e_ms = shard.max_over_ranks([ms_total, e2e_s * 1e3], device=dev)
 
     if rank == 0:
-        tokens_per_step = cfg.n * world
-        value = tokens_per_step * args.steps / (ms_total * 1e-3)
-        e2e_value = tokens_per_step * e2e_steps / (e2e_ms * 1e-3) if e2e_steps else None
+        value = shard.whole_job_throughput(cfg.n, args.steps, ms_total * 1e-3, world)
+        e2e_value = shard.whole_job_throughput(cfg.n, e2e_steps, e2e_ms * 1e-3, world) if e2e_steps else None
         # dominant kernel: the tensor-core Gram kernel of gq_hessian_accumulate
         ga_ms, ga_n = kern["gram_accum"]
         flops_per_launch = float(g) * cfg.chunk * cfg.d_in * (cfg.d_in + 1)      # upper triangle, mul + add
@@ -319,7 +314,7 @@ def run_ours(args, cfg, g):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c1_7b_attn", choices=sorted(synth.CONFIGS))
