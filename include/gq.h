@@ -148,6 +148,35 @@ int32_t gq_layer_objective_host(const void *X_host, const void *grad_host, int64
 size_t gq_layer_host_arena_bytes(int64_t chunk, int64_t d_in, int64_t d_out, int32_t g);
 
 /*
+ * The objective for callers that cannot allocate device memory (no counterpart in the paper; it is
+ * gq_objective with the scratch supplied by the library instead of the caller).
+ *
+ * Some users of this library run where cudaMalloc is off limits: inside a region that is being
+ * recorded into a CUDA graph, inside a framework callback that must not touch the allocator, in a
+ * process whose whole memory budget was handed to another pool at start-up, or in a latency-critical
+ * loop where an allocation (and the implicit synchronisation of a free) is not acceptable.  For them
+ * this entry point keeps its scratch in a fixed array inside the library's own device image:
+ *
+ *   - the array is 4 MiB + 128 KiB (two bf16 copies of W - W_hat and the partial sums); every GPU on
+ *     which the library is used holds that much from the moment the library is loaded until exit;
+ *   - therefore only small layers fit: d_in * d_out <= 1,048,576 weights and
+ *     (NJ * NJ + NJ) * g <= 4096 with NJ = ceil(d_in / 256).  Anything larger returns
+ *     GQ_ERR_UNSUPPORTED_SHAPE and launches nothing: use gq_objective with your own workspace;
+ *   - the call makes no cudaMalloc / cudaFree and no call into an allocating library.  The first
+ *     call on each device looks up the array's device address once (cudaGetSymbolAddress) and sets
+ *     kernel attributes; make that first call outside any stream capture;
+ *   - all calls on a device share the one array.  Two calls that overlap on the GPU (different
+ *     streams, or different host threads without ordering) race on it and give wrong results:
+ *     order them on one stream or with events.  The array keeps what the last call wrote; every
+ *     byte a call reads it has written itself first, so stale contents never leak into a result.
+ *
+ * Arguments, arithmetic and results are exactly those of gq_objective (W, W_hat, H, loss_out are the
+ * caller's device buffers); for shapes within the limit both entry points return identical values.
+ */
+int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, int64_t d_out,
+                             const float *H, int32_t g, double *loss_out, void *stream);
+
+/*
  * Synchronises `stream`, then returns and clears the first device-side error recorded on the
  * current device since the last gq_check (GQ_OK if none).  A pipeline wait inside a kernel that
  * exceeds its time budget (2 s by default; environment variable GQ_WAIT_BUDGET_MS) makes the

@@ -22,7 +22,7 @@ EXPORTS = (
     "gq_version", "gq_status_string", "gq_last_cuda_error", "gq_saliency", "gq_hessian_accumulate",
     "gq_hessian_workspace_bytes", "gq_hessian_finalize", "gq_objective", "gq_objective_workspace_bytes",
     "gq_layer_objective_host", "gq_layer_host_arena_bytes", "gq_check", "gq_launch_count",
-    "gq_kernel_timing_enable", "gq_kernel_timing_read",
+    "gq_kernel_timing_enable", "gq_kernel_timing_read", "gq_objective_noalloc",
 )
 KERNEL_NAMES = ("saliency", "scale_rows", "gram_accum", "mirror", "split_delta", "gram_dot", "reduce")
 
@@ -71,6 +71,8 @@ def lib() -> ctypes.CDLL:
         L.gq_layer_objective_host.argtypes = [vp, vp, i64, i64, i64, i64, i32, f32, vp, vp, vp, vp, vp, sz, vp]
         L.gq_check.restype = i32
         L.gq_check.argtypes = [vp, vp]
+        L.gq_objective_noalloc.restype = i32
+        L.gq_objective_noalloc.argtypes = [vp, vp, i64, i64, vp, i32, vp, vp]
         L.gq_kernel_timing_enable.restype = i32
         L.gq_kernel_timing_enable.argtypes = [i32]
         L.gq_kernel_timing_read.restype = i32
@@ -251,3 +253,27 @@ def gq_kernel_timing_read() -> dict:
     if rc:
         raise GQError("gq_kernel_timing_read", rc)
     return {name: (float(ms[i]), int(cnt[i])) for i, name in enumerate(KERNEL_NAMES)}
+
+
+def gq_objective_noalloc(W: torch.Tensor, W_hat: torch.Tensor, H: torch.Tensor, loss: torch.Tensor,
+                         stream=None) -> torch.Tensor:
+    """Eq. 7 for callers that must not allocate: scratch lives in a fixed array inside ``libgq.so``.
+
+    Unlike :func:`gq_objective` this wrapper allocates nothing either, so ``loss`` (fp64 ``[g + 1]`` on the
+    device) has to be passed in.  Only small layers fit (``d_in * d_out <= 2**20``); larger ones raise
+    ``GQ_ERR_UNSUPPORTED_SHAPE``.  Calls that overlap on the GPU share the scratch and race."""
+    _dev(W, torch.float32, "W")
+    _dev(W_hat, torch.float32, "W_hat")
+    _dev(H, torch.float32, "H")
+    _dev(loss, torch.float64, "loss")
+    if W.dim() != 2 or W.shape != W_hat.shape or not W.is_contiguous() or not W_hat.is_contiguous():
+        raise ValueError("W and W_hat must be contiguous [d_out, d_in]")
+    d_out, d_in = W.shape
+    g = H.shape[0]
+    if tuple(H.shape) != (g, d_in, d_in) or not H.is_contiguous() or loss.numel() != g + 1:
+        raise ValueError("H must be contiguous [g, d_in, d_in] and loss must have g + 1 entries")
+    rc = lib().gq_objective_noalloc(W.data_ptr(), W_hat.data_ptr(), d_in, d_out, H.data_ptr(), g, loss.data_ptr(),
+                                    _stream_ptr(stream))
+    if rc:
+        raise GQError("gq_objective_noalloc", rc)
+    return loss

@@ -379,6 +379,102 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     return GQ_OK;
 }
 
+// ------------------------------------------------------------------------------------------------
+// gq_objective_noalloc: the objective with its scratch in a fixed device array of this library.
+// Limits (see include/gq.h): d_in * d_out <= 2^20 weights, (tile slots) * g <= 4096 work units.
+#define GQ_NOALLOC_MAX_WEIGHTS (1ll << 20)
+#define GQ_NOALLOC_MAX_UNITS 4096ll
+#define GQ_NOALLOC_MATRIX_BYTES (GQ_NOALLOC_MAX_WEIGHTS * 2)                 /* one bf16 copy of delta */
+#define GQ_NOALLOC_PARTIAL_BYTES (GQ_NOALLOC_MAX_UNITS * 4 * 8)              /* 4 fp64 sums per unit   */
+#define GQ_NOALLOC_SCRATCH_BYTES (2 * GQ_NOALLOC_MATRIX_BYTES + GQ_NOALLOC_PARTIAL_BYTES)
+
+}  // extern "C"
+
+namespace {
+// Lives in every CUDA context that loads the library, from load until exit: 4 MiB + 128 KiB.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[GQ_NOALLOC_SCRATCH_BYTES];
+// Device address of g_noalloc_scratch per device, looked up once (the name above is only a handle
+// on the host side and must never be passed to a kernel as if it were an address).
+unsigned char *g_noalloc_scratch_ptr[kMaxDevices];
+std::mutex g_noalloc_mutex;
+}  // namespace
+
+extern "C" {
+
+int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, int64_t d_out, const float *H,
+                             int32_t g, double *loss_out, void *stream)
+{
+    if (!W || !W_hat || !H || !loss_out) return GQ_ERR_INVALID_ARG;
+    if (int32_t rc = check_layer_shape(d_in, d_out, g, true)) return rc;
+    if (!aligned(W, 16) || !aligned(W_hat, 16) || !aligned(H, 16) || !aligned(loss_out, 8)) return GQ_ERR_ALIGNMENT;
+    const int tile_slots = tile_slots_for(d_in);
+    if (d_in * d_out > GQ_NOALLOC_MAX_WEIGHTS || static_cast<int64_t>(tile_slots) * g > GQ_NOALLOC_MAX_UNITS)
+        return GQ_ERR_UNSUPPORTED_SHAPE;       // larger layers must use gq_objective with a caller workspace
+    DeviceInfo *di;
+    if (int32_t rc = device_info(&di)) return rc;
+
+    // One-time set-up per device (with that device current): ask the runtime where the array lives.
+    int dev = 0;
+    GQ_CUDA(cudaGetDevice(&dev));
+    unsigned char *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!g_noalloc_scratch_ptr[dev]) {
+            unsigned char *ptr = nullptr;
+            GQ_CUDA(cudaGetSymbolAddress(reinterpret_cast<void **>(&ptr), g_noalloc_scratch));
+            if (!ptr) {
+                tl_last_cuda_error = static_cast<int32_t>(cudaErrorInvalidSymbol);
+                return GQ_ERR_CUDA;
+            }
+            g_noalloc_scratch_ptr[dev] = ptr;
+        }
+        scratch = g_noalloc_scratch_ptr[dev];
+    }
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    __nv_bfloat16 *hi = reinterpret_cast<__nv_bfloat16 *>(scratch);
+    __nv_bfloat16 *lo = reinterpret_cast<__nv_bfloat16 *>(scratch + GQ_NOALLOC_MATRIX_BYTES);
+    double *partials = reinterpret_cast<double *>(scratch + 2 * GQ_NOALLOC_MATRIX_BYTES);
+    const int64_t m = d_out / g;
+    // Every scratch byte that is read below is written first by this same call (hi/lo by the split
+    // kernel, one partial per (unit, warp) by the Gram kernel), so what an earlier call left behind
+    // is never observed and nothing has to be cleared.
+    {
+        const long long count8 = d_in * d_out / 8;
+        const int grid = grid_for(count8, 256, di->sm_count, 8);
+        gq::split_delta_kernel<<<grid, 256, 0, st>>>(W, W_hat, count8, hi, lo);
+        g_launches.fetch_add(1);
+        GQ_CUDA(cudaGetLastError());
+    }
+    CUtensorMap mapHi, mapLo;
+    if (int32_t rc = make_map(&mapHi, hi, d_in, m, g, d_in, m * d_in)) return rc;
+    if (int32_t rc = make_map(&mapLo, lo, d_in, m, g, d_in, m * d_in)) return rc;
+    gq::GramParams p{};
+    p.d = static_cast<int>(d_in);
+    p.rows = static_cast<int>(m);
+    p.g = g;
+    p.n_terms = 3;
+    p.term_a[0] = 0; p.term_b[0] = 0;
+    p.term_a[1] = 0; p.term_b[1] = 1;
+    p.term_a[2] = 1; p.term_b[2] = 0;
+    p.map_grouped[0] = 1;
+    p.map_grouped[1] = 1;
+    p.tile_slots = tile_slots;
+    p.units = tile_slots * g;
+    p.H = const_cast<float *>(H);
+    p.partials = partials;
+    p.status = di->status_ptr;
+    p.wait_budget_ns = wait_budget_ns();
+    const int grid = p.units < di->sm_count ? p.units : di->sm_count;
+    gq::gram_kernel<gq::EPI_DOT><<<grid, gq::GRAM_THREADS, gq::GRAM_SMEM_BYTES, st>>>(mapHi, mapLo, p);
+    g_launches.fetch_add(1);
+    GQ_CUDA(cudaGetLastError());
+    gq::reduce_partials_kernel<<<1, 1024, 0, st>>>(partials, p.tile_slots, g, loss_out);
+    g_launches.fetch_add(1);
+    GQ_CUDA(cudaGetLastError());
+    return GQ_OK;
+}
+
 int32_t gq_kernel_timing_enable(int32_t enable)
 {
     std::lock_guard<std::mutex> lock(g_timing_mutex);
