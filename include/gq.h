@@ -82,13 +82,18 @@ int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad,
  *              first chunk and keeps it resident between chunks.  After any number of calls only
  *              entries with a <= b are defined; entries below the diagonal hold unspecified finite
  *              values until gq_hessian_finalize() is called.
- *   flags      must be 0
+ *   flags      0, or GQ_HESSIAN_DETERMINISTIC (see below)
  *   workspace  device scratch of at least gq_hessian_workspace_bytes(n_max, d_in, g, flags)
  *              bytes, 1024-byte aligned; contents need not be preserved between calls.
  * Arithmetic: rows of X are multiplied by s_k in fp32 and rounded to bf16 once; products are
- * accumulated in fp32 on the tensor cores; each call adds its fp32 tile sums to H.  Every element
- * of H has a single writer, so results are bit-reproducible run to run.
+ * accumulated in fp32 on the tensor cores; each call adds its fp32 tile sums to H.
+ * Work is dealt to the SM pairs in whole 256 x 256 tiles; with flags == 0 the last, incomplete round
+ * of tiles is cut along the token axis so that every SM pair gets the same amount of work, and the
+ * pieces of such a tile are added to H with floating-point atomics: those entries can differ in the
+ * last bit from run to run.  With GQ_HESSIAN_DETERMINISTIC every element of H has a single writer
+ * and results are bit-reproducible run to run, at the price of an idle tail in the last round.
  */
+#define GQ_HESSIAN_DETERMINISTIC 1u
 int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld_x, const float *s,
                               int64_t ld_s, int32_t g, float *H, uint32_t flags, void *workspace,
                               size_t workspace_bytes, void *stream);
@@ -157,10 +162,10 @@ size_t gq_layer_host_arena_bytes(int64_t chunk, int64_t d_in, int64_t d_out, int
  * loop where an allocation (and the implicit synchronisation of a free) is not acceptable.  For them
  * this entry point keeps its scratch in a fixed array inside the library's own device image:
  *
- *   - the array is 4 MiB + 128 KiB (two bf16 copies of W - W_hat and the partial sums); every GPU on
+ *   - the array is 4 MiB + 256 KiB (two bf16 copies of W - W_hat and the partial sums); every GPU on
  *     which the library is used holds that much from the moment the library is loaded until exit;
  *   - therefore only small layers fit: d_in * d_out <= 1,048,576 weights and
- *     (NJ * NJ + NJ) * g <= 4096 with NJ = ceil(d_in / 256).  Anything larger returns
+ *     NJ * (NJ + 1) / 2 * g <= 4096 with NJ = ceil(d_in / 256).  Anything larger returns
  *     GQ_ERR_UNSUPPORTED_SHAPE and launches nothing: use gq_objective with your own workspace;
  *   - the call makes no cudaMalloc / cudaFree and no call into an allocating library.  The first
  *     call on each device looks up the array's device address once (cudaGetSymbolAddress) and sets

@@ -24,6 +24,7 @@ EXPORTS = (
     "gq_layer_objective_host", "gq_layer_host_arena_bytes", "gq_check", "gq_launch_count",
     "gq_kernel_timing_enable", "gq_kernel_timing_read", "gq_objective_noalloc",
 )
+GQ_HESSIAN_DETERMINISTIC = 1      # flag of gq_hessian_accumulate: single writer per element of H
 KERNEL_NAMES = ("saliency", "scale_rows", "gram_accum", "mirror", "split_delta", "gram_dot", "reduce")
 
 

@@ -149,18 +149,18 @@ split_delta_kernel(const float *__restrict__ W, const float *__restrict__ What, 
 }
 
 // ------------------------------------------------------------------------------------------------
-// loss[k] = sum over the group's tile partials (fixed order), loss[g] = sum_k loss[k].  One block.
-// partials: [tile_slots][g][4].
+// loss[k] = sum over the group's partial sums (fixed order), loss[g] = sum_k loss[k].  One block.
+// partials: [tiles][g][per_unit].
 __global__ void __launch_bounds__(1024)
-reduce_partials_kernel(const double *__restrict__ partials, int tile_slots, int g, double *__restrict__ loss)
+reduce_partials_kernel(const double *__restrict__ partials, int tiles, int g, int per_unit, double *__restrict__ loss)
 {
     __shared__ double red[1024];
     double total = 0.0;
     for (int k = 0; k < g; ++k) {
         double acc = 0.0;
-        for (int idx = threadIdx.x; idx < tile_slots * 4; idx += blockDim.x) {
-            const int t = idx >> 2, q = idx & 3;
-            acc += partials[(static_cast<size_t>(t) * g + k) * 4 + q];
+        for (int idx = threadIdx.x; idx < tiles * per_unit; idx += blockDim.x) {
+            const int t = idx / per_unit, q = idx - t * per_unit;
+            acc += partials[(static_cast<size_t>(t) * g + k) * per_unit + q];
         }
         red[threadIdx.x] = acc;
         __syncthreads();

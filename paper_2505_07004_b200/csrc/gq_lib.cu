@@ -62,6 +62,7 @@ __device__ uint32_t g_status_word[4];
 struct DeviceInfo {
     bool ready = false;
     int sm_count = 0;
+    int max_pairs = 0;          // CTA pairs (clusters of two) of the Gram kernel that can be resident at once
     uint32_t *status_ptr = nullptr;
 };
 DeviceInfo g_dev[kMaxDevices];
@@ -96,6 +97,28 @@ int32_t device_info(DeviceInfo **out)
                                      gq::GRAM_SMEM_BYTES));
         GQ_CUDA(cudaFuncSetAttribute(gq::gram_kernel<gq::EPI_DOT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      gq::GRAM_SMEM_BYTES));
+        {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(static_cast<unsigned>(di.sm_count & ~1));
+            cfg.blockDim = dim3(gq::GRAM_THREADS);
+            cfg.dynamicSmemBytes = gq::GRAM_SMEM_BYTES;
+            cudaLaunchAttribute attr;
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = 2;
+            attr.val.clusterDim.y = 1;
+            attr.val.clusterDim.z = 1;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            int clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&clusters, gq::gram_kernel<gq::EPI_ACCUM>, &cfg) != cudaSuccess ||
+                clusters < 1) {
+                (void)cudaGetLastError();
+                clusters = di.sm_count / 2;
+            }
+            if (clusters > di.sm_count / 2) clusters = di.sm_count / 2;
+            if (clusters < 1) clusters = 1;
+            di.max_pairs = clusters;
+        }
         if (!g_encode) {
             void *fn = nullptr;
             cudaDriverEntryPointQueryResult qres;
@@ -153,10 +176,11 @@ int grid_for(long long work_items, int threads, int sm_count, int blocks_per_sm)
     return static_cast<int>(blocks);
 }
 
-int tile_slots_for(int64_t d)
+// Number of 256 x 256 tiles that touch the upper triangle of a d x d matrix.
+int tiles_for(int64_t d)
 {
     const int64_t nj = (d + gq::TILE_N - 1) / gq::TILE_N;
-    return static_cast<int>(nj * nj + nj);
+    return static_cast<int>(nj * (nj + 1) / 2);
 }
 
 int32_t check_layer_shape(int64_t d_in, int64_t d_out, int32_t g, bool need_out)
@@ -185,7 +209,8 @@ ObjectiveLayout objective_layout(int64_t d_in, int64_t d_out, int32_t g)
     L.hi_off = 0;
     L.lo_off = mat;
     L.partials_off = 2 * mat;
-    L.total = L.partials_off + round_up(static_cast<size_t>(tile_slots_for(d_in)) * g * 4 * sizeof(double), 1024);
+    L.total = L.partials_off +
+              round_up(static_cast<size_t>(tiles_for(d_in)) * g * gq::PARTIALS_PER_UNIT * sizeof(double), 1024);
     return L;
 }
 
@@ -240,7 +265,9 @@ int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad,
 
 size_t gq_hessian_workspace_bytes(int64_t n_max, int64_t d_in, int32_t g, uint32_t flags)
 {
-    if (flags != 0 || n_max < 0 || check_layer_shape(d_in, 0, g, false) != GQ_OK) return 0;
+    if ((flags & ~static_cast<uint32_t>(GQ_HESSIAN_DETERMINISTIC)) != 0 || n_max < 0 ||
+        check_layer_shape(d_in, 0, g, false) != GQ_OK)
+        return 0;
     return hessian_ws_bytes(n_max, d_in, g);
 }
 
@@ -248,7 +275,8 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
                               int32_t g, float *H, uint32_t flags, void *workspace, size_t workspace_bytes,
                               void *stream)
 {
-    if (n < 0 || ld_x < d_in || ld_s < n || flags != 0) return GQ_ERR_INVALID_ARG;
+    if (n < 0 || ld_x < d_in || ld_s < n || (flags & ~static_cast<uint32_t>(GQ_HESSIAN_DETERMINISTIC)) != 0)
+        return GQ_ERR_INVALID_ARG;
     if (int32_t rc = check_layer_shape(d_in, 0, g, false)) return rc;
     if (n > (1ll << 31) - 64) return GQ_ERR_UNSUPPORTED_SHAPE;
     if (ld_x % 8 != 0) return GQ_ERR_ALIGNMENT;
@@ -284,13 +312,17 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
     p.term_b[0] = 1;
     p.map_grouped[0] = 0;
     p.map_grouped[1] = 1;
-    p.tile_slots = tile_slots_for(d_in);
-    p.units = p.tile_slots * g;
+    const int units = tiles_for(d_in) * g;
+    const int ksteps = static_cast<int>((n + gq::TILE_K - 1) / gq::TILE_K);
+    const bool balanced = (flags & GQ_HESSIAN_DETERMINISTIC) == 0;
+    int pairs = di->max_pairs;
+    if (!balanced && units < pairs) pairs = units;
+    gq::plan_schedule(p, units, ksteps, pairs, balanced);
     p.H = H;
     p.partials = nullptr;
     p.status = di->status_ptr;
     p.wait_budget_ns = wait_budget_ns();
-    const int grid = p.units < di->sm_count ? p.units : di->sm_count;
+    const int grid = 2 * ((p.full_waves == 0 && p.tail_pairs > 0) ? p.tail_pairs : pairs);
     {
         LaunchScope scope(GQ_KERNEL_GRAM_ACCUM, st);
         gq::gram_kernel<gq::EPI_ACCUM><<<grid, gq::GRAM_THREADS, gq::GRAM_SMEM_BYTES, st>>>(mapX, mapY, p);
@@ -359,13 +391,15 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     p.term_a[2] = 1; p.term_b[2] = 0;
     p.map_grouped[0] = 1;
     p.map_grouped[1] = 1;
-    p.tile_slots = tile_slots_for(d_in);
-    p.units = p.tile_slots * g;
+    const int tiles = tiles_for(d_in);
+    const int units = tiles * g;
+    const int ksteps = 3 * static_cast<int>((m + gq::TILE_K - 1) / gq::TILE_K);
+    gq::plan_schedule(p, units, ksteps, units < di->max_pairs ? units : di->max_pairs, false);
     p.H = const_cast<float *>(H);
     p.partials = partials;
     p.status = di->status_ptr;
     p.wait_budget_ns = wait_budget_ns();
-    const int grid = p.units < di->sm_count ? p.units : di->sm_count;
+    const int grid = 2 * p.pairs;
     {
         LaunchScope scope(GQ_KERNEL_GRAM_DOT, st);
         gq::gram_kernel<gq::EPI_DOT><<<grid, gq::GRAM_THREADS, gq::GRAM_SMEM_BYTES, st>>>(mapHi, mapLo, p);
@@ -373,7 +407,7 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     GQ_CUDA(cudaGetLastError());
     {
         LaunchScope scope(GQ_KERNEL_REDUCE, st);
-        gq::reduce_partials_kernel<<<1, 1024, 0, st>>>(partials, p.tile_slots, g, loss_out);
+        gq::reduce_partials_kernel<<<1, 1024, 0, st>>>(partials, tiles, g, gq::PARTIALS_PER_UNIT, loss_out);
     }
     GQ_CUDA(cudaGetLastError());
     return GQ_OK;
@@ -381,17 +415,17 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
 
 // ------------------------------------------------------------------------------------------------
 // gq_objective_noalloc: the objective with its scratch in a fixed device array of this library.
-// Limits (see include/gq.h): d_in * d_out <= 2^20 weights, (tile slots) * g <= 4096 work units.
+// Limits (see include/gq.h): d_in * d_out <= 2^20 weights, (256 x 256 tiles) * g <= 4096 work units.
 #define GQ_NOALLOC_MAX_WEIGHTS (1ll << 20)
 #define GQ_NOALLOC_MAX_UNITS 4096ll
 #define GQ_NOALLOC_MATRIX_BYTES (GQ_NOALLOC_MAX_WEIGHTS * 2)                 /* one bf16 copy of delta */
-#define GQ_NOALLOC_PARTIAL_BYTES (GQ_NOALLOC_MAX_UNITS * 4 * 8)              /* 4 fp64 sums per unit   */
+#define GQ_NOALLOC_PARTIAL_BYTES (GQ_NOALLOC_MAX_UNITS * 8 * 8)              /* 8 fp64 sums per unit   */
 #define GQ_NOALLOC_SCRATCH_BYTES (2 * GQ_NOALLOC_MATRIX_BYTES + GQ_NOALLOC_PARTIAL_BYTES)
 
 }  // extern "C"
 
 namespace {
-// Lives in every CUDA context that loads the library, from load until exit: 4 MiB + 128 KiB.
+// Lives in every CUDA context that loads the library, from load until exit: 4 MiB + 256 KiB.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[GQ_NOALLOC_SCRATCH_BYTES];
 // Device address of g_noalloc_scratch per device, looked up once (the name above is only a handle
 // on the host side and must never be passed to a kernel as if it were an address).
@@ -407,8 +441,8 @@ int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, i
     if (!W || !W_hat || !H || !loss_out) return GQ_ERR_INVALID_ARG;
     if (int32_t rc = check_layer_shape(d_in, d_out, g, true)) return rc;
     if (!aligned(W, 16) || !aligned(W_hat, 16) || !aligned(H, 16) || !aligned(loss_out, 8)) return GQ_ERR_ALIGNMENT;
-    const int tile_slots = tile_slots_for(d_in);
-    if (d_in * d_out > GQ_NOALLOC_MAX_WEIGHTS || static_cast<int64_t>(tile_slots) * g > GQ_NOALLOC_MAX_UNITS)
+    const int tiles = tiles_for(d_in);
+    if (d_in * d_out > GQ_NOALLOC_MAX_WEIGHTS || static_cast<int64_t>(tiles) * g > GQ_NOALLOC_MAX_UNITS)
         return GQ_ERR_UNSUPPORTED_SHAPE;       // larger layers must use gq_objective with a caller workspace
     DeviceInfo *di;
     if (int32_t rc = device_info(&di)) return rc;
@@ -459,17 +493,18 @@ int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, i
     p.term_a[2] = 1; p.term_b[2] = 0;
     p.map_grouped[0] = 1;
     p.map_grouped[1] = 1;
-    p.tile_slots = tile_slots;
-    p.units = tile_slots * g;
+    const int units = tiles * g;
+    const int ksteps = 3 * static_cast<int>((m + gq::TILE_K - 1) / gq::TILE_K);
+    gq::plan_schedule(p, units, ksteps, units < di->max_pairs ? units : di->max_pairs, false);
     p.H = const_cast<float *>(H);
     p.partials = partials;
     p.status = di->status_ptr;
     p.wait_budget_ns = wait_budget_ns();
-    const int grid = p.units < di->sm_count ? p.units : di->sm_count;
+    const int grid = 2 * p.pairs;
     gq::gram_kernel<gq::EPI_DOT><<<grid, gq::GRAM_THREADS, gq::GRAM_SMEM_BYTES, st>>>(mapHi, mapLo, p);
     g_launches.fetch_add(1);
     GQ_CUDA(cudaGetLastError());
-    gq::reduce_partials_kernel<<<1, 1024, 0, st>>>(partials, p.tile_slots, g, loss_out);
+    gq::reduce_partials_kernel<<<1, 1024, 0, st>>>(partials, tiles, g, gq::PARTIALS_PER_UNIT, loss_out);
     g_launches.fetch_add(1);
     GQ_CUDA(cudaGetLastError());
     return GQ_OK;

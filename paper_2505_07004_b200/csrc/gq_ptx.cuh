@@ -1,6 +1,7 @@
 // Thin inline-PTX wrappers for the sm_100a features the kernels use:
-// mbarrier, TMA tiled loads (cp.async.bulk.tensor), tcgen05 (TMEM alloc, MMA, commit, ld).
-// No multicast form of any copy is used anywhere in this library.
+// clusters of two CTAs, mbarrier, TMA tiled loads (cp.async.bulk.tensor), tcgen05 with a CTA pair
+// (TMEM alloc, MMA, commit, ld).  No copy in this library uses a multicast form; the only multicast
+// is the mbarrier arrival of tcgen05.commit, which signals both CTAs of a pair.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -30,6 +31,34 @@ __device__ __forceinline__ bool elect_one()
     return pred != 0;
 }
 
+// ---------------------------------------------------------------- cluster of two CTAs
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Address of this CTA's shared-memory location `addr` as seen in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+// Barrier over all threads of both CTAs (the non-.aligned forms: callers may arrive from divergent code).
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+
+// ---------------------------------------------------------------- global memory
+// dst[0..3] += {a, b, c, d} performed by the memory system (no value returned); dst 16-byte aligned.
+__device__ __forceinline__ void red_add_f32x4(float *dst, float a, float b, float c, float d)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
@@ -51,6 +80,24 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// Arrive on a barrier that lives in another (or this) CTA of the cluster; `cluster_addr` from map_to_cta.
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Wait variant that pairs with mbar_arrive_cluster (acquire at cluster scope).
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
@@ -69,30 +116,33 @@ __device__ __forceinline__ void prefetch_tensormap(const void *map)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
-// 3-D tiled load global -> this CTA's shared memory, completion on an mbarrier.
+// 3-D tiled load global -> this CTA's shared memory.  The bytes are counted on the mbarrier at
+// `bar_cluster_addr`, which may belong to the other CTA of the pair (cta_group::2 form).
 // c0 (innermost coordinate) times the element size must be a multiple of 16 bytes.
-__device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const void *map, uint32_t bar, int32_t c0,
-                                            int32_t c1, int32_t c2)
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t smem_dst, const void *map, uint32_t bar_cluster_addr,
+                                                 int32_t c0, int32_t c1, int32_t c2)
 {
     asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
 
-// ---------------------------------------------------------------- tcgen05 / TMEM
+// ---------------------------------------------------------------- tcgen05 / TMEM (CTA pair)
+// Allocation, release of the permit and deallocation are each executed by one warp of BOTH CTAs.
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_result, uint32_t ncols)
 {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols)
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols)
                  : "memory");
 }
 __device__ __forceinline__ void tmem_relinquish()
 {
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
 {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before_sync()
 {
@@ -102,21 +152,33 @@ __device__ __forceinline__ void tc_fence_after_sync()
 {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate; issued by one thread.
+// D[tmem] (+)= A[smem] * B[smem] over the CTA pair: bf16 inputs, fp32 accumulate, M = 256 (128 rows of
+// A and of D per CTA), each CTA supplies half of the N columns of B.  Issued by one thread of the
+// pair's first CTA; the descriptors hold addresses in that CTA and the same offsets are used in its peer.
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                           uint32_t accumulate)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-// Arrive (count 1) on an mbarrier once every tcgen05.mma issued so far by this thread has finished.
-__device__ __forceinline__ void umma_commit(uint32_t bar)
+// Arrive (count 1) on the mbarrier at the same shared-memory offset in BOTH CTAs of the pair once
+// every tcgen05.mma issued so far by this thread has finished.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    const uint16_t mask = 3;
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"(mask)
+        : "memory");
+}
+// Same, but only the issuing CTA's barrier is signalled.
+__device__ __forceinline__ void umma_commit_local(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 // 32 lanes x 32 consecutive 32-bit columns: thread t of the warp receives lane (base lane + t).
 __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])

@@ -45,12 +45,13 @@ def test_workspace_sizes(L):
     # scaled operands: g * n_max * d_in bf16
     assert L.gq_hessian_workspace_bytes(8192, 4096, 4, 0) == 4 * 8192 * 4096 * 2
     assert L.gq_hessian_workspace_bytes(1, 8, 1, 0) == 1024            # rounded up to 1 KiB
-    assert L.gq_hessian_workspace_bytes(8192, 4096, 4, 1) == 0         # unknown flag
+    assert L.gq_hessian_workspace_bytes(8192, 4096, 4, 1) == 4 * 8192 * 4096 * 2   # GQ_HESSIAN_DETERMINISTIC
+    assert L.gq_hessian_workspace_bytes(8192, 4096, 4, 2) == 0         # unknown flag
     assert L.gq_hessian_workspace_bytes(8192, 4100, 4, 0) == 0         # d_in % 8 != 0
     assert L.gq_hessian_workspace_bytes(8192, 4096, 0, 0) == 0
-    # objective: two bf16 copies of delta + 4 fp64 partial sums per (tile slot, group)
+    # objective: two bf16 copies of delta + 8 fp64 partial sums per (upper-triangular 256 x 256 tile, group)
     nj = 4096 // 256
-    assert L.gq_objective_workspace_bytes(4096, 4096, 4) == 2 * 4096 * 4096 * 2 + (nj * nj + nj) * 4 * 4 * 8
+    assert L.gq_objective_workspace_bytes(4096, 4096, 4) == 2 * 4096 * 4096 * 2 + (nj * (nj + 1) // 2) * 4 * 8 * 8
     assert L.gq_objective_workspace_bytes(4096, 4096, 3) == 0          # d_out % g != 0
     assert L.gq_objective_workspace_bytes(4096, 24, 6) == 0            # (d_out / g) % 8 != 0
     assert L.gq_layer_host_arena_bytes(0, 4096, 4096, 4) == 0
@@ -73,7 +74,7 @@ def test_host_side_validation_needs_no_gpu(L):
     assert L.gq_saliency(None, 4, 64, 64, 2, 1.0, p16, 4, None) == INVALID
     assert L.gq_saliency(None, 0, 64, 64, 2, 1.0, None, 0, None) == 0          # empty call: no-op
     # hessian
-    assert L.gq_hessian_accumulate(p16, 4, 64, 64, p16, 4, 2, p16, 1, p16, 4096, None) == INVALID   # flags
+    assert L.gq_hessian_accumulate(p16, 4, 64, 64, p16, 4, 2, p16, 2, p16, 4096, None) == INVALID   # flags
     assert L.gq_hessian_accumulate(p16, 4, 60, 64, p16, 4, 2, p16, 0, p16, 4096, None) == SHAPE     # d_in % 8
     assert L.gq_hessian_accumulate(p16, 4, 64, 64, p16, 4, 2, p16, 0, None, 0, None) == WS
     assert L.gq_hessian_accumulate(p16, 4, 64, 64, p16, 4, 2, p16 + 4, 0, p16, 4096, None) == ALIGN
