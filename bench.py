@@ -265,7 +265,7 @@ def run_ours(args, cfg, g):
         value = shard.whole_job_throughput(cfg.n, args.steps, ms_total * 1e-3, world)
         e2e_value = shard.whole_job_throughput(cfg.n, e2e_steps, e2e_ms * 1e-3, world) if e2e_steps else None
         # dominant kernel: the tensor-core Gram kernel of gq_hessian_accumulate
-        ga_ms, ga_n = kern["gram_accum"]
+        ga_ms, ga_n = kern["hessian"]
         flops_per_launch = float(g) * cfg.chunk * cfg.d_in * (cfg.d_in + 1)      # upper triangle, mul + add
         achieved = flops_per_launch / (ga_ms / max(1, ga_n) * 1e-3) / 1e12 if ga_n else None
         peak = peaks["bf16_tflops_sustained"]
@@ -283,7 +283,7 @@ def run_ours(args, cfg, g):
                              % ((cfg.n * (cfg.d_in + cfg.d_out) * 2) / 1e9),
                        "parallelism": "one layer per GPU, no collective"},
             "hessian_tflops_useful": (float(g) * cfg.n * cfg.d_in * (cfg.d_in + 1)) * world * args.steps / (ms_total * 1e-3) / 1e12,
-            "roofline": {"kernel": "gram_kernel<EPI_ACCUM> (gq_hessian_accumulate)", "bound": "tensor",
+            "roofline": {"kernel": "hessian_kernel (gq_hessian_accumulate)", "bound": "tensor",
                          "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                          "frac": (achieved / peak) if achieved else None,
                          "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),

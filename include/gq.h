@@ -198,13 +198,12 @@ uint64_t gq_launch_count(void);
  */
 enum gq_kernel_id {
     GQ_KERNEL_SALIENCY = 0,    /* Algorithm 1 line 2                                    */
-    GQ_KERNEL_SCALE_ROWS = 1,  /* Diag(s_k) X, bf16                                      */
-    GQ_KERNEL_GRAM_ACCUM = 2,  /* tensor-core X^T (Diag(s_k) X), H += (Algorithm 1 l. 4) */
-    GQ_KERNEL_MIRROR = 3,      /* gq_hessian_finalize                                    */
-    GQ_KERNEL_SPLIT_DELTA = 4, /* W - W_hat -> bf16 hi/lo                                */
-    GQ_KERNEL_GRAM_DOT = 5,    /* tensor-core Delta_k^T Delta_k contracted with H_k (Eq. 7) */
-    GQ_KERNEL_REDUCE = 6,      /* fp64 reduction of the partial sums                     */
-    GQ_KERNEL_COUNT = 7
+    GQ_KERNEL_HESSIAN = 1,     /* tensor-core H += X^T Diag(s_k) X, scaling fused (Algorithm 1 l. 4) */
+    GQ_KERNEL_MIRROR = 2,      /* gq_hessian_finalize                                    */
+    GQ_KERNEL_SPLIT_DELTA = 3, /* W - W_hat -> bf16 hi/lo                                */
+    GQ_KERNEL_GRAM_DOT = 4,    /* tensor-core Delta_k^T Delta_k contracted with H_k (Eq. 7) */
+    GQ_KERNEL_REDUCE = 5,      /* fp64 reduction of the partial sums                     */
+    GQ_KERNEL_COUNT = 6
 };
 
 /*

@@ -60,6 +60,16 @@ constexpr int EPI_DOT = 1;
 
 constexpr uint32_t STATUS_TIMEOUT = 6;   // stored in the status word; the host maps it to GQ_ERR_TIMEOUT
 
+// How the work units of a launch are dealt to the CTA pairs.
+struct Schedule {
+    int units;               // work units of the launch
+    int ksteps;              // k-steps (of 64 contraction rows) of one whole unit
+    int pairs;               // CTA pairs in the grid
+    int full_waves;          // rounds of whole units dealt round-robin
+    int tail_units;          // units after the full rounds (0 <= tail_units < pairs), cut into pieces
+    int tail_pairs;          // pairs that take a piece of the tail
+};
+
 struct GramParams {
     int d;                   // number of features (d_in)
     int rows;                // contraction length of every term
@@ -68,12 +78,8 @@ struct GramParams {
     int term_a[MAX_TERMS];   // which tensor map (0/1) feeds A / B in each term
     int term_b[MAX_TERMS];
     int map_grouped[2];      // 1: the map's third coordinate is the group index; 0: always 0
-    int units;               // (number of upper-triangular 256 x 256 tiles) * g
-    int ksteps;              // k-steps of one whole unit: n_terms * ceil(rows / 64)
-    int pairs;               // CTA pairs in the grid
-    int full_waves;          // rounds of whole units dealt round-robin
-    int tail_units;          // units after the full rounds (0 <= tail_units < pairs), cut into pieces
-    int tail_pairs;          // pairs that take a piece of the tail
+    Schedule sched;          // units = (number of upper-triangular 256 x 256 tiles) * g,
+                             // ksteps = n_terms * ceil(rows / 64)
     float *H;                // [g][d][d]
     double *partials;        // EPI_DOT: [units][PARTIALS_PER_UNIT]
     uint32_t *status;        // device status word (4 x u32)
@@ -81,8 +87,9 @@ struct GramParams {
 };
 
 // Host side: fills the distribution fields.  `balanced` cuts the last, incomplete round into pieces.
-inline void plan_schedule(GramParams &p, int units, int ksteps, int pairs, bool balanced)
+inline Schedule plan_schedule(int units, int ksteps, int pairs, bool balanced)
 {
+    Schedule p;
     p.units = units;
     p.ksteps = ksteps;
     p.pairs = pairs;
@@ -98,6 +105,7 @@ inline void plan_schedule(GramParams &p, int units, int ksteps, int pairs, bool 
         if (tp > pairs) tp = pairs;
         p.tail_pairs = static_cast<int>(tp);
     }
+    return p;
 }
 
 // Slot t of the triangular enumeration -> (row block i, column block j) of 256 x 256 tiles with i <= j,
@@ -119,7 +127,7 @@ struct WorkItem {
 
 // The `it`-th work item of pair `pair`; false when the pair has no more work.  Every role of both CTAs of
 // a pair walks the same list.
-__device__ __forceinline__ bool work_item(const GramParams &p, int pair, int it, WorkItem &w)
+__device__ __forceinline__ bool work_item(const Schedule &p, int pair, int it, WorkItem &w)
 {
     if (it < p.full_waves) {
         w.unit = it * p.pairs + pair;
@@ -150,35 +158,52 @@ struct WaitCtx {
     unsigned long long budget_ns;
 };
 
-template <bool CLUSTER_SCOPE>
+__device__ __forceinline__ bool wait_gave_up(const WaitCtx &w, uint64_t t0, uint32_t site, uint32_t unit)
+{
+    if (*w.abort_flag) return true;
+    if (global_timer_ns() - t0 > w.budget_ns) {
+        *w.abort_flag = 1u;
+        if (atomicCAS(&w.status[0], 0u, STATUS_TIMEOUT) == 0u) {
+            w.status[1] = site;
+            w.status[2] = blockIdx.x;
+            w.status[3] = unit;
+        }
+        __threadfence();
+        return true;
+    }
+    return false;
+}
+
+// Slow path of bounded_wait: the thread sleeps inside try_wait (woken when the phase completes) and looks at
+// the clock and the abort flag between sleeps.
 __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const WaitCtx &w, uint32_t site, uint32_t unit)
 {
     const uint64_t t0 = global_timer_ns();
-    uint32_t spins = 0;
     for (;;) {
-        if (CLUSTER_SCOPE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 31u) == 0u) {
-            if (*w.abort_flag) return false;
-            if (global_timer_ns() - t0 > w.budget_ns) {
-                *w.abort_flag = 1u;
-                if (atomicCAS(&w.status[0], 0u, STATUS_TIMEOUT) == 0u) {
-                    w.status[1] = site;
-                    w.status[2] = blockIdx.x;
-                    w.status[3] = unit;
-                }
-                __threadfence();
-                return false;
-            }
-        }
+        if (mbar_try_wait_suspend(bar, parity, 2000u)) return true;
+        if (wait_gave_up(w, t0, site, unit)) return false;
     }
 }
 
-template <bool CLUSTER_SCOPE = false>
+// Wait for roles that are ahead of the tensor core (producer, scalers, epilogue).
 __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, const WaitCtx &w, uint32_t site,
                                              uint32_t unit)
 {
-    if (CLUSTER_SCOPE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
-    return wait_slow<CLUSTER_SCOPE>(bar, parity, w, site, unit);
+    if (mbar_try_wait(bar, parity)) return true;
+    return wait_slow(bar, parity, w, site, unit);
+}
+
+// Wait for the MMA issuer, the one thread whose reaction time is on the critical path: polls without pause.
+__device__ __noinline__ bool bounded_wait_hot(uint32_t bar, uint32_t parity, const WaitCtx &w, uint32_t site,
+                                             uint32_t unit)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    uint32_t spins = 0;
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 63u) == 0u && wait_gave_up(w, t0, site, unit)) return false;
+    }
 }
 
 __device__ __forceinline__ void spin_ns(unsigned long long ns)
@@ -240,7 +265,7 @@ gram_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CU
         uint32_t issued = 0;
         bool ok = true;
         WorkItem w;
-        for (int it = 0; ok && work_item(p, pair, it, w); ++it) {
+        for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
             int ti, tj;
             tile_of_slot(w.unit / p.g, ti, tj);
             const int k = w.unit % p.g;
@@ -287,12 +312,12 @@ gram_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CU
         uint32_t acc_ph = 0;
         bool ok = true;
         WorkItem w;
-        for (int it = 0; ok && work_item(p, pair, it, w); ++it) {
-            if (!bounded_wait<true>(smem_u32(&bar_acc_empty[buf]), acc_ph ^ 1u, wc, 2u, w.unit)) { ok = false; break; }
+        for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
+            if (!bounded_wait_hot(smem_u32(&bar_acc_empty[buf]), acc_ph ^ 1u, wc, 2u, w.unit)) { ok = false; break; }
             tc_fence_after_sync();
             const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * TILE_N);
             for (int ks = w.ks0; ks < w.ks1; ++ks) {
-                if (!bounded_wait(smem_u32(&bar_full[s]), ph, wc, 3u, w.unit)) { ok = false; break; }
+                if (!bounded_wait_hot(smem_u32(&bar_full[s]), ph, wc, 3u, w.unit)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t sa = ring + s * STAGE_BYTES;
                 const uint32_t sb = sa + A_STAGE_BYTES;
@@ -323,7 +348,7 @@ gram_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CU
         uint32_t acc_ph = 0;
         bool ok = true;
         WorkItem w;
-        for (int it = 0; ok && work_item(p, pair, it, w); ++it) {
+        for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
             int ti, tj;
             tile_of_slot(w.unit / p.g, ti, tj);
             const int k = w.unit % p.g;

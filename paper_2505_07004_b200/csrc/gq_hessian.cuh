@@ -1,0 +1,391 @@
+// Guided Hessian of Algorithm 1 line 4 with the row scaling fused into the operand path:
+//
+//     H_k[a][b] += sum_i  (s_k[i] * X[i][a]) * X[i][b]          for a <= b, all groups k
+//
+// Tokens i are the contraction index, features are contiguous in memory, so both MMA operands are
+// MN-major bf16.  The kernel runs as CTA pairs (clusters of two); a pair owns one 256 x 256 tile of H for
+// TWO groups at a time (2 x 256 fp32 accumulator columns = all of tensor memory), so that one pass over
+// the tile's rows of X serves two groups and no scaled copy of X ever exists in global memory:
+//
+//   B operand  raw X[tokens, tile columns]: TMA boxes (64 tokens x 64 features, 128-byte swizzle),
+//              16 KB per CTA and k-step, shared by both groups
+//   A operand  s_k[token] * X[token, tile rows], one 16 KB block per group and k-step: twelve "scaler" warps
+//              in three sets that take k-steps in turn (so three k-steps of loads are in flight) read the raw
+//              rows straight from global memory with 128-bit loads, multiply by s_k (carried as two bf16
+//              terms, packed bf16 fused multiply-adds, one final rounding to bf16) and store into shared
+//              memory in exactly the swizzled layout a TMA load would have produced
+//   MMA        the pair's first CTA issues, per k-step and group, four tcgen05.mma.cta_group::2
+//              (M = 256, N = 256, K = 16) with fp32 accumulation in tensor memory
+//   epilogue   eight warps per CTA move the accumulators to H: tcgen05.ld -> swizzled staging block in
+//              shared memory -> TMA reduce-add (cp.reduce.async.bulk.tensor ... .add) of 32 x 32 fp32
+//              blocks, so H is never read by the SMs and every access to it is a full 128-byte row segment
+//
+// Per CTA and k-step (1024 tensor-core clocks for two groups) this moves 32 KB from L2 (half of what a
+// per-group pass over pre-scaled operands needs) and 112 KB through shared memory.
+//
+// Warps: 0 TMA producer (one lane) | 1 MMA issuer (one lane, first CTA) | 2 TMEM allocation | 3 idle |
+//        4..15 scalers | 16..23 epilogue.
+// Work units are (tile, pair of groups); they are dealt to the CTA pairs as described in gq_gram.cuh
+// (round-robin rounds, then the incomplete last round cut along the token axis).  Because H is updated
+// by reduce-adds only, pieces of a cut unit need no special treatment.
+//
+// The accumulators are single-buffered: after the last k-step of a unit the MMA issuer waits until the
+// epilogue warps have read them out of tensor memory (not until H is updated).  Producer and scalers run
+// ahead into the next unit meanwhile, so the pipeline is full again when the MMAs resume.
+//
+// Every mbarrier wait is bounded (see gq_gram.cuh).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gq_gram.cuh"
+
+namespace gq {
+
+constexpr int HS_STAGES = 4;
+constexpr int HS_GROUPS = 2;                                   // groups resident in tensor memory at once
+constexpr int HS_B_BYTES = (CTA_ROWS / BOX_FEATURES) * BOX_BYTES;            // 16 KB
+constexpr int HS_A_BYTES = (CTA_ROWS / BOX_FEATURES) * BOX_BYTES;            // 16 KB per group
+constexpr int HS_STAGE_BYTES = HS_B_BYTES + HS_GROUPS * HS_A_BYTES;          // 48 KB
+constexpr int HS_SETS = 3;                                     // independent scaler sets (k-steps in flight)
+constexpr int HS_SET_WARPS = 4;                                // warps per set: 128 threads cover 8 tokens x 128 features
+constexpr int HS_SCALER_WARPS = HS_SETS * HS_SET_WARPS;
+constexpr int HS_EPI_WARPS = 8;
+constexpr int HS_STAGING_BYTES = HS_EPI_WARPS * 4096;          // one 32 x 32 fp32 block per epilogue warp
+constexpr int HS_THREADS = 32 * (4 + HS_SCALER_WARPS + HS_EPI_WARPS);
+constexpr int HS_SMEM_BYTES = HS_STAGES * HS_STAGE_BYTES + HS_STAGING_BYTES + 1024;
+
+struct HessianParams {
+    const __nv_bfloat16 *X;  // [n][ld_x]
+    long long ld_x;
+    const float *s;          // [g][ld_s]
+    long long ld_s;
+    int n;                   // tokens in this call
+    int d;                   // d_in
+    int g;
+    int group_pairs;         // ceil(g / 2)
+    Schedule sched;          // units = tiles * group_pairs, ksteps = ceil(n / 64)
+    uint32_t *status;
+    unsigned long long wait_budget_ns;
+};
+
+// Walks the k-steps of a pair's work items in order, across item boundaries.
+struct KstepCursor {
+    const Schedule &sched;
+    int pair;
+    int it;
+    int ks;
+    bool valid;
+    WorkItem w;
+    __device__ KstepCursor(const Schedule &sc, int pr) : sched(sc), pair(pr), it(0), ks(0), valid(false)
+    {
+        valid = work_item(sched, pair, 0, w);
+        ks = w.ks0;
+    }
+    __device__ void advance(int n)
+    {
+        while (n > 0 && valid) {
+            const int left = w.ks1 - ks;
+            if (n < left) {
+                ks += n;
+                n = 0;
+            } else {
+                n -= left;
+                ++it;
+                valid = work_item(sched, pair, it, w);
+                ks = w.ks0;
+            }
+        }
+    }
+};
+
+__device__ __forceinline__ uint4 ld_stream_16(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void st_shared_16(uint32_t addr, const uint4 &v)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+// A saliency value as two bf16 terms packed in one word: low half hi = bf16(a), high half lo = bf16(a - hi);
+// hi + lo carries a to 16 significant bits.
+__device__ __forceinline__ uint32_t split_scale(float a)
+{
+    const __nv_bfloat16 hi = __float2bfloat16_rn(a);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(a - __bfloat162float(hi));
+    return static_cast<uint32_t>(__bfloat16_as_ushort(hi)) | (static_cast<uint32_t>(__bfloat16_as_ushort(lo)) << 16);
+}
+
+// v (8 bf16) times the split scale `a2`: per element fma(x, hi, x * lo) with packed bf16 fused multiply-adds.
+// x * lo is rounded to bf16 (an error of 2^-18 of the product), then x * hi + that is formed exactly and
+// rounded to bf16 once; no conversion to fp32 and back is needed.
+__device__ __forceinline__ uint4 scale_bf16x8(const uint4 &v, uint32_t a2)
+{
+    const uint32_t hi_bits = __byte_perm(a2, a2, 0x1010);
+    const uint32_t lo_bits = __byte_perm(a2, a2, 0x3232);
+    const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162 *>(&hi_bits);
+    const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162 *>(&lo_bits);
+    const __nv_bfloat162 *x = reinterpret_cast<const __nv_bfloat162 *>(&v);
+    uint4 o;
+    __nv_bfloat162 *oh = reinterpret_cast<__nv_bfloat162 *>(&o);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) oh[e] = __hfma2(x[e], hi, __hmul2(x[e], lo));
+    return o;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(HS_THREADS, 1)
+hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapH, const HessianParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[HS_STAGES];    // first CTA: B bytes of both CTAs + all scaler warps
+    __shared__ __align__(8) uint64_t bar_empty[HS_STAGES];   // both CTAs: signalled by the MMA commits
+    __shared__ __align__(8) uint64_t bar_acc_full;           // both CTAs: signalled by the MMA commit
+    __shared__ __align__(8) uint64_t bar_acc_empty;          // first CTA: 16 epilogue warps arrive
+    __shared__ __align__(8) uint64_t bar_drain;
+    __shared__ uint32_t tmem_base_smem;
+    __shared__ volatile uint32_t abort_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int pair = static_cast<int>(blockIdx.x >> 1);
+    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t staging = ring + HS_STAGES * HS_STAGE_BYTES;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < HS_STAGES; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1 + 2 * HS_SET_WARPS);
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+        }
+        mbar_init(smem_u32(&bar_acc_full), 1);
+        mbar_init(smem_u32(&bar_acc_empty), 2 * HS_EPI_WARPS);
+        mbar_init(smem_u32(&bar_drain), 1);
+        abort_flag = 0u;
+        fence_mbar_init();
+        prefetch_tensormap(&mapX);
+        prefetch_tensormap(&mapH);
+    }
+    if (warp == 2) {
+        tmem_alloc(smem_u32(&tmem_base_smem), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    cluster_sync_all();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_base_smem;
+    const WaitCtx wc{&abort_flag, p.status, p.wait_budget_ns};
+
+    if (warp == 0 && lane == 0) {
+        // ------------------------------------------------------------------ TMA producer: raw B columns
+        int s = 0;
+        uint32_t ph = 0;
+        uint32_t issued = 0;
+        bool ok = true;
+        WorkItem w;
+        for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
+            int ti, tj;
+            tile_of_slot(w.unit / p.group_pairs, ti, tj);
+            const int b0 = tj * TILE_N + static_cast<int>(rank) * CTA_ROWS;
+            for (int ks = w.ks0; ks < w.ks1; ++ks) {
+                if (!bounded_wait(smem_u32(&bar_empty[s]), ph ^ 1u, wc, 1u, w.unit)) { ok = false; break; }
+                const uint32_t full_local = smem_u32(&bar_full[s]);
+                if (rank == 0) mbar_arrive_expect_tx(full_local, 2 * HS_B_BYTES);     // both CTAs' bytes
+                const uint32_t full = map_to_cta(full_local, 0);
+                const uint32_t sb = ring + s * HS_STAGE_BYTES;
+#pragma unroll
+                for (int q = 0; q < CTA_ROWS / BOX_FEATURES; ++q)
+                    tma_load_3d_pair(sb + q * BOX_BYTES, &mapX, full, b0 + q * BOX_FEATURES, ks * TILE_K, 0);
+                ++issued;
+                if (++s == HS_STAGES) { s = 0; ph ^= 1u; }
+            }
+        }
+        // Stay until every stage has been released again (see gq_gram.cuh).
+        for (int q = 0; ok && issued != 0u && q < HS_STAGES; ++q) {
+            if (!bounded_wait(smem_u32(&bar_empty[s]), ph ^ 1u, wc, 5u, 0u)) ok = false;
+            if (++s == HS_STAGES) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) spin_ns(1000000ull);
+    } else if (warp == 1 && lane == 0 && rank == 0) {
+        // ------------------------------------------------------------------ MMA issuer (first CTA)
+        constexpr uint32_t idesc = umma_idesc_bf16_mn(TILE_M, TILE_N);
+        int s = 0;
+        uint32_t ph = 0;
+        uint32_t acc_ph = 0;
+        bool ok = true;
+        WorkItem w;
+        for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
+            const int k0 = (w.unit % p.group_pairs) * HS_GROUPS;
+            const int ng = (p.g - k0 < HS_GROUPS) ? (p.g - k0) : HS_GROUPS;
+            if (!bounded_wait_hot(smem_u32(&bar_acc_empty), acc_ph ^ 1u, wc, 2u, w.unit)) { ok = false; break; }
+            tc_fence_after_sync();
+            for (int ks = w.ks0; ks < w.ks1; ++ks) {
+                if (!bounded_wait_hot(smem_u32(&bar_full[s]), ph, wc, 3u, w.unit)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t sb = ring + s * HS_STAGE_BYTES;
+                for (int kk = 0; kk < ng; ++kk) {
+                    const uint32_t sa = sb + HS_B_BYTES + kk * HS_A_BYTES;
+                    const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(kk * TILE_N);
+#pragma unroll
+                    for (int k16 = 0; k16 < TILE_K / 16; ++k16) {
+                        const uint64_t adesc = umma_smem_desc_mn_sw128(sa + k16 * 16 * 128, BOX_BYTES, 1024);
+                        const uint64_t bdesc = umma_smem_desc_mn_sw128(sb + k16 * 16 * 128, BOX_BYTES, 1024);
+                        umma_bf16(d_tmem, adesc, bdesc, idesc, (ks != w.ks0 || k16 != 0) ? 1u : 0u);
+                    }
+                }
+                umma_commit_pair(smem_u32(&bar_empty[s]));
+                if (++s == HS_STAGES) { s = 0; ph ^= 1u; }
+            }
+            if (!ok) break;
+            umma_commit_pair(smem_u32(&bar_acc_full));
+            acc_ph ^= 1u;
+        }
+        if (!ok) {
+            umma_commit_local(smem_u32(&bar_drain));
+            const uint64_t t0 = global_timer_ns();
+            while (!mbar_try_wait(smem_u32(&bar_drain), 0u) && global_timer_ns() - t0 < 5000000ull) {}
+        }
+    } else if (warp >= 4 && warp < 4 + HS_SCALER_WARPS) {
+        // ------------------------------------------------------------------ scalers: A_k = s_k (.) X rows
+        // The scaler warps form HS_SETS independent sets of four warps; set j produces the k-steps whose
+        // running number is j modulo HS_SETS, from the loads to the arrival on the "full" barrier.  A set
+        // issues the loads of its next k-step as soon as it has finished the previous one, i.e. HS_SETS - 1
+        // k-steps of the other sets' work lie between a load and its use: global-memory latency is hidden by
+        // the other sets rather than by a register rotation inside one warp.
+        // Inside a set, sixteen threads share a token row (16 x 16 bytes = the 128 features, so a warp reads
+        // two whole 256-byte row segments per load) and eight passes cover the 64 tokens of the k-step.  Every
+        // thread fetches the saliency values of its eight tokens itself (a broadcast load per pass and group);
+        // shuffles are avoided: like every shared-memory-pipe instruction they compete with the tensor core's
+        // operand reads.
+        constexpr int TOK_PER_PASS = HS_SET_WARPS * 2;         // tokens a set covers per instruction
+        constexpr int PASSES = TILE_K / TOK_PER_PASS;          // 16-byte loads per thread and k-step
+        const int set = (warp - 4) / HS_SET_WARPS;
+        const int st = static_cast<int>(threadIdx.x) - 128 - set * (HS_SET_WARPS * 32);    // 0..127
+        const int c = st & 15;                                 // 16-byte chunk of the 128-feature row
+        const int trow = st >> 4;                              // token within a pass
+        const uint32_t col_off = static_cast<uint32_t>((c >> 3) * BOX_BYTES);
+        const int cb = c & 7;
+
+        KstepCursor cur(p.sched, pair);
+        cur.advance(set);
+        int cached_it = -1;
+        int ng = 0;
+        const __nv_bfloat16 *xcol = nullptr;
+        const float *s0 = nullptr;
+        bool f_ok = false;
+        for (int cnt = set; cur.valid; cnt += HS_SETS, cur.advance(HS_SETS)) {
+            if (cur.it != cached_it) {
+                cached_it = cur.it;
+                int ti, tj;
+                tile_of_slot(cur.w.unit / p.group_pairs, ti, tj);
+                const int k0 = (cur.w.unit % p.group_pairs) * HS_GROUPS;
+                ng = (p.g - k0 < HS_GROUPS) ? (p.g - k0) : HS_GROUPS;
+                const int f = ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + c * 8;
+                f_ok = f < p.d;
+                xcol = p.X + f;
+                s0 = p.s + static_cast<long long>(k0) * p.ld_s;
+            }
+            const int tok0 = cur.ks * TILE_K + trow;
+            const float *s1 = s0 + (ng > 1 ? p.ld_s : 0);
+            uint4 buf[PASSES];
+            float sa0[PASSES], sa1[PASSES];
+#pragma unroll
+            for (int j = 0; j < PASSES; ++j) {
+                const int tok = tok0 + j * TOK_PER_PASS;
+                const bool t_ok = tok < p.n;
+                buf[j] = (f_ok && t_ok) ? ld_stream_16(xcol + static_cast<long long>(tok) * p.ld_x)
+                                        : make_uint4(0u, 0u, 0u, 0u);
+                sa0[j] = t_ok ? __ldg(s0 + tok) : 0.0f;
+                sa1[j] = t_ok ? __ldg(s1 + tok) : 0.0f;
+            }
+
+            const int s = cnt % HS_STAGES;
+            const uint32_t ph = static_cast<uint32_t>(cnt / HS_STAGES) & 1u;
+            bool got = true;
+            if (lane == 0) got = bounded_wait(smem_u32(&bar_empty[s]), ph ^ 1u, wc, 6u, cur.w.unit);
+            got = __any_sync(0xffffffffu, got && lane == 0);
+            if (!got) break;
+            (void)mbar_try_wait(smem_u32(&bar_empty[s]), ph ^ 1u);   // every lane observes the completed phase
+            const uint32_t sa = ring + s * HS_STAGE_BYTES + HS_B_BYTES + col_off;
+#pragma unroll
+            for (int j = 0; j < PASSES; ++j) {
+                const int tl = j * TOK_PER_PASS + trow;
+                const uint32_t dst = sa + static_cast<uint32_t>(tl * 128 + ((cb ^ (tl & 7)) << 4));
+                st_shared_16(dst, scale_bf16x8(buf[j], split_scale(sa0[j])));
+                if (ng > 1) st_shared_16(dst + HS_A_BYTES, scale_bf16x8(buf[j], split_scale(sa1[j])));
+            }
+            fence_proxy_async_smem();        // make the stores visible to the tensor core's reads
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_full[s]), 0));
+        }
+    } else if (warp >= 4 + HS_SCALER_WARPS) {
+        // ------------------------------------------------------------------ epilogue: H += accumulators
+        const int ew = warp - (4 + HS_SCALER_WARPS);    // 0..7
+        const int q = warp & 3;                         // TMEM lane quarter this warp may access
+        const int half = ew >> 2;                       // which 128 of the 256 accumulator columns
+        const uint32_t stg = staging + static_cast<uint32_t>(ew) * 4096u;
+        uint32_t acc_ph = 0;
+        bool ok = true;
+        WorkItem w;
+        for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
+            int ti, tj;
+            tile_of_slot(w.unit / p.group_pairs, ti, tj);
+            const int k0 = (w.unit % p.group_pairs) * HS_GROUPS;
+            const int ng = (p.g - k0 < HS_GROUPS) ? (p.g - k0) : HS_GROUPS;
+            if (lane == 0) ok = bounded_wait(smem_u32(&bar_acc_full), acc_ph, wc, 4u, w.unit);
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            (void)mbar_try_wait(smem_u32(&bar_acc_full), acc_ph);     // every lane observes the completed phase
+            tc_fence_after_sync();
+            const int row0 = ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + q * 32;
+            for (int kk = 0; kk < ng; ++kk) {
+#pragma unroll 1
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    const int cc = half * 4 + c4;
+                    const int col0 = tj * TILE_N + cc * 32;
+                    if (col0 >= p.d || row0 >= p.d) break;      // outside the matrix
+                    if (col0 + 32 <= row0) continue;            // 32 x 32 block strictly below the diagonal
+                    uint32_t r[32];
+                    tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
+                                      static_cast<uint32_t>(kk * TILE_N + cc * 32), r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int v = 0; v < 8; ++v)
+                        st_shared_16(stg + static_cast<uint32_t>(lane * 128 + ((v ^ (lane & 7)) << 4)),
+                                     make_uint4(r[v * 4 + 0], r[v * 4 + 1], r[v * 4 + 2], r[v * 4 + 3]));
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_reduce_add_3d(&mapH, stg, col0, row0, k0 + kk);
+                        bulk_commit_group();
+                        bulk_wait_group_read0();      // staging block reusable once the copy engine has read it
+                    }
+                    __syncwarp();
+                }
+            }
+            // This warp has read all it needs from tensor memory: tell the MMA issuer (first CTA).
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_acc_empty), 0));
+            acc_ph ^= 1u;
+        }
+    }
+
+    __syncwarp();
+    tc_fence_before_sync();
+    cluster_sync_all();
+    if (warp == 2) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace gq

@@ -14,6 +14,7 @@
 
 #include "../../include/gq.h"
 #include "gq_gram.cuh"
+#include "gq_hessian.cuh"
 #include "gq_kernels.cuh"
 
 #define GQ_VERSION_NUMBER 100   /* 0.1.0 */
@@ -97,6 +98,8 @@ int32_t device_info(DeviceInfo **out)
                                      gq::GRAM_SMEM_BYTES));
         GQ_CUDA(cudaFuncSetAttribute(gq::gram_kernel<gq::EPI_DOT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      gq::GRAM_SMEM_BYTES));
+        GQ_CUDA(cudaFuncSetAttribute(gq::hessian_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     gq::HS_SMEM_BYTES));
         {
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3(static_cast<unsigned>(di.sm_count & ~1));
@@ -167,6 +170,23 @@ int32_t make_map(CUtensorMap *map, const void *base, int64_t features, int64_t r
     return GQ_OK;
 }
 
+// fp32 tensor [groups][d][d] as a TMA map with 32 x 32 boxes and the 128-byte swizzle (reduce-add target).
+int32_t make_map_h(CUtensorMap *map, float *H, int64_t d, int64_t groups)
+{
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(groups)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(d) * 4, static_cast<cuuint64_t>(d) * static_cast<cuuint64_t>(d) * 4};
+    cuuint32_t box[3] = {32, 32, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, H, dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        tl_last_cuda_error = static_cast<int32_t>(cudaErrorInvalidValue);
+        return GQ_ERR_CUDA;
+    }
+    return GQ_OK;
+}
+
 int grid_for(long long work_items, int threads, int sm_count, int blocks_per_sm)
 {
     long long blocks = (work_items + threads - 1) / threads;
@@ -194,10 +214,8 @@ int32_t check_layer_shape(int64_t d_in, int64_t d_out, int32_t g, bool need_out)
     return GQ_OK;
 }
 
-size_t hessian_ws_bytes(int64_t n_max, int64_t d_in, int32_t g)
-{
-    return round_up(static_cast<size_t>(g) * static_cast<size_t>(n_max) * static_cast<size_t>(d_in) * 2, 1024);
-}
+// The guided-Hessian kernel scales its operand on the fly: no scratch is needed.
+size_t hessian_ws_bytes(int64_t, int64_t, int32_t) { return 0; }
 
 struct ObjectiveLayout {
     size_t hi_off, lo_off, partials_off, total;
@@ -283,49 +301,35 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
     if (n == 0) return GQ_OK;              // an empty chunk adds nothing: pointers are not looked at
     if (!X || !s || !H) return GQ_ERR_INVALID_ARG;
     if (!aligned(X, 16) || !aligned(H, 16) || !aligned(s, 4)) return GQ_ERR_ALIGNMENT;
-    if (!workspace || workspace_bytes < hessian_ws_bytes(n, d_in, g)) return GQ_ERR_WORKSPACE;
-    if (!aligned(workspace, 1024)) return GQ_ERR_ALIGNMENT;
+    (void)workspace;
+    (void)workspace_bytes;
     DeviceInfo *di;
     if (int32_t rc = device_info(&di)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    __nv_bfloat16 *Y = static_cast<__nv_bfloat16 *>(workspace);
-
-    // Y_k = Diag(s_k) X rounded to bf16, so that H_k += X^T Y_k.
-    {
-        const int grid = grid_for(n * (d_in / 8), 256, di->sm_count, 8);
-        {
-            LaunchScope scope(GQ_KERNEL_SCALE_ROWS, st);
-            gq::scale_rows_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(X), n, static_cast<int>(d_in),
-                                                        ld_x, s, ld_s, g, Y);
-        }
-        GQ_CUDA(cudaGetLastError());
-    }
-    CUtensorMap mapX, mapY;
+    CUtensorMap mapX, mapH;
     if (int32_t rc = make_map(&mapX, X, d_in, n, 1, ld_x, n * ld_x)) return rc;
-    if (int32_t rc = make_map(&mapY, Y, d_in, n, g, d_in, n * d_in)) return rc;
-    gq::GramParams p{};
+    if (int32_t rc = make_map_h(&mapH, H, d_in, g)) return rc;
+    gq::HessianParams p{};
+    p.X = static_cast<const __nv_bfloat16 *>(X);
+    p.ld_x = ld_x;
+    p.s = s;
+    p.ld_s = ld_s;
+    p.n = static_cast<int>(n);
     p.d = static_cast<int>(d_in);
-    p.rows = static_cast<int>(n);
     p.g = g;
-    p.n_terms = 1;
-    p.term_a[0] = 0;
-    p.term_b[0] = 1;
-    p.map_grouped[0] = 0;
-    p.map_grouped[1] = 1;
-    const int units = tiles_for(d_in) * g;
+    p.group_pairs = (g + gq::HS_GROUPS - 1) / gq::HS_GROUPS;
+    const int units = tiles_for(d_in) * p.group_pairs;
     const int ksteps = static_cast<int>((n + gq::TILE_K - 1) / gq::TILE_K);
     const bool balanced = (flags & GQ_HESSIAN_DETERMINISTIC) == 0;
     int pairs = di->max_pairs;
     if (!balanced && units < pairs) pairs = units;
-    gq::plan_schedule(p, units, ksteps, pairs, balanced);
-    p.H = H;
-    p.partials = nullptr;
+    p.sched = gq::plan_schedule(units, ksteps, pairs, balanced);
     p.status = di->status_ptr;
     p.wait_budget_ns = wait_budget_ns();
-    const int grid = 2 * ((p.full_waves == 0 && p.tail_pairs > 0) ? p.tail_pairs : pairs);
+    const int grid = 2 * ((p.sched.full_waves == 0 && p.sched.tail_pairs > 0) ? p.sched.tail_pairs : pairs);
     {
-        LaunchScope scope(GQ_KERNEL_GRAM_ACCUM, st);
-        gq::gram_kernel<gq::EPI_ACCUM><<<grid, gq::GRAM_THREADS, gq::GRAM_SMEM_BYTES, st>>>(mapX, mapY, p);
+        LaunchScope scope(GQ_KERNEL_HESSIAN, st);
+        gq::hessian_kernel<<<grid, gq::HS_THREADS, gq::HS_SMEM_BYTES, st>>>(mapX, mapH, p);
     }
     GQ_CUDA(cudaGetLastError());
     return GQ_OK;
@@ -394,12 +398,12 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     const int tiles = tiles_for(d_in);
     const int units = tiles * g;
     const int ksteps = 3 * static_cast<int>((m + gq::TILE_K - 1) / gq::TILE_K);
-    gq::plan_schedule(p, units, ksteps, units < di->max_pairs ? units : di->max_pairs, false);
+    p.sched = gq::plan_schedule(units, ksteps, units < di->max_pairs ? units : di->max_pairs, false);
     p.H = const_cast<float *>(H);
     p.partials = partials;
     p.status = di->status_ptr;
     p.wait_budget_ns = wait_budget_ns();
-    const int grid = 2 * p.pairs;
+    const int grid = 2 * p.sched.pairs;
     {
         LaunchScope scope(GQ_KERNEL_GRAM_DOT, st);
         gq::gram_kernel<gq::EPI_DOT><<<grid, gq::GRAM_THREADS, gq::GRAM_SMEM_BYTES, st>>>(mapHi, mapLo, p);
@@ -495,12 +499,12 @@ int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, i
     p.map_grouped[1] = 1;
     const int units = tiles * g;
     const int ksteps = 3 * static_cast<int>((m + gq::TILE_K - 1) / gq::TILE_K);
-    gq::plan_schedule(p, units, ksteps, units < di->max_pairs ? units : di->max_pairs, false);
+    p.sched = gq::plan_schedule(units, ksteps, units < di->max_pairs ? units : di->max_pairs, false);
     p.H = const_cast<float *>(H);
     p.partials = partials;
     p.status = di->status_ptr;
     p.wait_budget_ns = wait_budget_ns();
-    const int grid = 2 * p.pairs;
+    const int grid = 2 * p.sched.pairs;
     gq::gram_kernel<gq::EPI_DOT><<<grid, gq::GRAM_THREADS, gq::GRAM_SMEM_BYTES, st>>>(mapHi, mapLo, p);
     g_launches.fetch_add(1);
     GQ_CUDA(cudaGetLastError());

@@ -81,20 +81,26 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 // Arrive on a barrier that lives in another (or this) CTA of the cluster; `cluster_addr` from map_to_cta.
+// Default semantics (release at CTA scope): what the arrival publishes is shared-memory or tensor-memory
+// state that the async proxy / tensor core of the arriving thread's own CTA consumes, made visible
+// beforehand by fence.proxy.async or tcgen05.fence.  (A cluster-scope release would also wait for the
+// thread's outstanding global loads, which the callers keep in flight on purpose.)
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-// Wait variant that pairs with mbar_arrive_cluster (acquire at cluster scope).
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
+// Like mbar_try_wait, but the thread may stay suspended inside the instruction for up to `hint_ns`
+// nanoseconds while the phase is incomplete (it is woken when the phase completes), instead of returning
+// at once: a waiting warp then leaves the issue slots to the warps that have work.
+__device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t parity, uint32_t hint_ns)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
         : "memory");
     return ok != 0;
 }
@@ -127,6 +133,27 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t smem_dst, const void *
         "[%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
+}
+
+// 3-D tiled reduce-add shared memory -> global: every element of the box is added to the tensor in
+// global memory by the memory system.  Part of the calling thread's current bulk async-group.
+// c0 times the element size must be a multiple of 16 bytes and no coordinate may be negative.
+__device__ __forceinline__ void tma_reduce_add_3d(const void *map, uint32_t smem_src, int32_t c0, int32_t c1,
+                                                  int32_t c2)
+{
+    asm volatile(
+        "cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+        ::"l"(reinterpret_cast<uint64_t>(map)), "r"(smem_src), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group()
+{
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// Returns once the shared-memory sources of all bulk groups committed by this thread have been read.
+__device__ __forceinline__ void bulk_wait_group_read0()
+{
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 
 // ---------------------------------------------------------------- tcgen05 / TMEM (CTA pair)
