@@ -74,8 +74,7 @@ int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad,
  * for every group k and every a <= b (the upper triangle including the diagonal).  No 1/n factor.
  *
  *   X          bf16 [n, ld_x], 16-byte aligned, ld_x >= d_in, ld_x % 8 == 0
- *   n          tokens in this chunk, 0 <= n <= the n_max the workspace was sized for (0 is a no-op:
- *              sizes are still validated, pointers are not)
+ *   n          tokens in this chunk, >= 0 (0 is a no-op: sizes are still validated, pointers are not)
  *   d_in       d_in % 8 == 0, 8 <= d_in <= 65536
  *   s          fp32 [g, ld_s], s >= 0 (as produced by gq_saliency), ld_s >= n
  *   H          fp32 [g, d_in, d_in] row-major, 16-byte aligned.  The caller zeroes it before the
@@ -83,22 +82,25 @@ int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad,
  *              entries with a <= b are defined; entries below the diagonal hold unspecified finite
  *              values until gq_hessian_finalize() is called.
  *   flags      0, or GQ_HESSIAN_DETERMINISTIC (see below)
- *   workspace  device scratch of at least gq_hessian_workspace_bytes(n_max, d_in, g, flags)
- *              bytes, 1024-byte aligned; contents need not be preserved between calls.
- * Arithmetic: rows of X are multiplied by s_k in fp32 and rounded to bf16 once; products are
- * accumulated in fp32 on the tensor cores; each call adds its fp32 tile sums to H.
- * Work is dealt to the SM pairs in whole 256 x 256 tiles; with flags == 0 the last, incomplete round
- * of tiles is cut along the token axis so that every SM pair gets the same amount of work, and the
- * pieces of such a tile are added to H with floating-point atomics: those entries can differ in the
- * last bit from run to run.  With GQ_HESSIAN_DETERMINISTIC every element of H has a single writer
- * and results are bit-reproducible run to run, at the price of an idle tail in the last round.
+ *   workspace  not used by the current kernels (gq_hessian_workspace_bytes() returns 0); may be NULL.
+ *              The parameters stay in the signature so that callers written against it keep working.
+ * Arithmetic: the kernel never writes a scaled copy of X to global memory.  While X is staged for the
+ * tensor cores every element is multiplied by s_k[i], with s_k[i] carried as the sum of two bf16 terms
+ * (16 significant bits) and packed bf16 fused multiply-adds, and rounded to bf16 once; the products
+ * (s_k[i] X[i][a]) * X[i][b] are accumulated in fp32 in tensor memory (two groups per pass over X), and
+ * each call adds its fp32 tile sums to H with reduce-add transactions, so H is never read by the SMs.
+ * Work is dealt to the SM pairs in whole 256 x 256 tiles of two groups; with flags == 0 the last,
+ * incomplete round of tiles is cut along the token axis so that every SM pair gets the same amount of
+ * work, and the pieces of such a tile reach H in no fixed order: those entries can differ in the last
+ * bit from run to run.  With GQ_HESSIAN_DETERMINISTIC every element of H receives exactly one add per
+ * call and results are bit-reproducible run to run, at the price of an idle tail in the last round.
  */
 #define GQ_HESSIAN_DETERMINISTIC 1u
 int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld_x, const float *s,
                               int64_t ld_s, int32_t g, float *H, uint32_t flags, void *workspace,
                               size_t workspace_bytes, void *stream);
 
-/* Scratch bytes gq_hessian_accumulate needs for chunks of up to n_max tokens (0 on bad arguments). */
+/* Scratch bytes gq_hessian_accumulate needs for chunks of up to n_max tokens: currently always 0. */
 size_t gq_hessian_workspace_bytes(int64_t n_max, int64_t d_in, int32_t g, uint32_t flags);
 
 /*

@@ -25,7 +25,7 @@
 //
 // Warps: 0 TMA producer (one lane) | 1 MMA issuer (one lane, first CTA) | 2 TMEM allocation | 3 idle |
 //        4..15 scalers | 16..23 epilogue.
-// Work units are (tile, pair of groups); they are dealt to the CTA pairs as described in gq_gram.cuh
+// Work units are (tile, pair of groups); they are dealt to the CTA pairs as described in gq_pipeline.cuh
 // (round-robin rounds, then the incomplete last round cut along the token axis).  Because H is updated
 // by reduce-adds only, pieces of a cut unit need no special treatment.
 //
@@ -33,14 +33,14 @@
 // epilogue warps have read them out of tensor memory (not until H is updated).  Producer and scalers run
 // ahead into the next unit meanwhile, so the pipeline is full again when the MMAs resume.
 //
-// Every mbarrier wait is bounded (see gq_gram.cuh).
+// Every mbarrier wait is bounded (see gq_pipeline.cuh).
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#include "gq_gram.cuh"
+#include "gq_pipeline.cuh"
 
 namespace gq {
 
@@ -69,36 +69,6 @@ struct HessianParams {
     Schedule sched;          // units = tiles * group_pairs, ksteps = ceil(n / 64)
     uint32_t *status;
     unsigned long long wait_budget_ns;
-};
-
-// Walks the k-steps of a pair's work items in order, across item boundaries.
-struct KstepCursor {
-    const Schedule &sched;
-    int pair;
-    int it;
-    int ks;
-    bool valid;
-    WorkItem w;
-    __device__ KstepCursor(const Schedule &sc, int pr) : sched(sc), pair(pr), it(0), ks(0), valid(false)
-    {
-        valid = work_item(sched, pair, 0, w);
-        ks = w.ks0;
-    }
-    __device__ void advance(int n)
-    {
-        while (n > 0 && valid) {
-            const int left = w.ks1 - ks;
-            if (n < left) {
-                ks += n;
-                n = 0;
-            } else {
-                n -= left;
-                ++it;
-                valid = work_item(sched, pair, it, w);
-                ks = w.ks0;
-            }
-        }
-    }
 };
 
 __device__ __forceinline__ uint4 ld_stream_16(const void *p)
@@ -208,7 +178,8 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                 if (++s == HS_STAGES) { s = 0; ph ^= 1u; }
             }
         }
-        // Stay until every stage has been released again (see gq_gram.cuh).
+        // Stay until every stage has been released again: the release is an arrival on this CTA's barriers,
+        // which must not come after the CTA has gone.
         for (int q = 0; ok && issued != 0u && q < HS_STAGES; ++q) {
             if (!bounded_wait(smem_u32(&bar_empty[s]), ph ^ 1u, wc, 5u, 0u)) ok = false;
             if (++s == HS_STAGES) { s = 0; ph ^= 1u; }

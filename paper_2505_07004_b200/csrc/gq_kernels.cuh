@@ -1,4 +1,4 @@
-// Bandwidth-bound kernels of libgq: saliency reduction, row scaling, mirror, weight-error split,
+// Bandwidth-bound kernels of libgq: saliency reduction, mirror, weight-error split,
 // final fp64 reduction.  All use 128-bit accesses and grid-stride loops over a grid sized from the
 // SM count.
 #pragma once
@@ -70,32 +70,6 @@ saliency_kernel(const __nv_bfloat16 *__restrict__ grad, long long n, int m, long
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
         if (lane == 0) s[static_cast<long long>(k) * ld_s + i] = sum * coef;
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
-// Row scaling for Algorithm 1 line 4:  Y[k][i][a] = bf16( s[k][i] * X[i][a] ), so that
-// H_k = X^T Diag(s_k) X = X^T Y_k.  One thread handles 8 features of one token for all groups.
-__global__ void __launch_bounds__(256)
-scale_rows_kernel(const __nv_bfloat16 *__restrict__ X, long long n, int d, long long ld_x, const float *__restrict__ s,
-                  long long ld_s, int g, __nv_bfloat16 *__restrict__ Y)
-{
-    const int vec_per_row = d >> 3;
-    const long long total = n * vec_per_row;
-    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
-    const long long group_stride = n * static_cast<long long>(d);
-    for (long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total; idx += stride) {
-        const long long i = idx / vec_per_row;
-        const int a = static_cast<int>(idx - i * vec_per_row) << 3;
-        float x[8];
-        bf16x8_to_float(__ldg(reinterpret_cast<const uint4 *>(X + i * ld_x + a)), x);
-        for (int k = 0; k < g; ++k) {
-            const float sk = __ldg(s + static_cast<long long>(k) * ld_s + i);
-            float y[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) y[e] = sk * x[e];
-            *reinterpret_cast<uint4 *>(Y + k * group_stride + i * d + a) = float_to_bf16x8(y);
-        }
     }
 }
 

@@ -13,8 +13,8 @@
 #include <vector>
 
 #include "../../include/gq.h"
-#include "gq_gram.cuh"
 #include "gq_hessian.cuh"
+#include "gq_objective.cuh"
 #include "gq_kernels.cuh"
 
 #define GQ_VERSION_NUMBER 100   /* 0.1.0 */
@@ -63,7 +63,7 @@ __device__ uint32_t g_status_word[4];
 struct DeviceInfo {
     bool ready = false;
     int sm_count = 0;
-    int max_pairs = 0;          // CTA pairs (clusters of two) of the Gram kernel that can be resident at once
+    int max_pairs = 0;          // CTA pairs (clusters of two) of a tensor-core kernel that can be resident at once
     uint32_t *status_ptr = nullptr;
 };
 DeviceInfo g_dev[kMaxDevices];
@@ -94,17 +94,15 @@ int32_t device_info(DeviceInfo **out)
         void *sym = nullptr;
         GQ_CUDA(cudaGetSymbolAddress(&sym, g_status_word));
         di.status_ptr = static_cast<uint32_t *>(sym);
-        GQ_CUDA(cudaFuncSetAttribute(gq::gram_kernel<gq::EPI_ACCUM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     gq::GRAM_SMEM_BYTES));
-        GQ_CUDA(cudaFuncSetAttribute(gq::gram_kernel<gq::EPI_DOT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     gq::GRAM_SMEM_BYTES));
+        GQ_CUDA(cudaFuncSetAttribute(gq::objective_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     gq::OBJ_SMEM_BYTES));
         GQ_CUDA(cudaFuncSetAttribute(gq::hessian_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      gq::HS_SMEM_BYTES));
         {
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3(static_cast<unsigned>(di.sm_count & ~1));
-            cfg.blockDim = dim3(gq::GRAM_THREADS);
-            cfg.dynamicSmemBytes = gq::GRAM_SMEM_BYTES;
+            cfg.blockDim = dim3(gq::HS_THREADS);
+            cfg.dynamicSmemBytes = gq::HS_SMEM_BYTES;
             cudaLaunchAttribute attr;
             attr.id = cudaLaunchAttributeClusterDimension;
             attr.val.clusterDim.x = 2;
@@ -113,7 +111,7 @@ int32_t device_info(DeviceInfo **out)
             cfg.attrs = &attr;
             cfg.numAttrs = 1;
             int clusters = 0;
-            if (cudaOccupancyMaxActiveClusters(&clusters, gq::gram_kernel<gq::EPI_ACCUM>, &cfg) != cudaSuccess ||
+            if (cudaOccupancyMaxActiveClusters(&clusters, gq::hessian_kernel, &cfg) != cudaSuccess ||
                 clusters < 1) {
                 (void)cudaGetLastError();
                 clusters = di.sm_count / 2;
@@ -385,7 +383,7 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     CUtensorMap mapHi, mapLo;
     if (int32_t rc = make_map(&mapHi, hi, d_in, m, g, d_in, m * d_in)) return rc;
     if (int32_t rc = make_map(&mapLo, lo, d_in, m, g, d_in, m * d_in)) return rc;
-    gq::GramParams p{};
+    gq::ObjectiveParams p{};
     p.d = static_cast<int>(d_in);
     p.rows = static_cast<int>(m);
     p.g = g;
@@ -399,14 +397,14 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     const int units = tiles * g;
     const int ksteps = 3 * static_cast<int>((m + gq::TILE_K - 1) / gq::TILE_K);
     p.sched = gq::plan_schedule(units, ksteps, units < di->max_pairs ? units : di->max_pairs, false);
-    p.H = const_cast<float *>(H);
+    p.H = H;
     p.partials = partials;
     p.status = di->status_ptr;
     p.wait_budget_ns = wait_budget_ns();
     const int grid = 2 * p.sched.pairs;
     {
         LaunchScope scope(GQ_KERNEL_GRAM_DOT, st);
-        gq::gram_kernel<gq::EPI_DOT><<<grid, gq::GRAM_THREADS, gq::GRAM_SMEM_BYTES, st>>>(mapHi, mapLo, p);
+        gq::objective_kernel<<<grid, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(mapHi, mapLo, p);
     }
     GQ_CUDA(cudaGetLastError());
     {
@@ -475,7 +473,7 @@ int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, i
     double *partials = reinterpret_cast<double *>(scratch + 2 * GQ_NOALLOC_MATRIX_BYTES);
     const int64_t m = d_out / g;
     // Every scratch byte that is read below is written first by this same call (hi/lo by the split
-    // kernel, one partial per (unit, warp) by the Gram kernel), so what an earlier call left behind
+    // kernel, one partial per (unit, CTA, warp) by the objective kernel), so what an earlier call left behind
     // is never observed and nothing has to be cleared.
     {
         const long long count8 = d_in * d_out / 8;
@@ -487,7 +485,7 @@ int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, i
     CUtensorMap mapHi, mapLo;
     if (int32_t rc = make_map(&mapHi, hi, d_in, m, g, d_in, m * d_in)) return rc;
     if (int32_t rc = make_map(&mapLo, lo, d_in, m, g, d_in, m * d_in)) return rc;
-    gq::GramParams p{};
+    gq::ObjectiveParams p{};
     p.d = static_cast<int>(d_in);
     p.rows = static_cast<int>(m);
     p.g = g;
@@ -500,12 +498,12 @@ int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, i
     const int units = tiles * g;
     const int ksteps = 3 * static_cast<int>((m + gq::TILE_K - 1) / gq::TILE_K);
     p.sched = gq::plan_schedule(units, ksteps, units < di->max_pairs ? units : di->max_pairs, false);
-    p.H = const_cast<float *>(H);
+    p.H = H;
     p.partials = partials;
     p.status = di->status_ptr;
     p.wait_budget_ns = wait_budget_ns();
     const int grid = 2 * p.sched.pairs;
-    gq::gram_kernel<gq::EPI_DOT><<<grid, gq::GRAM_THREADS, gq::GRAM_SMEM_BYTES, st>>>(mapHi, mapLo, p);
+    gq::objective_kernel<<<grid, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(mapHi, mapLo, p);
     g_launches.fetch_add(1);
     GQ_CUDA(cudaGetLastError());
     gq::reduce_partials_kernel<<<1, 1024, 0, st>>>(partials, tiles, g, gq::PARTIALS_PER_UNIT, loss_out);
