@@ -31,8 +31,10 @@ __device__ __forceinline__ uint4 float_to_bf16x8(const float (&f)[8])
 // ------------------------------------------------------------------------------------------------
 // Algorithm 1 line 2.  One warp per (token, group) segment of m = d_out / g gradients:
 //   s[k][i] = (grad_scale^2 / m) * sum_j grad[i][m k + j]^2.
-// A lane reads 16 bytes (8 bf16) per step, four steps are kept in flight; the lane-to-element
-// assignment and the butterfly reduction are fixed, so the result does not depend on the grid.
+// A lane reads 16 bytes (8 bf16) per load and issues eight (long segments) or four loads (the last ones
+// predicated off at the end of the segment) before it touches the first result.
+// The lane-to-element assignment and the butterfly reduction are fixed, so the result does not depend on
+// the grid.
 __global__ void __launch_bounds__(256)
 saliency_kernel(const __nv_bfloat16 *__restrict__ grad, long long n, int m, long long ld_grad, int g, float coef,
                 float *__restrict__ s, long long ld_s)
@@ -48,10 +50,23 @@ saliency_kernel(const __nv_bfloat16 *__restrict__ grad, long long n, int m, long
         const uint4 *src = reinterpret_cast<const uint4 *>(grad + i * ld_grad + static_cast<long long>(k) * m);
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         int v = lane;
-        for (; v + 96 < vecs; v += 128) {
+        for (; v + 224 < vecs; v += 256) {               // eight full loads in flight
+            uint4 x[8];
+#pragma unroll
+            for (int t = 0; t < 8; ++t) x[t] = __ldcs(src + v + 32 * t);
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                float f[8];
+                bf16x8_to_float(x[t], f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[t & 3] = fmaf(f[e], f[e], acc[t & 3]);
+            }
+        }
+        for (; v < vecs; v += 128) {                     // rest: four loads, predicated off past the end
             uint4 x[4];
 #pragma unroll
-            for (int t = 0; t < 4; ++t) x[t] = __ldcs(src + v + 32 * t);
+            for (int t = 0; t < 4; ++t)
+                x[t] = (v + 32 * t < vecs) ? __ldcs(src + v + 32 * t) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
                 float f[8];
@@ -59,12 +74,6 @@ saliency_kernel(const __nv_bfloat16 *__restrict__ grad, long long n, int m, long
 #pragma unroll
                 for (int e = 0; e < 8; ++e) acc[t] = fmaf(f[e], f[e], acc[t]);
             }
-        }
-        for (int t = 0; v < vecs; v += 32, ++t) {
-            float f[8];
-            bf16x8_to_float(__ldcs(src + v), f);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[t & 3] = fmaf(f[e], f[e], acc[t & 3]);
         }
         float sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
 #pragma unroll
