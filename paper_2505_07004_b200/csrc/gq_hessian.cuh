@@ -5,7 +5,8 @@
 // Tokens i are the contraction index, features are contiguous in memory, so both MMA operands are
 // MN-major bf16.  The kernel runs as CTA pairs (clusters of two); a pair owns one 256 x 256 tile of H for
 // TWO groups at a time (2 x 256 fp32 accumulator columns = all of tensor memory), so that one pass over
-// the tile's rows of X serves two groups and no scaled copy of X ever exists in global memory:
+// the tile's rows of X serves two groups and no scaled copy of X ever exists in global memory.  (When g is
+// odd the last group is processed two neighbouring column tiles at a time instead: see UnitDesc.)
 //
 //   B operand  raw X[tokens, tile columns]: TMA boxes (64 tokens x 64 features, 128-byte swizzle),
 //              16 KB per CTA and k-step, shared by both groups
@@ -25,7 +26,7 @@
 //
 // Warps: 0 TMA producer (one lane) | 1 MMA issuer (one lane, first CTA) | 2 TMEM allocation | 3 idle |
 //        4..15 scalers | 16..23 epilogue.
-// Work units are (tile, pair of groups); they are dealt to the CTA pairs as described in gq_pipeline.cuh
+// Work units are (tile, pair of groups), plus (row block, pair of column tiles) for an odd last group; they are dealt to the CTA pairs as described in gq_pipeline.cuh
 // (round-robin rounds, then the incomplete last round cut along the token axis).  Because H is updated
 // by reduce-adds only, pieces of a cut unit need no special treatment.
 //
@@ -45,10 +46,9 @@
 namespace gq {
 
 constexpr int HS_STAGES = 4;
-constexpr int HS_GROUPS = 2;                                   // groups resident in tensor memory at once
-constexpr int HS_B_BYTES = (CTA_ROWS / BOX_FEATURES) * BOX_BYTES;            // 16 KB
-constexpr int HS_A_BYTES = (CTA_ROWS / BOX_FEATURES) * BOX_BYTES;            // 16 KB per group
-constexpr int HS_STAGE_BYTES = HS_B_BYTES + HS_GROUPS * HS_A_BYTES;          // 48 KB
+constexpr int HS_GROUPS = 2;                                   // accumulators resident in tensor memory at once
+constexpr int HS_SLOT_BYTES = (CTA_ROWS / BOX_FEATURES) * BOX_BYTES;         // one operand block: 16 KB
+constexpr int HS_STAGE_BYTES = 3 * HS_SLOT_BYTES;                            // 48 KB
 constexpr int HS_SETS = 3;                                     // independent scaler sets (k-steps in flight)
 constexpr int HS_SET_WARPS = 4;                                // warps per set: 128 threads cover 8 tokens x 128 features
 constexpr int HS_SCALER_WARPS = HS_SETS * HS_SET_WARPS;
@@ -65,11 +65,46 @@ struct HessianParams {
     int n;                   // tokens in this call
     int d;                   // d_in
     int g;
-    int group_pairs;         // ceil(g / 2)
-    Schedule sched;          // units = tiles * group_pairs, ksteps = ceil(n / 64)
+    int nj;                  // ceil(d / 256): tile blocks per side
+    int full_pairs;          // g / 2: pairs of groups that share a pass over X
+    int narrow_units;        // tiles * full_pairs: units (tile, pair of groups)
+    Schedule sched;          // units = narrow_units + (g odd ? column-pair slots : 0), ksteps = ceil(n / 64)
     uint32_t *status;
     unsigned long long wait_budget_ns;
 };
+
+// What a work unit computes.  A unit always fills (up to) two 256-column accumulators from one pass over
+// the tile rows of X:
+//   pair unit  one tile, two groups: accumulator kk holds group grp[kk]; B (raw columns) is shared, the
+//              scalers produce one A block per group;
+//   wide unit  (the last group when g is odd) one group, two neighbouring column tiles: accumulator kk
+//              holds column tile tj[kk]; the scaled A block is shared, there is one B block per tile.
+//              An accumulator whose tile lies below the diagonal or outside the matrix is not used.
+// Shared-memory stage = three 16 KB slots: [B | A(g0) | A(g1)] for a pair unit, [B(tj0) | A | B(tj1)] for a
+// wide unit.
+struct UnitDesc {
+    int ti;          // row block of the tile(s)
+    int tj[2];       // column block of accumulator 0 / 1
+    int grp[2];      // group of accumulator 0 / 1
+    bool use[2];
+    bool wide;
+    __device__ int a_slot(int kk) const { return wide ? 1 : 1 + kk; }
+    __device__ int b_slot(int kk) const { return (wide && kk) ? 2 : 0; }
+    __device__ int scaled_groups() const { return wide ? 1 : 2; }
+};
+
+// Slot t of the enumeration of (row block i, column-block pair q) with i <= 2q + 1, pairs outermost.
+__device__ __forceinline__ void colpair_of_slot(int t, int &i, int &q)
+{
+    int qq = static_cast<int>((sqrtf(4.0f * static_cast<float>(t) + 1.0f) - 1.0f) * 0.5f);
+    while (qq * qq + qq > t) --qq;
+    while ((qq + 1) * (qq + 1) + (qq + 1) <= t) ++qq;
+    q = qq;
+    i = t - qq * qq - qq;
+}
+
+struct HessianParams;
+__device__ __forceinline__ UnitDesc decode_unit(const HessianParams &p, int unit);
 
 __device__ __forceinline__ uint4 ld_stream_16(const void *p)
 {
@@ -110,6 +145,33 @@ __device__ __forceinline__ uint4 scale_bf16x8(const uint4 &v, uint32_t a2)
 #pragma unroll
     for (int e = 0; e < 4; ++e) oh[e] = __hfma2(x[e], hi, __hmul2(x[e], lo));
     return o;
+}
+
+__device__ __forceinline__ UnitDesc decode_unit(const HessianParams &p, int unit)
+{
+    UnitDesc u;
+    if (unit < p.narrow_units) {
+        int ti, tj;
+        tile_of_slot(unit / p.full_pairs, ti, tj);
+        const int k0 = (unit % p.full_pairs) * 2;
+        u.ti = ti;
+        u.tj[0] = u.tj[1] = tj;
+        u.grp[0] = k0;
+        u.grp[1] = k0 + 1;
+        u.use[0] = u.use[1] = true;
+        u.wide = false;
+    } else {
+        int i, q;
+        colpair_of_slot(unit - p.narrow_units, i, q);
+        u.ti = i;
+        u.tj[0] = 2 * q;
+        u.tj[1] = 2 * q + 1;
+        u.grp[0] = u.grp[1] = p.g - 1;
+        u.use[0] = 2 * q >= i;
+        u.use[1] = 2 * q + 1 < p.nj;
+        u.wide = true;
+    }
+    return u;
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(HS_THREADS, 1)
@@ -162,18 +224,21 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
         bool ok = true;
         WorkItem w;
         for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
-            int ti, tj;
-            tile_of_slot(w.unit / p.group_pairs, ti, tj);
-            const int b0 = tj * TILE_N + static_cast<int>(rank) * CTA_ROWS;
+            const UnitDesc u = decode_unit(p, w.unit);
+            const int n_b = u.wide ? (u.use[0] ? 1 : 0) + (u.use[1] ? 1 : 0) : 1;      // B blocks per stage
             for (int ks = w.ks0; ks < w.ks1; ++ks) {
                 if (!bounded_wait(smem_u32(&bar_empty[s]), ph ^ 1u, wc, 1u, w.unit)) { ok = false; break; }
                 const uint32_t full_local = smem_u32(&bar_full[s]);
-                if (rank == 0) mbar_arrive_expect_tx(full_local, 2 * HS_B_BYTES);     // both CTAs' bytes
+                if (rank == 0) mbar_arrive_expect_tx(full_local, 2 * n_b * HS_SLOT_BYTES);   // both CTAs' bytes
                 const uint32_t full = map_to_cta(full_local, 0);
-                const uint32_t sb = ring + s * HS_STAGE_BYTES;
+                for (int kk = 0; kk < (u.wide ? 2 : 1); ++kk) {
+                    if (!u.use[kk]) continue;
+                    const uint32_t sb = ring + s * HS_STAGE_BYTES + u.b_slot(kk) * HS_SLOT_BYTES;
+                    const int b0 = u.tj[kk] * TILE_N + static_cast<int>(rank) * CTA_ROWS;
 #pragma unroll
-                for (int q = 0; q < CTA_ROWS / BOX_FEATURES; ++q)
-                    tma_load_3d_pair(sb + q * BOX_BYTES, &mapX, full, b0 + q * BOX_FEATURES, ks * TILE_K, 0);
+                    for (int q = 0; q < CTA_ROWS / BOX_FEATURES; ++q)
+                        tma_load_3d_pair(sb + q * BOX_BYTES, &mapX, full, b0 + q * BOX_FEATURES, ks * TILE_K, 0);
+                }
                 ++issued;
                 if (++s == HS_STAGES) { s = 0; ph ^= 1u; }
             }
@@ -194,16 +259,17 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
         bool ok = true;
         WorkItem w;
         for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
-            const int k0 = (w.unit % p.group_pairs) * HS_GROUPS;
-            const int ng = (p.g - k0 < HS_GROUPS) ? (p.g - k0) : HS_GROUPS;
+            const UnitDesc u = decode_unit(p, w.unit);
             if (!bounded_wait_hot(smem_u32(&bar_acc_empty), acc_ph ^ 1u, wc, 2u, w.unit)) { ok = false; break; }
             tc_fence_after_sync();
             for (int ks = w.ks0; ks < w.ks1; ++ks) {
                 if (!bounded_wait_hot(smem_u32(&bar_full[s]), ph, wc, 3u, w.unit)) { ok = false; break; }
                 tc_fence_after_sync();
-                const uint32_t sb = ring + s * HS_STAGE_BYTES;
-                for (int kk = 0; kk < ng; ++kk) {
-                    const uint32_t sa = sb + HS_B_BYTES + kk * HS_A_BYTES;
+                const uint32_t stage = ring + s * HS_STAGE_BYTES;
+                for (int kk = 0; kk < HS_GROUPS; ++kk) {
+                    if (!u.use[kk]) continue;
+                    const uint32_t sa = stage + u.a_slot(kk) * HS_SLOT_BYTES;
+                    const uint32_t sb = stage + u.b_slot(kk) * HS_SLOT_BYTES;
                     const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(kk * TILE_N);
 #pragma unroll
                     for (int k16 = 0; k16 < TILE_K / 16; ++k16) {
@@ -255,14 +321,12 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
         for (int cnt = set; cur.valid; cnt += HS_SETS, cur.advance(HS_SETS)) {
             if (cur.it != cached_it) {
                 cached_it = cur.it;
-                int ti, tj;
-                tile_of_slot(cur.w.unit / p.group_pairs, ti, tj);
-                const int k0 = (cur.w.unit % p.group_pairs) * HS_GROUPS;
-                ng = (p.g - k0 < HS_GROUPS) ? (p.g - k0) : HS_GROUPS;
-                const int f = ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + c * 8;
+                const UnitDesc u = decode_unit(p, cur.w.unit);
+                ng = u.scaled_groups();
+                const int f = u.ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + c * 8;
                 f_ok = f < p.d;
                 xcol = p.X + f;
-                s0 = p.s + static_cast<long long>(k0) * p.ld_s;
+                s0 = p.s + static_cast<long long>(u.grp[0]) * p.ld_s;
             }
             const int tok0 = cur.ks * TILE_K + trow;
             const float *s1 = s0 + (ng > 1 ? p.ld_s : 0);
@@ -285,13 +349,13 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
             got = __any_sync(0xffffffffu, got && lane == 0);
             if (!got) break;
             (void)mbar_try_wait(smem_u32(&bar_empty[s]), ph ^ 1u);   // every lane observes the completed phase
-            const uint32_t sa = ring + s * HS_STAGE_BYTES + HS_B_BYTES + col_off;
+            const uint32_t sa = ring + s * HS_STAGE_BYTES + HS_SLOT_BYTES + col_off;     // slot 1 (and 2)
 #pragma unroll
             for (int j = 0; j < PASSES; ++j) {
                 const int tl = j * TOK_PER_PASS + trow;
                 const uint32_t dst = sa + static_cast<uint32_t>(tl * 128 + ((cb ^ (tl & 7)) << 4));
                 st_shared_16(dst, scale_bf16x8(buf[j], split_scale(sa0[j])));
-                if (ng > 1) st_shared_16(dst + HS_A_BYTES, scale_bf16x8(buf[j], split_scale(sa1[j])));
+                if (ng > 1) st_shared_16(dst + HS_SLOT_BYTES, scale_bf16x8(buf[j], split_scale(sa1[j])));
             }
             fence_proxy_async_smem();        // make the stores visible to the tensor core's reads
             __syncwarp();
@@ -307,21 +371,19 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
         bool ok = true;
         WorkItem w;
         for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
-            int ti, tj;
-            tile_of_slot(w.unit / p.group_pairs, ti, tj);
-            const int k0 = (w.unit % p.group_pairs) * HS_GROUPS;
-            const int ng = (p.g - k0 < HS_GROUPS) ? (p.g - k0) : HS_GROUPS;
+            const UnitDesc u = decode_unit(p, w.unit);
             if (lane == 0) ok = bounded_wait(smem_u32(&bar_acc_full), acc_ph, wc, 4u, w.unit);
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             (void)mbar_try_wait(smem_u32(&bar_acc_full), acc_ph);     // every lane observes the completed phase
             tc_fence_after_sync();
-            const int row0 = ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + q * 32;
-            for (int kk = 0; kk < ng; ++kk) {
+            const int row0 = u.ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + q * 32;
+            for (int kk = 0; kk < HS_GROUPS; ++kk) {
+                if (!u.use[kk]) continue;
 #pragma unroll 1
                 for (int c4 = 0; c4 < 4; ++c4) {
                     const int cc = half * 4 + c4;
-                    const int col0 = tj * TILE_N + cc * 32;
+                    const int col0 = u.tj[kk] * TILE_N + cc * 32;
                     if (col0 >= p.d || row0 >= p.d) break;      // outside the matrix
                     if (col0 + 32 <= row0) continue;            // 32 x 32 block strictly below the diagonal
                     uint32_t r[32];
@@ -335,7 +397,7 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        tma_reduce_add_3d(&mapH, stg, col0, row0, k0 + kk);
+                        tma_reduce_add_3d(&mapH, stg, col0, row0, u.grp[kk]);
                         bulk_commit_group();
                         bulk_wait_group_read0();      // staging block reusable once the copy engine has read it
                     }

@@ -201,6 +201,14 @@ int tiles_for(int64_t d)
     return static_cast<int>(nj * (nj + 1) / 2);
 }
 
+// Number of (row block, pair of neighbouring column blocks) slots that touch the upper triangle.
+int colpair_slots_for(int64_t d)
+{
+    const int64_t nj = (d + gq::TILE_N - 1) / gq::TILE_N;
+    const int64_t q = nj / 2;                     // complete column pairs: pair q' has 2 q' + 2 row blocks
+    return static_cast<int>(q * (q + 1) + ((nj & 1) ? nj : 0));
+}
+
 int32_t check_layer_shape(int64_t d_in, int64_t d_out, int32_t g, bool need_out)
 {
     if (g < 1 || d_in < 1) return GQ_ERR_INVALID_ARG;
@@ -315,8 +323,10 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
     p.n = static_cast<int>(n);
     p.d = static_cast<int>(d_in);
     p.g = g;
-    p.group_pairs = (g + gq::HS_GROUPS - 1) / gq::HS_GROUPS;
-    const int units = tiles_for(d_in) * p.group_pairs;
+    p.nj = static_cast<int>((d_in + gq::TILE_N - 1) / gq::TILE_N);
+    p.full_pairs = g / 2;
+    p.narrow_units = tiles_for(d_in) * p.full_pairs;
+    const int units = p.narrow_units + ((g & 1) ? colpair_slots_for(d_in) : 0);
     const int ksteps = static_cast<int>((n + gq::TILE_K - 1) / gq::TILE_K);
     const bool balanced = (flags & GQ_HESSIAN_DETERMINISTIC) == 0;
     int pairs = di->max_pairs;

@@ -134,7 +134,7 @@ __device__ __forceinline__ bool wait_gave_up(const WaitCtx &w, uint64_t t0, uint
 
 // Slow path of bounded_wait: the thread sleeps inside try_wait (woken when the phase completes) and looks at
 // the clock and the abort flag between sleeps.
-__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const WaitCtx &w, uint32_t site, uint32_t unit)
+__device__ __forceinline__ bool wait_slow(uint32_t bar, uint32_t parity, const WaitCtx &w, uint32_t site, uint32_t unit)
 {
     const uint64_t t0 = global_timer_ns();
     for (;;) {
@@ -152,7 +152,7 @@ __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, cons
 }
 
 // Wait for the MMA issuer, the one thread whose reaction time is on the critical path: polls without pause.
-__device__ __noinline__ bool bounded_wait_hot(uint32_t bar, uint32_t parity, const WaitCtx &w, uint32_t site,
+__device__ __forceinline__ bool bounded_wait_hot(uint32_t bar, uint32_t parity, const WaitCtx &w, uint32_t site,
                                              uint32_t unit)
 {
     if (mbar_try_wait(bar, parity)) return true;

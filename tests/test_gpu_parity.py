@@ -108,6 +108,9 @@ def test_saliency_empty_and_errors(dev):
     (300, 1032, 2, [300]),                  # 5 column blocks, tail of 8 features
     (96, 640, 5, [0, 96]),                  # an empty chunk is a no-op
     (1500, 3080, 2, [1000, 500]),           # 182 units on 74 SM pairs: two whole rounds plus a cut tail
+    (200, 1288, 1, [200]),                  # one group: units of two column tiles (6 column blocks)
+    (150, 1800, 3, [90, 60]),               # odd g: pair units for groups 0-1, column-pair units for group 2
+    (70, 1096, 1, [70]),                    # one group, odd number of column blocks (5): a lone last column
 ])
 def test_hessian_parity_small(dev, n, d_in, g, chunks, flags):
     gen = torch.Generator(device=dev).manual_seed(n + d_in)
