@@ -66,6 +66,7 @@ struct HessianParams {
     int d;                   // d_in
     int g;
     int nj;                  // ceil(d / 256): tile blocks per side
+    int raster;              // edge (in tiles) of the super-blocks of the tile order, see tile_of_slot_blocked
     int full_pairs;          // g / 2: pairs of groups that share a pass over X
     int narrow_units;        // tiles * full_pairs: units (tile, pair of groups)
     Schedule sched;          // units = narrow_units + (g odd ? column-pair slots : 0), ksteps = ceil(n / 64)
@@ -152,7 +153,7 @@ __device__ __forceinline__ UnitDesc decode_unit(const HessianParams &p, int unit
     UnitDesc u;
     if (unit < p.narrow_units) {
         int ti, tj;
-        tile_of_slot(unit / p.full_pairs, ti, tj);
+        tile_of_slot_blocked(unit / p.full_pairs, p.nj, p.raster, ti, tj);
         const int k0 = (unit % p.full_pairs) * 2;
         u.ti = ti;
         u.tj[0] = u.tj[1] = tj;

@@ -201,6 +201,17 @@ int tiles_for(int64_t d)
     return static_cast<int>(nj * (nj + 1) / 2);
 }
 
+// Edge of the super-blocks of the tile order: the pairs that run at the same time (pairs / units per tile
+// of them work on distinct tiles) should cover a roughly square patch of tiles.
+int raster_for(int pairs, int units_per_tile)
+{
+    int tiles_at_once = pairs / units_per_tile;
+    if (tiles_at_once < 1) tiles_at_once = 1;
+    int r = 1;
+    while ((r + 1) * (r + 1) <= tiles_at_once) ++r;
+    return r;
+}
+
 // Number of (row block, pair of neighbouring column blocks) slots that touch the upper triangle.
 int colpair_slots_for(int64_t d)
 {
@@ -325,6 +336,7 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
     p.g = g;
     p.nj = static_cast<int>((d_in + gq::TILE_N - 1) / gq::TILE_N);
     p.full_pairs = g / 2;
+    p.raster = raster_for(di->max_pairs, p.full_pairs > 0 ? p.full_pairs : 1);
     p.narrow_units = tiles_for(d_in) * p.full_pairs;
     const int units = p.narrow_units + ((g & 1) ? colpair_slots_for(d_in) : 0);
     const int ksteps = static_cast<int>((n + gq::TILE_K - 1) / gq::TILE_K);
@@ -398,6 +410,8 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     p.rows = static_cast<int>(m);
     p.g = g;
     p.n_terms = 3;                     // hi^T hi + hi^T lo + lo^T hi
+    p.nj = static_cast<int>((d_in + gq::TILE_N - 1) / gq::TILE_N);
+    p.raster = raster_for(di->max_pairs, g);
     p.term_a[0] = 0; p.term_b[0] = 0;
     p.term_a[1] = 0; p.term_b[1] = 1;
     p.term_a[2] = 1; p.term_b[2] = 0;
@@ -500,6 +514,8 @@ int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, i
     p.rows = static_cast<int>(m);
     p.g = g;
     p.n_terms = 3;
+    p.nj = static_cast<int>((d_in + gq::TILE_N - 1) / gq::TILE_N);
+    p.raster = raster_for(di->max_pairs, g);
     p.term_a[0] = 0; p.term_b[0] = 0;
     p.term_a[1] = 0; p.term_b[1] = 1;
     p.term_a[2] = 1; p.term_b[2] = 0;

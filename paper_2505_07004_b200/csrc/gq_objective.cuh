@@ -41,6 +41,8 @@ struct ObjectiveParams {
     int d;                   // number of features (d_in)
     int rows;                // contraction length of every term
     int g;                   // groups
+    int nj;                  // ceil(d / 256): tile blocks per side
+    int raster;              // edge (in tiles) of the super-blocks of the tile order
     int n_terms;
     int term_a[MAX_TERMS];   // which tensor map (0/1) feeds A / B in each term
     int term_b[MAX_TERMS];
@@ -107,7 +109,7 @@ objective_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
         WorkItem w;
         for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
             int ti, tj;
-            tile_of_slot(w.unit / p.g, ti, tj);
+            tile_of_slot_blocked(w.unit / p.g, p.nj, p.raster, ti, tj);
             const int k = w.unit % p.g;
             const int a0 = ti * TILE_M + static_cast<int>(rank) * CTA_ROWS;
             const int b0 = tj * TILE_N + static_cast<int>(rank) * CTA_ROWS;
@@ -190,7 +192,7 @@ objective_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
         WorkItem w;
         for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
             int ti, tj;
-            tile_of_slot(w.unit / p.g, ti, tj);
+            tile_of_slot_blocked(w.unit / p.g, p.nj, p.raster, ti, tj);
             const int k = w.unit % p.g;
             ok = bounded_wait(smem_u32(&bar_acc_full[buf]), acc_ph, wc, 4u, w.unit);
             ok = __all_sync(0xffffffffu, ok);

@@ -77,6 +77,46 @@ __device__ __forceinline__ void tile_of_slot(int t, int &i, int &j)
     i = t - jj * (jj + 1) / 2;
 }
 
+// The same set of tiles in an order that keeps tiles which are worked on at the same time close together in
+// BOTH directions: the upper triangle is cut into super-blocks of R x R tiles (column super-blocks outermost,
+// row super-blocks inside, tiles of a super-block row by row), so that a round of P consecutive tiles touches
+// about 2 sqrt(P) row/column blocks of X instead of P + 1.  Every (i <= j) appears exactly once for
+// t in [0, NJ (NJ + 1) / 2).
+__host__ __device__ inline void tile_of_slot_blocked(int t, int nj, int R, int &i, int &j)
+{
+    if (R <= 1) {
+        // plain column-major triangle
+        int jj = static_cast<int>((sqrtf(8.0f * static_cast<float>(t) + 1.0f) - 1.0f) * 0.5f);
+        while (jj * (jj + 1) / 2 > t) --jj;
+        while ((jj + 1) * (jj + 2) / 2 <= t) ++jj;
+        j = jj;
+        i = t - jj * (jj + 1) / 2;
+        return;
+    }
+    const int tri = R * (R + 1) / 2;
+    // tiles before super-column J (all of them complete): R^2 J (J - 1) / 2 + J tri
+    int J = static_cast<int>(sqrtf(2.0f * static_cast<float>(t) / static_cast<float>(R * R)));
+    auto before = [&](int JJ) { return R * R * (JJ * (JJ - 1) / 2) + JJ * tri; };
+    while (J > 0 && before(J) > t) --J;
+    while ((J + 1) * R < nj && before(J + 1) <= t) ++J;
+    int rem = t - before(J);
+    const int rj = (nj - J * R < R) ? (nj - J * R) : R;       // columns in this super-column
+    const int off_diag = J * R * rj;                          // tiles of the super-blocks above the diagonal one
+    if (rem < off_diag) {
+        const int I = rem / (R * rj);
+        rem -= I * R * rj;
+        i = I * R + rem / rj;
+        j = J * R + rem % rj;
+    } else {
+        rem -= off_diag;                                      // triangle of rj x rj tiles, column-major
+        int lj = static_cast<int>((sqrtf(8.0f * static_cast<float>(rem) + 1.0f) - 1.0f) * 0.5f);
+        while (lj * (lj + 1) / 2 > rem) --lj;
+        while ((lj + 1) * (lj + 2) / 2 <= rem) ++lj;
+        i = J * R + rem - lj * (lj + 1) / 2;
+        j = J * R + lj;
+    }
+}
+
 struct WorkItem {
     int unit;      // (tile slot) * g + group
     int ks0, ks1;  // k-step range [ks0, ks1) of the unit's `ksteps`
