@@ -82,11 +82,12 @@ int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad,
  *              entries with a <= b are defined; entries below the diagonal hold unspecified finite
  *              values until gq_hessian_finalize() is called.
  *   flags      0, or GQ_HESSIAN_DETERMINISTIC (see below)
- *   workspace  not used by the current kernels (gq_hessian_workspace_bytes() returns 0); may be NULL.
- *              The parameters stay in the signature so that callers written against it keep working.
- * Arithmetic: the kernel never writes a scaled copy of X to global memory.  While X is staged for the
- * tensor cores every element is multiplied by s_k[i], with s_k[i] carried as the sum of two bf16 terms
- * (16 significant bits) and packed bf16 fused multiply-adds, and rounded to bf16 once; the products
+ *   workspace  device scratch of at least gq_hessian_workspace_bytes(n_max, d_in, g, flags) bytes with
+ *              n_max >= n, 1024-byte aligned (8 bytes per token and pair of groups: s in the form the
+ *              kernel consumes); contents need not be preserved between calls.
+ * Arithmetic: the kernel never writes a scaled copy of X to global memory.  A small first kernel rewrites
+ * s_k[i] as the sum of two bf16 terms (16 significant bits).  While X is staged for the tensor cores
+ * every element is multiplied by that pair with packed bf16 fused multiply-adds and rounded to bf16 once; the products
  * (s_k[i] X[i][a]) * X[i][b] are accumulated in fp32 in tensor memory (two groups per pass over X), and
  * each call adds its fp32 tile sums to H with reduce-add transactions, so H is never read by the SMs.
  * Work is dealt to the SM pairs in whole 256 x 256 tiles of two groups; with flags == 0 the last,
@@ -100,7 +101,7 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
                               int64_t ld_s, int32_t g, float *H, uint32_t flags, void *workspace,
                               size_t workspace_bytes, void *stream);
 
-/* Scratch bytes gq_hessian_accumulate needs for chunks of up to n_max tokens: currently always 0. */
+/* Scratch bytes gq_hessian_accumulate needs for chunks of up to n_max tokens (0 on bad arguments). */
 size_t gq_hessian_workspace_bytes(int64_t n_max, int64_t d_in, int32_t g, uint32_t flags);
 
 /*
@@ -205,7 +206,8 @@ enum gq_kernel_id {
     GQ_KERNEL_SPLIT_DELTA = 3, /* W - W_hat -> bf16 hi/lo                                */
     GQ_KERNEL_GRAM_DOT = 4,    /* tensor-core Delta_k^T Delta_k contracted with H_k (Eq. 7) */
     GQ_KERNEL_REDUCE = 5,      /* fp64 reduction of the partial sums                     */
-    GQ_KERNEL_COUNT = 6
+    GQ_KERNEL_SPLIT_SALIENCY = 6, /* s -> pairs of bf16 terms for the Hessian kernel's scalers */
+    GQ_KERNEL_COUNT = 7
 };
 
 /*

@@ -25,7 +25,7 @@ EXPORTS = (
     "gq_kernel_timing_enable", "gq_kernel_timing_read", "gq_objective_noalloc",
 )
 GQ_HESSIAN_DETERMINISTIC = 1      # flag of gq_hessian_accumulate: single writer per element of H
-KERNEL_NAMES = ("saliency", "hessian", "mirror", "split_delta", "gram_dot", "reduce")
+KERNEL_NAMES = ("saliency", "hessian", "mirror", "split_delta", "gram_dot", "reduce", "split_saliency")
 
 
 class GQError(RuntimeError):

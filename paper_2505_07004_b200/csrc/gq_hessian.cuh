@@ -60,8 +60,7 @@ constexpr int HS_SMEM_BYTES = HS_STAGES * HS_STAGE_BYTES + HS_STAGING_BYTES + 10
 struct HessianParams {
     const __nv_bfloat16 *X;  // [n][ld_x]
     long long ld_x;
-    const float *s;          // [g][ld_s]
-    long long ld_s;
+    const uint2 *s2;         // [ceil(g / 2)][n]: split saliency of groups (2 q, 2 q + 1), see split_saliency_kernel
     int n;                   // tokens in this call
     int d;                   // d_in
     int g;
@@ -122,6 +121,13 @@ __device__ __forceinline__ void st_shared_16(uint32_t addr, const uint4 &v)
                  : "memory");
 }
 
+// Saliency as the scalers use it.  A value a is carried as two bf16 terms packed in one word: low half
+// hi = bf16(a), high half lo = bf16(a - hi); hi + lo has 16 significant bits.  The words of groups 2 q and
+// 2 q + 1 of a token sit side by side, so a scaler thread fetches both with one 8-byte load and does no
+// conversion work in its loop (sixteen threads share a token; converting there would be done sixteen times).
+__global__ void __launch_bounds__(256)
+split_saliency_kernel(const float *__restrict__ s, long long ld_s, int n, int g, uint2 *__restrict__ out);
+
 // A saliency value as two bf16 terms packed in one word: low half hi = bf16(a), high half lo = bf16(a - hi);
 // hi + lo carries a to 16 significant bits.
 __device__ __forceinline__ uint32_t split_scale(float a)
@@ -129,6 +135,22 @@ __device__ __forceinline__ uint32_t split_scale(float a)
     const __nv_bfloat16 hi = __float2bfloat16_rn(a);
     const __nv_bfloat16 lo = __float2bfloat16_rn(a - __bfloat162float(hi));
     return static_cast<uint32_t>(__bfloat16_as_ushort(hi)) | (static_cast<uint32_t>(__bfloat16_as_ushort(lo)) << 16);
+}
+
+__global__ void __launch_bounds__(256)
+split_saliency_kernel(const float *__restrict__ s, long long ld_s, int n, int g, uint2 *__restrict__ out)
+{
+    const int slots = (g + 1) / 2;
+    const long long total = static_cast<long long>(slots) * n;
+    for (long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total;
+         idx += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const int q = static_cast<int>(idx / n);
+        const int i = static_cast<int>(idx - static_cast<long long>(q) * n);
+        uint2 v;
+        v.x = split_scale(s[static_cast<long long>(2 * q) * ld_s + i]);
+        v.y = (2 * q + 1 < g) ? split_scale(s[static_cast<long long>(2 * q + 1) * ld_s + i]) : 0u;
+        out[idx] = v;
+    }
 }
 
 // v (8 bf16) times the split scale `a2`: per element fma(x, hi, x * lo) with packed bf16 fused multiply-adds.
@@ -300,8 +322,8 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
         // the other sets rather than by a register rotation inside one warp.
         // Inside a set, sixteen threads share a token row (16 x 16 bytes = the 128 features, so a warp reads
         // two whole 256-byte row segments per load) and eight passes cover the 64 tokens of the k-step.  Every
-        // thread fetches the saliency values of its eight tokens itself (a broadcast load per pass and group);
-        // shuffles are avoided: like every shared-memory-pipe instruction they compete with the tensor core's
+        // thread fetches the (pre-split) saliency words of its eight tokens itself, one broadcast 8-byte load per
+        // pass for both groups; shuffles are avoided: like every shared-memory-pipe instruction they compete with the tensor core's
         // operand reads.
         constexpr int TOK_PER_PASS = HS_SET_WARPS * 2;         // tokens a set covers per instruction
         constexpr int PASSES = TILE_K / TOK_PER_PASS;          // 16-byte loads per thread and k-step
@@ -317,7 +339,7 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
         int cached_it = -1;
         int ng = 0;
         const __nv_bfloat16 *xcol = nullptr;
-        const float *s0 = nullptr;
+        const uint2 *s2 = nullptr;
         bool f_ok = false;
         for (int cnt = set; cur.valid; cnt += HS_SETS, cur.advance(HS_SETS)) {
             if (cur.it != cached_it) {
@@ -327,20 +349,29 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                 const int f = u.ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + c * 8;
                 f_ok = f < p.d;
                 xcol = p.X + f;
-                s0 = p.s + static_cast<long long>(u.grp[0]) * p.ld_s;
+                s2 = p.s2 + static_cast<long long>(u.grp[0] >> 1) * p.n;
             }
             const int tok0 = cur.ks * TILE_K + trow;
-            const float *s1 = s0 + (ng > 1 ? p.ld_s : 0);
             uint4 buf[PASSES];
-            float sa0[PASSES], sa1[PASSES];
+            uint2 sv[PASSES];
+            {
+                const __nv_bfloat16 *src = xcol + static_cast<long long>(tok0) * p.ld_x;
+                const long long step = static_cast<long long>(TOK_PER_PASS) * p.ld_x;
+                const uint2 *ssrc = s2 + tok0;
+                if (f_ok && (cur.ks + 1) * TILE_K <= p.n) {         // whole k-step inside the chunk: no predicates
 #pragma unroll
-            for (int j = 0; j < PASSES; ++j) {
-                const int tok = tok0 + j * TOK_PER_PASS;
-                const bool t_ok = tok < p.n;
-                buf[j] = (f_ok && t_ok) ? ld_stream_16(xcol + static_cast<long long>(tok) * p.ld_x)
-                                        : make_uint4(0u, 0u, 0u, 0u);
-                sa0[j] = t_ok ? __ldg(s0 + tok) : 0.0f;
-                sa1[j] = t_ok ? __ldg(s1 + tok) : 0.0f;
+                    for (int j = 0; j < PASSES; ++j) {
+                        buf[j] = ld_stream_16(src + j * step);
+                        sv[j] = __ldg(ssrc + j * TOK_PER_PASS);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < PASSES; ++j) {
+                        const bool t_ok = tok0 + j * TOK_PER_PASS < p.n;
+                        buf[j] = (f_ok && t_ok) ? ld_stream_16(src + j * step) : make_uint4(0u, 0u, 0u, 0u);
+                        sv[j] = t_ok ? __ldg(ssrc + j * TOK_PER_PASS) : make_uint2(0u, 0u);
+                    }
+                }
             }
 
             const int s = cnt % HS_STAGES;
@@ -355,8 +386,8 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
             for (int j = 0; j < PASSES; ++j) {
                 const int tl = j * TOK_PER_PASS + trow;
                 const uint32_t dst = sa + static_cast<uint32_t>(tl * 128 + ((cb ^ (tl & 7)) << 4));
-                st_shared_16(dst, scale_bf16x8(buf[j], split_scale(sa0[j])));
-                if (ng > 1) st_shared_16(dst + HS_SLOT_BYTES, scale_bf16x8(buf[j], split_scale(sa1[j])));
+                st_shared_16(dst, scale_bf16x8(buf[j], sv[j].x));
+                if (ng > 1) st_shared_16(dst + HS_SLOT_BYTES, scale_bf16x8(buf[j], sv[j].y));
             }
             fence_proxy_async_smem();        // make the stores visible to the tensor core's reads
             __syncwarp();

@@ -231,8 +231,11 @@ int32_t check_layer_shape(int64_t d_in, int64_t d_out, int32_t g, bool need_out)
     return GQ_OK;
 }
 
-// The guided-Hessian kernel scales its operand on the fly: no scratch is needed.
-size_t hessian_ws_bytes(int64_t, int64_t, int32_t) { return 0; }
+// Scratch of gq_hessian_accumulate: the split saliency words, 8 bytes per (pair of groups, token).
+size_t hessian_ws_bytes(int64_t n_max, int64_t, int32_t g)
+{
+    return round_up(static_cast<size_t>((g + 1) / 2) * static_cast<size_t>(n_max) * 8, 1024);
+}
 
 struct ObjectiveLayout {
     size_t hi_off, lo_off, partials_off, total;
@@ -318,19 +321,27 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
     if (n == 0) return GQ_OK;              // an empty chunk adds nothing: pointers are not looked at
     if (!X || !s || !H) return GQ_ERR_INVALID_ARG;
     if (!aligned(X, 16) || !aligned(H, 16) || !aligned(s, 4)) return GQ_ERR_ALIGNMENT;
-    (void)workspace;
-    (void)workspace_bytes;
+    if (!workspace || workspace_bytes < hessian_ws_bytes(n, d_in, g)) return GQ_ERR_WORKSPACE;
+    if (!aligned(workspace, 1024)) return GQ_ERR_ALIGNMENT;
     DeviceInfo *di;
     if (int32_t rc = device_info(&di)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     CUtensorMap mapX, mapH;
     if (int32_t rc = make_map(&mapX, X, d_in, n, 1, ld_x, n * ld_x)) return rc;
     if (int32_t rc = make_map_h(&mapH, H, d_in, g)) return rc;
+    {
+        const int grid_s = grid_for(static_cast<long long>((g + 1) / 2) * n, 256, di->sm_count, 4);
+        {
+            LaunchScope scope(GQ_KERNEL_SPLIT_SALIENCY, st);
+            gq::split_saliency_kernel<<<grid_s, 256, 0, st>>>(s, ld_s, static_cast<int>(n), g,
+                                                             static_cast<uint2 *>(workspace));
+        }
+        GQ_CUDA(cudaGetLastError());
+    }
     gq::HessianParams p{};
     p.X = static_cast<const __nv_bfloat16 *>(X);
     p.ld_x = ld_x;
-    p.s = s;
-    p.ld_s = ld_s;
+    p.s2 = static_cast<const uint2 *>(workspace);
     p.n = static_cast<int>(n);
     p.d = static_cast<int>(d_in);
     p.g = g;

@@ -42,9 +42,12 @@ def test_version_and_status_strings(L):
 
 
 def test_workspace_sizes(L):
-    # the Hessian kernel scales its operand on the fly: no scratch for any shape or flag
-    assert L.gq_hessian_workspace_bytes(8192, 4096, 4, 0) == 0
-    assert L.gq_hessian_workspace_bytes(8192, 4096, 4, 1) == 0         # GQ_HESSIAN_DETERMINISTIC
+    # split saliency words: 8 bytes per (pair of groups, token); no scaled copy of X
+    assert L.gq_hessian_workspace_bytes(8192, 4096, 4, 0) == 2 * 8192 * 8
+    assert L.gq_hessian_workspace_bytes(8192, 4096, 5, 1) == 3 * 8192 * 8      # GQ_HESSIAN_DETERMINISTIC, odd g
+    assert L.gq_hessian_workspace_bytes(1, 8, 1, 0) == 1024                    # rounded up to 1 KiB
+    assert L.gq_hessian_workspace_bytes(8192, 4096, 4, 2) == 0                 # unknown flag
+    assert L.gq_hessian_workspace_bytes(8192, 4100, 4, 0) == 0                 # d_in % 8 != 0
     # objective: two bf16 copies of delta + 8 fp64 partial sums per (upper-triangular 256 x 256 tile, group)
     nj = 4096 // 256
     assert L.gq_objective_workspace_bytes(4096, 4096, 4) == 2 * 4096 * 4096 * 2 + (nj * (nj + 1) // 2) * 4 * 8 * 8
@@ -73,6 +76,7 @@ def test_host_side_validation_needs_no_gpu(L):
     assert L.gq_hessian_accumulate(p16, 4, 64, 64, p16, 4, 2, p16, 2, p16, 4096, None) == INVALID   # flags
     assert L.gq_hessian_accumulate(p16, 4, 60, 64, p16, 4, 2, p16, 0, p16, 4096, None) == SHAPE     # d_in % 8
     assert L.gq_hessian_accumulate(p16, 4, 64, 64, p16, 4, 2, p16 + 4, 0, p16, 4096, None) == ALIGN
+    assert L.gq_hessian_accumulate(p16, 4, 64, 64, p16, 4, 2, p16, 0, None, 0, None) == WS
     assert L.gq_hessian_accumulate(None, 0, 64, 64, None, 0, 2, None, 0, None, 0, None) == 0        # empty chunk
     assert L.gq_hessian_finalize(None, 64, 2, None) == INVALID
     # objective

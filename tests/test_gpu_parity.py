@@ -156,6 +156,9 @@ def test_hessian_errors(dev):
     H = torch.zeros((2, 64, 64), dtype=torch.float32, device=dev)
     ws = libgq.alloc_workspace(libgq.gq_hessian_workspace_bytes(16, 64, 2), dev)
     with pytest.raises(libgq.GQError) as e:
+        libgq.gq_hessian_accumulate(X, s, H, ws[:16])
+    assert "GQ_ERR_WORKSPACE" in str(e.value)
+    with pytest.raises(libgq.GQError) as e:
         libgq.gq_hessian_accumulate(X, s, H, ws, flags=2)
     assert "GQ_ERR_INVALID_ARG" in str(e.value)
     Xbad = torch.zeros((16, 68), dtype=torch.bfloat16, device=dev)
