@@ -286,30 +286,42 @@ def test_large_shapes_token_prefix(dev, name, prefix):
         torch.cuda.empty_cache()
 
 
-def test_bench_workload_full_size_sampled(dev):
-    """Config 1 at full size (131072 tokens, 16 chunks), as bench.py runs it.
+@pytest.mark.parametrize("name,g,n_tokens,s_chunks", [
+    ("c1_7b_attn", 4, None, None),      # the workload bench.py times, in full: 131072 tokens, 16 chunks
+    ("c2_7b_down", 4, None, 2),         # in full: 131072 tokens, d_in 11008 (H 1.9 GB); saliency checked on 2 chunks
+    ("c3_70b_mlp", 2, 8192, None),      # full d_in 28672 (H 6.6 GB resident), two 4096-token chunks
+    ("c4_sweep", 16, 32768, None),      # sixteen groups, two 16384-token chunks
+    ("c4_sweep", 1, 32768, 1),          # one group (units of two column tiles)
+])
+def test_full_shapes_sampled(dev, name, g, n_tokens, s_chunks):
+    """The large configurations at full layer size, launched exactly as bench.py launches them.
 
-    The oracle cannot form 4 x 4096^2 x 131072 products in seconds, so it is run exactly on a sampled
-    sub-problem: for 48 sampled input features F it computes H_k[F][:, F] from the columns X[:, F] alone,
-    which are the same entries of the full H_k; s is checked in full; the objective is checked with the
-    weight error restricted to the sampled features (W_hat = W elsewhere), which needs only those entries."""
-    cfg = synth.CONFIGS["c1_7b_attn"]
-    g = cfg.g
+    The oracle cannot form g x d_in^2 x n products in seconds, so it is run exactly on a sampled
+    sub-problem: for ~48 sampled input features F it computes H_k[F][:, F] from the columns X[:, F] alone,
+    which are the same entries of the full H_k; s is checked against the oracle on whole chunks; the objective
+    is checked with the weight error restricted to the sampled features (W_hat = W elsewhere), which needs
+    only those entries of H."""
+    base = synth.CONFIGS[name]
+    cfg = synth.LayerConfig(base.name, base.n if n_tokens is None else n_tokens, base.chunk, base.d_in, base.d_out,
+                            (g,), base.x_kind, base.outlier_frac, base.outlier_mult)
     xs, gs, ss, H, W, What, loss = run_layer(cfg, dev)
     rng = np.random.default_rng(0)
     syn = synth.LayerSynth(cfg, dev, seed=0)
-    F = np.sort(np.concatenate([rng.choice(cfg.d_in, 40, replace=False),
-                                syn.outlier_features[:8].cpu().numpy()]))
-    F = np.unique(F)
+    F = np.unique(np.concatenate([rng.choice(cfg.d_in, 40, replace=False), syn.outlier_features[:8].cpu().numpy()]))
     Ft = torch.from_numpy(F).to(dev)
     xb = np.concatenate([synth.bf16_bits(x[:, Ft].contiguous()) for x in xs])          # [n, |F|]
-    # saliency: the oracle on the whole gradient (one pass over 1 GB on the host)
-    s_ref = np.concatenate([orc.saliency(synth.bf16_bits(gc), g) for gc in gs], axis=1)
-    check_s(torch.cat(ss, dim=1), s_ref)
-    H_ref = orc.hessian(xb, s_ref)                                                     # [g, |F|, |F|]
+    # saliency: the oracle on whole chunks of the gradient
+    n_s = len(gs) if s_chunks is None else s_chunks
+    s_ref_part = np.concatenate([orc.saliency(synth.bf16_bits(gc), g) for gc in gs[:n_s]], axis=1)
+    check_s(torch.cat(ss[:n_s], dim=1), s_ref_part)
+    # H on the sampled features, from the GPU's saliency where the oracle's was not computed (it was checked
+    # above on the chunks where both exist, to 1e-4)
+    s_all = torch.cat(ss, dim=1).cpu().numpy().astype(np.float64)
+    s_all[:, :s_ref_part.shape[1]] = s_ref_part
+    H_ref = orc.hessian(xb, s_all)                                                     # [g, |F|, |F|]
     H_sub = H[:, Ft][:, :, Ft]
     check_H(H_sub, H_ref)
-    Hc = H[0].cpu()
+    Hc = H[g - 1, :2048, :2048].cpu()
     assert torch.equal(Hc, Hc.T)
     # objective: restrict to the sampled features by zeroing delta elsewhere (W_hat = W off F)
     mask = torch.zeros(cfg.d_in, dtype=torch.bool, device=dev)
@@ -321,6 +333,8 @@ def test_bench_workload_full_size_sampled(dev):
     loss_ref = orc.objective(W[:, Ft].contiguous().cpu().numpy(), What[:, Ft].contiguous().cpu().numpy(), H_ref)
     check_loss(loss_f, loss_ref)
     assert np.all(loss.cpu().numpy() > 0)
+    del xs, gs, ss, H, W, What, What_f, ows
+    torch.cuda.empty_cache()
 
 
 # ------------------------------------------------------------------------------------------ host path
