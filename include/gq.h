@@ -185,6 +185,37 @@ int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, i
                              const float *H, int32_t g, double *loss_out, void *stream);
 
 /*
+ * Cyclic coordinate descent on the objective of Eq. 7 with fixed per-channel codebooks: the assignment
+ * step of the layer-wise quantiser (Section 4.2, Eq. 10; Appendix B.2, Algorithm 4).  For every group k and
+ * every channel j in J_k, `cycles` times, the coordinates i = 0 .. d_in - 1 are visited in order and set to
+ *     W_hat[j][i] = Round_j( W[j][i] - (1 / H_k[i][i]) * sum_{c != i} H_k[i][c] * (W_hat[j][c] - W[j][c]) ),
+ * Round_j = the nearest of codebook[j][0 .. m-1] (ties: the smaller index), using the current W_hat of all
+ * other coordinates.  Started from a W_hat whose entries are codebook values this never increases a
+ * channel's objective (Proposition 1).
+ *
+ *   W          fp32 [d_out, d_in], 16-byte aligned (row j = output channel j)
+ *   W_hat      fp32 [d_out, d_in], in: the starting point, out: the result (every entry a codebook value)
+ *   Q          uint8 [d_out, d_in], out: index of W_hat[j][i] in codebook[j]
+ *   codebook   fp32 [d_out, m], 1 <= m <= 16 (need not be sorted)
+ *   H          fp32 [g, d_in, d_in], FULL symmetric matrices (after gq_hessian_finalize), 16-byte aligned.
+ *              A coordinate with H_k[i][i] <= 0 is rounded to the codebook value nearest to W[j][i].
+ *   cycles     >= 0 (0 only transposes W_hat through the workspace and back; Q is then all zero)
+ *   workspace  device scratch of at least gq_cd_workspace_bytes(d_in, d_out, g) bytes, 1024-byte aligned
+ * Same shape rules as gq_objective.
+ * Arithmetic: coordinates are processed in blocks of 256.  The contributions of the coordinates outside
+ * a block are formed on the tensor cores from bf16 hi + lo splits of H and W_hat - W (three products,
+ * fp32 accumulation: about 16 significant bits per factor); everything inside a block, and the rounding
+ * decision, is fp32.  Decisions can therefore differ from exact arithmetic only where the rounding
+ * target lies within about 1e-5 (relative to the values involved) of the midpoint between two codebook
+ * values; from such a coordinate on that channel follows its own, equally valid, descent path.
+ */
+int32_t gq_cd_cycles(const float *W, float *W_hat, uint8_t *Q, const float *codebook, int32_t m,
+                     int64_t d_in, int64_t d_out, const float *H, int32_t g, int32_t cycles,
+                     void *workspace, size_t workspace_bytes, void *stream);
+
+size_t gq_cd_workspace_bytes(int64_t d_in, int64_t d_out, int32_t g);
+
+/*
  * Synchronises `stream`, then returns and clears the first device-side error recorded on the
  * current device since the last gq_check (GQ_OK if none).  A pipeline wait inside a kernel that
  * exceeds its time budget (2 s by default; environment variable GQ_WAIT_BUDGET_MS) makes the
@@ -207,7 +238,10 @@ enum gq_kernel_id {
     GQ_KERNEL_GRAM_DOT = 4,    /* tensor-core Delta_k^T Delta_k contracted with H_k (Eq. 7) */
     GQ_KERNEL_REDUCE = 5,      /* fp64 reduction of the partial sums                     */
     GQ_KERNEL_SPLIT_SALIENCY = 6, /* s -> pairs of bf16 terms for the Hessian kernel's scalers */
-    GQ_KERNEL_COUNT = 7
+    GQ_KERNEL_CD_PANEL = 7,    /* coordinate descent: tensor-core product with the coordinates outside a block */
+    GQ_KERNEL_CD_BLOCK = 8,    /* coordinate descent: the 256 coordinates of a block, in order */
+    GQ_KERNEL_CD_AUX = 9,      /* coordinate descent: transposes and bf16 splits */
+    GQ_KERNEL_COUNT = 10
 };
 
 /*

@@ -104,6 +104,20 @@ def cd_rowwise(W, W_hat0, codebook, H, cycles: int = 1):
     return What.astype(np.float32), Q
 
 
+def coordinate_target(w_j: np.ndarray, what_j: np.ndarray, Hk: np.ndarray, i: int):
+    """The argument of Round_j in Eq. 10 for coordinate i of one channel, given the channel's current
+    quantised weights: ``W_ij - sum_{c != i} H_ic / H_ii (What_cj - W_cj)``; also returns the magnitude
+    ``|W_ij| + sum_{c != i} |H_ic / H_ii (What_cj - W_cj)|`` of what was summed."""
+    w = np.asarray(w_j, dtype=np.float64)
+    e = np.asarray(what_j, dtype=np.float64) - w
+    h = np.asarray(Hk[i], dtype=np.float64)
+    if h[i] <= 0:
+        return float(w[i]), float(abs(w[i]))
+    terms = h / h[i] * e
+    terms[i] = 0.0
+    return float(w[i] - terms.sum()), float(abs(w[i]) + np.abs(terms).sum())
+
+
 def channel_objective(delta: np.ndarray, Hk: np.ndarray) -> float:
     """delta^T H_k delta (one term of Eq. 7)."""
     return float(delta @ Hk @ delta)

@@ -22,10 +22,11 @@ EXPORTS = (
     "gq_version", "gq_status_string", "gq_last_cuda_error", "gq_saliency", "gq_hessian_accumulate",
     "gq_hessian_workspace_bytes", "gq_hessian_finalize", "gq_objective", "gq_objective_workspace_bytes",
     "gq_layer_objective_host", "gq_layer_host_arena_bytes", "gq_check", "gq_launch_count",
-    "gq_kernel_timing_enable", "gq_kernel_timing_read", "gq_objective_noalloc",
+    "gq_kernel_timing_enable", "gq_kernel_timing_read", "gq_objective_noalloc", "gq_cd_cycles", "gq_cd_workspace_bytes",
 )
 GQ_HESSIAN_DETERMINISTIC = 1      # flag of gq_hessian_accumulate: single writer per element of H
-KERNEL_NAMES = ("saliency", "hessian", "mirror", "split_delta", "gram_dot", "reduce", "split_saliency")
+KERNEL_NAMES = ("saliency", "hessian", "mirror", "split_delta", "gram_dot", "reduce", "split_saliency", "cd_panel",
+                "cd_block", "cd_aux")
 
 
 class GQError(RuntimeError):
@@ -74,6 +75,10 @@ def lib() -> ctypes.CDLL:
         L.gq_check.argtypes = [vp, vp]
         L.gq_objective_noalloc.restype = i32
         L.gq_objective_noalloc.argtypes = [vp, vp, i64, i64, vp, i32, vp, vp]
+        L.gq_cd_workspace_bytes.restype = sz
+        L.gq_cd_workspace_bytes.argtypes = [i64, i64, i32]
+        L.gq_cd_cycles.restype = i32
+        L.gq_cd_cycles.argtypes = [vp, vp, vp, vp, i32, i64, i64, vp, i32, i32, vp, sz, vp]
         L.gq_kernel_timing_enable.restype = i32
         L.gq_kernel_timing_enable.argtypes = [i32]
         L.gq_kernel_timing_read.restype = i32
@@ -278,3 +283,34 @@ def gq_objective_noalloc(W: torch.Tensor, W_hat: torch.Tensor, H: torch.Tensor, 
     if rc:
         raise GQError("gq_objective_noalloc", rc)
     return loss
+
+
+def gq_cd_workspace_bytes(d_in: int, d_out: int, g: int) -> int:
+    return int(lib().gq_cd_workspace_bytes(d_in, d_out, g))
+
+
+def gq_cd_cycles(W: torch.Tensor, W_hat: torch.Tensor, codebook: torch.Tensor, H: torch.Tensor, cycles: int,
+                 workspace: torch.Tensor, Q: Optional[torch.Tensor] = None, stream=None):
+    """Cyclic coordinate descent with fixed codebooks (Eq. 10, Algorithm 4): updates ``W_hat`` in place and
+    returns ``(W_hat, Q)`` with ``Q`` the uint8 codebook indices."""
+    _dev(W, torch.float32, "W")
+    _dev(W_hat, torch.float32, "W_hat")
+    _dev(codebook, torch.float32, "codebook")
+    _dev(H, torch.float32, "H")
+    if W.dim() != 2 or W.shape != W_hat.shape or not W.is_contiguous() or not W_hat.is_contiguous():
+        raise ValueError("W and W_hat must be contiguous [d_out, d_in]")
+    d_out, d_in = W.shape
+    g = H.shape[0]
+    if tuple(H.shape) != (g, d_in, d_in) or not H.is_contiguous():
+        raise ValueError("H must be a contiguous [g, d_in, d_in] tensor")
+    if codebook.dim() != 2 or codebook.shape[0] != d_out or not codebook.is_contiguous():
+        raise ValueError("codebook must be a contiguous [d_out, m] tensor")
+    if Q is None:
+        Q = torch.empty((d_out, d_in), dtype=torch.uint8, device=W.device)
+    _dev(Q, torch.uint8, "Q")
+    rc = lib().gq_cd_cycles(W.data_ptr(), W_hat.data_ptr(), Q.data_ptr(), codebook.data_ptr(), codebook.shape[1], d_in,
+                            d_out, H.data_ptr(), g, int(cycles), workspace.data_ptr(),
+                            workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc:
+        raise GQError("gq_cd_cycles", rc)
+    return W_hat, Q

@@ -15,6 +15,7 @@
 #include "../../include/gq.h"
 #include "gq_hessian.cuh"
 #include "gq_objective.cuh"
+#include "gq_cd.cuh"
 #include "gq_kernels.cuh"
 
 #define GQ_VERSION_NUMBER 100   /* 0.1.0 */
@@ -94,8 +95,12 @@ int32_t device_info(DeviceInfo **out)
         void *sym = nullptr;
         GQ_CUDA(cudaGetSymbolAddress(&sym, g_status_word));
         di.status_ptr = static_cast<uint32_t *>(sym);
-        GQ_CUDA(cudaFuncSetAttribute(gq::objective_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     gq::OBJ_SMEM_BYTES));
+        GQ_CUDA(cudaFuncSetAttribute(gq::pair_gemm_kernel<gq::MODE_OBJECTIVE>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, gq::OBJ_SMEM_BYTES));
+        GQ_CUDA(cudaFuncSetAttribute(gq::pair_gemm_kernel<gq::MODE_PANEL>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, gq::OBJ_SMEM_BYTES));
+        GQ_CUDA(cudaFuncSetAttribute(gq::cd_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     gq::CD_SMEM_BYTES));
         GQ_CUDA(cudaFuncSetAttribute(gq::hessian_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      gq::HS_SMEM_BYTES));
         {
@@ -249,6 +254,30 @@ ObjectiveLayout objective_layout(int64_t d_in, int64_t d_out, int32_t g)
     L.partials_off = 2 * mat;
     L.total = L.partials_off +
               round_up(static_cast<size_t>(tiles_for(d_in)) * g * gq::PARTIALS_PER_UNIT * sizeof(double), 1024);
+    return L;
+}
+
+struct CdLayout {
+    size_t wt, wht, et, ehi, elo, hhi, hlo, rdiag, p, qt, total;
+};
+CdLayout cd_layout(int64_t d_in, int64_t d_out, int32_t g)
+{
+    CdLayout L;
+    const size_t mat4 = round_up(static_cast<size_t>(d_in) * d_out * 4, 1024);
+    const size_t mat2 = round_up(static_cast<size_t>(d_in) * d_out * 2, 1024);
+    const size_t h2 = round_up(static_cast<size_t>(g) * d_in * d_in * 2, 1024);
+    size_t o = 0;
+    L.wt = o; o += mat4;
+    L.wht = o; o += mat4;
+    L.et = o; o += mat4;
+    L.ehi = o; o += mat2;
+    L.elo = o; o += mat2;
+    L.hhi = o; o += h2;
+    L.hlo = o; o += h2;
+    L.rdiag = o; o += round_up(static_cast<size_t>(g) * d_in * 4, 1024);
+    L.p = o; o += round_up(static_cast<size_t>(gq::CD_BLOCK) * d_out * 4, 1024);
+    L.qt = o; o += round_up(static_cast<size_t>(d_in) * d_out, 1024);
+    L.total = o;
     return L;
 }
 
@@ -416,7 +445,7 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     CUtensorMap mapHi, mapLo;
     if (int32_t rc = make_map(&mapHi, hi, d_in, m, g, d_in, m * d_in)) return rc;
     if (int32_t rc = make_map(&mapLo, lo, d_in, m, g, d_in, m * d_in)) return rc;
-    gq::ObjectiveParams p{};
+    gq::PairGemmParams p{};
     p.d = static_cast<int>(d_in);
     p.rows = static_cast<int>(m);
     p.g = g;
@@ -439,7 +468,7 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     const int grid = 2 * p.sched.pairs;
     {
         LaunchScope scope(GQ_KERNEL_GRAM_DOT, st);
-        gq::objective_kernel<<<grid, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(mapHi, mapLo, p);
+        gq::pair_gemm_kernel<gq::MODE_OBJECTIVE><<<grid, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(mapHi, mapLo, mapHi, mapLo, p);
     }
     GQ_CUDA(cudaGetLastError());
     {
@@ -520,7 +549,7 @@ int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, i
     CUtensorMap mapHi, mapLo;
     if (int32_t rc = make_map(&mapHi, hi, d_in, m, g, d_in, m * d_in)) return rc;
     if (int32_t rc = make_map(&mapLo, lo, d_in, m, g, d_in, m * d_in)) return rc;
-    gq::ObjectiveParams p{};
+    gq::PairGemmParams p{};
     p.d = static_cast<int>(d_in);
     p.rows = static_cast<int>(m);
     p.g = g;
@@ -540,11 +569,126 @@ int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, i
     p.status = di->status_ptr;
     p.wait_budget_ns = wait_budget_ns();
     const int grid = 2 * p.sched.pairs;
-    gq::objective_kernel<<<grid, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(mapHi, mapLo, p);
+    gq::pair_gemm_kernel<gq::MODE_OBJECTIVE><<<grid, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(mapHi, mapLo, mapHi, mapLo, p);
     g_launches.fetch_add(1);
     GQ_CUDA(cudaGetLastError());
     gq::reduce_partials_kernel<<<1, 1024, 0, st>>>(partials, tiles, g, gq::PARTIALS_PER_UNIT, loss_out);
     g_launches.fetch_add(1);
+    GQ_CUDA(cudaGetLastError());
+    return GQ_OK;
+}
+
+size_t gq_cd_workspace_bytes(int64_t d_in, int64_t d_out, int32_t g)
+{
+    if (check_layer_shape(d_in, d_out, g, true) != GQ_OK) return 0;
+    return cd_layout(d_in, d_out, g).total;
+}
+
+int32_t gq_cd_cycles(const float *W, float *W_hat, uint8_t *Q, const float *codebook, int32_t m, int64_t d_in,
+                     int64_t d_out, const float *H, int32_t g, int32_t cycles, void *workspace,
+                     size_t workspace_bytes, void *stream)
+{
+    if (!W || !W_hat || !Q || !codebook || !H || cycles < 0 || m < 1) return GQ_ERR_INVALID_ARG;
+    if (int32_t rc = check_layer_shape(d_in, d_out, g, true)) return rc;
+    if (m > gq::CD_MAX_LEVELS) return GQ_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned(W, 16) || !aligned(W_hat, 16) || !aligned(H, 16) || !aligned(codebook, 4)) return GQ_ERR_ALIGNMENT;
+    const CdLayout L = cd_layout(d_in, d_out, g);
+    if (!workspace || workspace_bytes < L.total) return GQ_ERR_WORKSPACE;
+    if (!aligned(workspace, 1024)) return GQ_ERR_ALIGNMENT;
+    DeviceInfo *di;
+    if (int32_t rc = device_info(&di)) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    float *Wt = reinterpret_cast<float *>(ws + L.wt);
+    float *Wht = reinterpret_cast<float *>(ws + L.wht);
+    float *Et = reinterpret_cast<float *>(ws + L.et);
+    __nv_bfloat16 *Ehi = reinterpret_cast<__nv_bfloat16 *>(ws + L.ehi);
+    __nv_bfloat16 *Elo = reinterpret_cast<__nv_bfloat16 *>(ws + L.elo);
+    __nv_bfloat16 *Hhi = reinterpret_cast<__nv_bfloat16 *>(ws + L.hhi);
+    __nv_bfloat16 *Hlo = reinterpret_cast<__nv_bfloat16 *>(ws + L.hlo);
+    float *rdiag = reinterpret_cast<float *>(ws + L.rdiag);
+    float *P = reinterpret_cast<float *>(ws + L.p);
+    uint8_t *Qt = ws + L.qt;
+    const int64_t mk = d_out / g;
+    const dim3 tgrid(static_cast<unsigned>((d_in + 31) / 32), static_cast<unsigned>((d_out + 31) / 32));
+    {
+        LaunchScope scope(GQ_KERNEL_CD_AUX, st);
+        gq::cd_prepare_kernel<<<tgrid, 256, 0, st>>>(W, W_hat, static_cast<int>(d_in), static_cast<int>(d_out), Wt, Wht,
+                                                     Et, Ehi, Elo);
+    }
+    GQ_CUDA(cudaGetLastError());
+    {
+        const long long count = static_cast<long long>(g) * d_in * d_in;
+        LaunchScope scope(GQ_KERNEL_CD_AUX, st);
+        gq::cd_split_h_kernel<<<grid_for(count, 256, di->sm_count, 8), 256, 0, st>>>(H, count, static_cast<int>(d_in), Hhi,
+                                                                                 Hlo, rdiag);
+    }
+    GQ_CUDA(cudaGetLastError());
+
+    CUtensorMap mapHhi, mapHlo, mapEhi, mapElo;
+    if (int32_t rc = make_map(&mapHhi, Hhi, d_in, d_in, g, d_in, d_in * d_in)) return rc;
+    if (int32_t rc = make_map(&mapHlo, Hlo, d_in, d_in, g, d_in, d_in * d_in)) return rc;
+    if (int32_t rc = make_map(&mapEhi, Ehi, d_out, d_in, 1, d_out, d_in * d_out)) return rc;
+    if (int32_t rc = make_map(&mapElo, Elo, d_out, d_in, 1, d_out, d_in * d_out)) return rc;
+    const int kblocks = static_cast<int>((d_in + gq::TILE_K - 1) / gq::TILE_K);
+    const int ch_tiles = static_cast<int>((mk + gq::TILE_N - 1) / gq::TILE_N);
+    const int slices = static_cast<int>((mk + gq::CD_CH - 1) / gq::CD_CH);
+
+    for (int32_t cyc = 0; cyc < cycles; ++cyc) {
+        for (int64_t s0 = 0; s0 < d_in; s0 += gq::CD_BLOCK) {
+            const int rows = static_cast<int>(d_in - s0 < gq::CD_BLOCK ? d_in - s0 : gq::CD_BLOCK);
+            const int blk_ksteps = (rows + gq::TILE_K - 1) / gq::TILE_K;
+            const int nk = kblocks - blk_ksteps;
+            GQ_CUDA(cudaMemsetAsync(P, 0, static_cast<size_t>(gq::CD_BLOCK) * d_out * sizeof(float), st));
+            if (nk > 0) {
+                gq::PairGemmParams pp{};
+                pp.d = static_cast<int>(d_in);
+                pp.g = g;
+                pp.n_terms = 3;                    // Hhi Ehi + Hhi Elo + Hlo Ehi
+                pp.term_a[0] = 0; pp.term_b[0] = 2;
+                pp.term_a[1] = 0; pp.term_b[1] = 3;
+                pp.term_a[2] = 1; pp.term_b[2] = 2;
+                pp.map_grouped[0] = 1; pp.map_grouped[1] = 1; pp.map_grouped[2] = 0; pp.map_grouped[3] = 0;
+                pp.s0 = static_cast<int>(s0);
+                pp.blk_ksteps = blk_ksteps;
+                pp.nk = nk;
+                pp.ch_tiles = ch_tiles;
+                pp.mk = static_cast<int>(mk);
+                pp.d_out = static_cast<int>(d_out);
+                pp.P = P;
+                const int tiles = g * ch_tiles;
+                int pieces = di->max_pairs / tiles;              // cut the contraction so that every pair has work
+                if (pieces < 1) pieces = 1;
+                if (pieces > 3 * nk) pieces = 3 * nk;
+                pp.pieces = pieces;
+                const int ksteps = (3 * nk + pieces - 1) / pieces;
+                const int units = tiles * pieces;
+                pp.sched = gq::plan_schedule(units, ksteps, units < di->max_pairs ? units : di->max_pairs, false);
+                pp.status = di->status_ptr;
+                pp.wait_budget_ns = wait_budget_ns();
+                {
+                    LaunchScope scope(GQ_KERNEL_CD_PANEL, st);
+                    gq::pair_gemm_kernel<gq::MODE_PANEL><<<2 * pp.sched.pairs, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(
+                        mapHhi, mapHlo, mapEhi, mapElo, pp);
+                }
+                GQ_CUDA(cudaGetLastError());
+            }
+            gq::CdBlockParams bp{};
+            bp.H = H; bp.rdiag = rdiag; bp.P = P; bp.Wt = Wt; bp.codebook = codebook; bp.Wht = Wht; bp.Et = Et;
+            bp.Ehi = Ehi; bp.Elo = Elo; bp.Qt = Qt;
+            bp.d_in = static_cast<int>(d_in); bp.d_out = static_cast<int>(d_out); bp.g = g; bp.mk = static_cast<int>(mk);
+            bp.m = m; bp.s0 = static_cast<int>(s0); bp.rows = rows; bp.slices = slices;
+            {
+                LaunchScope scope(GQ_KERNEL_CD_BLOCK, st);
+                gq::cd_block_kernel<<<g * slices, gq::CD_THREADS, gq::CD_SMEM_BYTES, st>>>(bp);
+            }
+            GQ_CUDA(cudaGetLastError());
+        }
+    }
+    {
+        LaunchScope scope(GQ_KERNEL_CD_AUX, st);
+        gq::cd_finish_kernel<<<tgrid, 256, 0, st>>>(Wht, Qt, static_cast<int>(d_in), static_cast<int>(d_out), W_hat, Q);
+    }
     GQ_CUDA(cudaGetLastError());
     return GQ_OK;
 }

@@ -1,24 +1,28 @@
-// Objective of Eq. 7 on the tensor cores:  loss_k = <H_k, Delta_k^T Delta_k>  with
+// Pair GEMM: the tensor-core kernel behind gq_objective (Eq. 7) and behind the panel products of the
+// coordinate-descent cycles (Appendix B.2, Algorithm 4).  Both are sums over a contraction index of
+// products of MN-major bf16 operands (rows = contraction index, contiguous columns = the output index),
 //
-//     D_k[a][b] = sum_terms sum_j  A_term[k][j][a] * B_term[k][j][b]        (j: output channels of group k)
+//     D[a][b] = sum_terms sum_r  A_term[r][a] * B_term[r][b],
 //
-// where Delta = W - W_hat is held as two bf16 matrices (hi + lo) and the three terms hi^T hi + hi^T lo +
-// lo^T hi are accumulated into the same tensor-memory tile, and with the symmetry of H_k
-//
-//     loss_k = sum_{a <= b} (2 - [a == b]) * D_k[a][b] * H_k[a][b].
-//
-// Operands are row-major bf16 matrices whose rows are the contraction index (output channels) and whose
-// columns are the d_in input features, so both MMA operands are "MN-major" (feature-contiguous).
-// CTA pairs, 256 x 256 tiles and the work distribution are described in gq_pipeline.cuh; work unit =
-// (upper-triangular tile, group), whole units only (each unit writes its own partial sums, so the result is
-// reproducible).  Roles inside a CTA:
+// with fp32 values carried as two bf16 matrices (hi + lo) and the three terms hi hi + hi lo + lo hi
+// accumulated into the same tensor-memory tile.  CTA pairs, 256 x 256 tiles and the work distribution are
+// described in gq_pipeline.cuh.  Roles inside a CTA:
 //   warp 0 (one lane)  TMA producer: 64-row x 64-feature boxes, 128-byte swizzle, ring of OBJ_STAGES stages;
 //                      byte counts of both CTAs are collected on the first CTA's "full" barriers
 //   warp 1 (one lane)  MMA issuer (first CTA of the pair only); its commits signal both CTAs
 //   warp 2             TMEM allocation / release (all 512 columns: two 256-column accumulators)
-//   warps 4..7         epilogue: tcgen05.ld the finished accumulator, multiply with the H_k tile read from
-//                      global memory, fp64 partial sum per (unit, CTA, warp); runs while the next tile is
-//                      computed into the other accumulator
+//   warps 4..7         epilogue: tcgen05.ld the finished accumulator while the next tile is computed into
+//                      the other accumulator
+//
+// MODE_OBJECTIVE   loss_k = <H_k, Delta_k^T Delta_k>: A, B = Delta = W - W_hat of group k (rows = output
+//                  channels), upper-triangular tiles only, epilogue
+//                  sum_{a <= b} (2 - [a == b]) * D[a][b] * H_k[a][b] as one fp64 partial per (unit, CTA, warp);
+//                  whole units only, so the result is reproducible.
+// MODE_PANEL       P[r][ch] += sum_{c outside the block} H_k[c][s0 + r] * E[c][ch] for the 256 rows of one
+//                  coordinate block: A = H_k (rows = contraction index c, by symmetry H[c][r] = H[r][c]),
+//                  B = E = (What - W)^T (rows = input coordinates c, columns = output channels); work unit =
+//                  (group, tile of 256 channels, piece of the contraction range); the pieces of a tile are
+//                  added into P with red.global.add.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -37,26 +41,88 @@ constexpr int OBJ_SMEM_BYTES = OBJ_STAGES * OBJ_STAGE_BYTES + 1024;   // + slack
 constexpr int MAX_TERMS = 3;
 constexpr int PARTIALS_PER_UNIT = 8;                   // one fp64 per (CTA of the pair, epilogue warp)
 
-struct ObjectiveParams {
+constexpr int MODE_OBJECTIVE = 0;
+constexpr int MODE_PANEL = 1;
+
+struct PairGemmParams {
     int d;                   // number of features (d_in)
-    int rows;                // contraction length of every term
+    int rows;                // MODE_OBJECTIVE: contraction length of every term
     int g;                   // groups
     int nj;                  // ceil(d / 256): tile blocks per side
     int raster;              // edge (in tiles) of the super-blocks of the tile order
     int n_terms;
-    int term_a[MAX_TERMS];   // which tensor map (0/1) feeds A / B in each term
+    int term_a[MAX_TERMS];   // which of the four tensor maps feeds A / B in each term
     int term_b[MAX_TERMS];
-    int map_grouped[2];      // 1: the map's third coordinate is the group index; 0: always 0
+    int map_grouped[4];      // 1: the map's third coordinate is the group index; 0: always 0
     Schedule sched;          // units = (number of upper-triangular 256 x 256 tiles) * g,
                              // ksteps = n_terms * ceil(rows / 64)
-    const float *H;          // [g][d][d], only a <= b is read
-    double *partials;        // [units][PARTIALS_PER_UNIT]
+    const float *H;          // MODE_OBJECTIVE: [g][d][d], only a <= b is read
+    double *partials;        // MODE_OBJECTIVE: [units][PARTIALS_PER_UNIT]
+    // MODE_PANEL
+    int s0;                  // first coordinate of the block
+    int blk_ksteps;          // 64-row k-steps covered by the block itself (left out of the contraction)
+    int nk;                  // 64-row k-steps outside the block (per term)
+    int ch_tiles;            // tiles of 256 channels per group
+    int pieces;              // pieces of the contraction range per (group, channel tile); sched.ksteps each
+    int mk;                  // channels per group
+    int d_out;
+    float *P;                // [256][d_out]
     uint32_t *status;        // device status word (4 x u32)
     unsigned long long wait_budget_ns;
 };
 
+// Where a work item's operands start and which k-steps it covers.
+struct ItemGeom {
+    int ti, tj;      // MODE_OBJECTIVE: tile
+    int k;           // group
+    int a0, b0;      // first A / B column this CTA loads
+    int ks0, ks1;    // k-steps [ks0, ks1) of the flattened (term, row block) range
+};
+
+template <int MODE>
+__device__ __forceinline__ bool item_geom(const PairGemmParams &p, const WorkItem &w, uint32_t rank, ItemGeom &ge)
+{
+    if (MODE == MODE_OBJECTIVE) {
+        tile_of_slot_blocked(w.unit / p.g, p.nj, p.raster, ge.ti, ge.tj);
+        ge.k = w.unit % p.g;
+        ge.a0 = ge.ti * TILE_M + static_cast<int>(rank) * CTA_ROWS;
+        ge.b0 = ge.tj * TILE_N + static_cast<int>(rank) * CTA_ROWS;
+        ge.ks0 = w.ks0;
+        ge.ks1 = w.ks1;
+        return true;
+    }
+    const int piece = w.unit % p.pieces;
+    const int t = (w.unit / p.pieces) % p.ch_tiles;
+    ge.k = w.unit / (p.pieces * p.ch_tiles);
+    ge.ti = 0;
+    ge.tj = t;
+    ge.a0 = p.s0 + static_cast<int>(rank) * CTA_ROWS;
+    ge.b0 = ge.k * p.mk + t * TILE_N + static_cast<int>(rank) * CTA_ROWS;
+    ge.ks0 = piece * p.sched.ksteps;
+    const int total = p.n_terms * p.nk;
+    ge.ks1 = (ge.ks0 + p.sched.ksteps < total) ? ge.ks0 + p.sched.ksteps : total;
+    return ge.ks1 > ge.ks0;          // a piece beyond the end of the range has nothing to do: every role skips it
+}
+
+// Term and first contraction row of flattened k-step ks.
+template <int MODE>
+__device__ __forceinline__ void kstep_coords(const PairGemmParams &p, int ks, int kblocks, int &term, int &row)
+{
+    if (MODE == MODE_OBJECTIVE) {
+        term = ks / kblocks;
+        row = (ks - term * kblocks) * TILE_K;
+    } else {
+        term = ks / p.nk;
+        const int kb = ks - term * p.nk;
+        row = (kb < p.s0 / TILE_K ? kb : kb + p.blk_ksteps) * TILE_K;
+    }
+}
+
+template <int MODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(OBJ_THREADS, 1)
-objective_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1, const ObjectiveParams p)
+pair_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1,
+                 const __grid_constant__ CUtensorMap map2, const __grid_constant__ CUtensorMap map3,
+                 const PairGemmParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[OBJ_STAGES];      // used in the pair's first CTA only
@@ -87,6 +153,8 @@ objective_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
         fence_mbar_init();
         prefetch_tensormap(&map0);
         prefetch_tensormap(&map1);
+        prefetch_tensormap(&map2);
+        prefetch_tensormap(&map3);
     }
     if (warp == 2) {
         tmem_alloc(smem_u32(&tmem_base_smem), TMEM_COLS);
@@ -108,19 +176,17 @@ objective_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
         bool ok = true;
         WorkItem w;
         for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
-            int ti, tj;
-            tile_of_slot_blocked(w.unit / p.g, p.nj, p.raster, ti, tj);
-            const int k = w.unit % p.g;
-            const int a0 = ti * TILE_M + static_cast<int>(rank) * CTA_ROWS;
-            const int b0 = tj * TILE_N + static_cast<int>(rank) * CTA_ROWS;
-            for (int ks = w.ks0; ks < w.ks1; ++ks) {
-                const int term = ks / kblocks;
-                const int r = ks - term * kblocks;
+            ItemGeom ge;
+            if (!item_geom<MODE>(p, w, rank, ge)) continue;
+            const void *maps[4] = {&map0, &map1, &map2, &map3};
+            for (int ks = ge.ks0; ks < ge.ks1; ++ks) {
+                int term, row;
+                kstep_coords<MODE>(p, ks, kblocks, term, row);
                 const int ma = p.term_a[term], mb = p.term_b[term];
-                const void *amap = ma ? static_cast<const void *>(&map1) : static_cast<const void *>(&map0);
-                const void *bmap = mb ? static_cast<const void *>(&map1) : static_cast<const void *>(&map0);
-                const int ka = p.map_grouped[ma] ? k : 0;
-                const int kb = p.map_grouped[mb] ? k : 0;
+                const void *amap = maps[ma];
+                const void *bmap = maps[mb];
+                const int ka = p.map_grouped[ma] ? ge.k : 0;
+                const int kb = p.map_grouped[mb] ? ge.k : 0;
                 if (!bounded_wait(smem_u32(&bar_empty[s]), ph ^ 1u, wc, 1u, w.unit)) { ok = false; break; }
                 const uint32_t full_local = smem_u32(&bar_full[s]);
                 if (rank == 0) mbar_arrive_expect_tx(full_local, 2 * OBJ_STAGE_BYTES);   // both CTAs' bytes
@@ -129,10 +195,10 @@ objective_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
                 const uint32_t sb = sa + OBJ_A_BYTES;
 #pragma unroll
                 for (int q = 0; q < CTA_ROWS / BOX_FEATURES; ++q)
-                    tma_load_3d_pair(sa + q * BOX_BYTES, amap, full, a0 + q * BOX_FEATURES, r * TILE_K, ka);
+                    tma_load_3d_pair(sa + q * BOX_BYTES, amap, full, ge.a0 + q * BOX_FEATURES, row, ka);
 #pragma unroll
                 for (int q = 0; q < CTA_ROWS / BOX_FEATURES; ++q)
-                    tma_load_3d_pair(sb + q * BOX_BYTES, bmap, full, b0 + q * BOX_FEATURES, r * TILE_K, kb);
+                    tma_load_3d_pair(sb + q * BOX_BYTES, bmap, full, ge.b0 + q * BOX_FEATURES, row, kb);
                 ++issued;
                 if (++s == OBJ_STAGES) { s = 0; ph ^= 1u; }
             }
@@ -155,10 +221,12 @@ objective_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
         bool ok = true;
         WorkItem w;
         for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
+            ItemGeom ge;
+            if (!item_geom<MODE>(p, w, rank, ge)) continue;
             if (!bounded_wait_hot(smem_u32(&bar_acc_empty[buf]), acc_ph ^ 1u, wc, 2u, w.unit)) { ok = false; break; }
             tc_fence_after_sync();
             const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * TILE_N);
-            for (int ks = w.ks0; ks < w.ks1; ++ks) {
+            for (int ks = ge.ks0; ks < ge.ks1; ++ks) {
                 if (!bounded_wait_hot(smem_u32(&bar_full[s]), ph, wc, 3u, w.unit)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t sa = ring + s * OBJ_STAGE_BYTES;
@@ -167,7 +235,7 @@ objective_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
                 for (int kk = 0; kk < TILE_K / 16; ++kk) {
                     const uint64_t adesc = umma_smem_desc_mn_sw128(sa + kk * 16 * 128, BOX_BYTES, 1024);
                     const uint64_t bdesc = umma_smem_desc_mn_sw128(sb + kk * 16 * 128, BOX_BYTES, 1024);
-                    umma_bf16(d_tmem, adesc, bdesc, idesc, (ks != w.ks0 || kk != 0) ? 1u : 0u);
+                    umma_bf16(d_tmem, adesc, bdesc, idesc, (ks != ge.ks0 || kk != 0) ? 1u : 0u);
                 }
                 umma_commit_pair(smem_u32(&bar_empty[s]));   // stage reusable in both CTAs once these MMAs have read it
                 if (++s == OBJ_STAGES) { s = 0; ph ^= 1u; }
@@ -191,30 +259,30 @@ objective_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
         bool ok = true;
         WorkItem w;
         for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
-            int ti, tj;
-            tile_of_slot_blocked(w.unit / p.g, p.nj, p.raster, ti, tj);
-            const int k = w.unit % p.g;
+            ItemGeom ge;
+            if (!item_geom<MODE>(p, w, rank, ge)) continue;
             ok = bounded_wait(smem_u32(&bar_acc_full[buf]), acc_ph, wc, 4u, w.unit);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after_sync();
-            const int row0 = ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + q * 32;
-            const int row = row0 + lane;
-            const bool row_ok = row < p.d;
-            const float *hrow = p.H + (static_cast<size_t>(k) * p.d + (row_ok ? row : 0)) * static_cast<size_t>(p.d);
-            double dsum = 0.0;
+            if (MODE == MODE_OBJECTIVE) {
+                const int ti = ge.ti, tj = ge.tj, k = ge.k;
+                const int row0 = ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + q * 32;
+                const int row = row0 + lane;
+                const bool row_ok = row < p.d;
+                const float *hrow = p.H + (static_cast<size_t>(k) * p.d + (row_ok ? row : 0)) * static_cast<size_t>(p.d);
+                double dsum = 0.0;
 #pragma unroll 1
-            for (int cc = 0; cc < TILE_N / 32; ++cc) {
-                const int col0 = tj * TILE_N + cc * 32;
-                if (col0 >= p.d) break;                    // right of the matrix
-                if (col0 + 32 <= row0) continue;           // 32 x 32 block strictly below the diagonal
-                if (row0 >= p.d) break;                    // below the matrix
-                uint32_t r[32];
-                tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
-                                  static_cast<uint32_t>(buf * TILE_N + cc * 32), r);
-                tmem_ld_wait();
-                if (!row_ok) continue;
-                {
+                for (int cc = 0; cc < TILE_N / 32; ++cc) {
+                    const int col0 = tj * TILE_N + cc * 32;
+                    if (col0 >= p.d) break;                    // right of the matrix
+                    if (col0 + 32 <= row0) continue;           // 32 x 32 block strictly below the diagonal
+                    if (row0 >= p.d) break;                    // below the matrix
+                    uint32_t r[32];
+                    tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
+                                      static_cast<uint32_t>(buf * TILE_N + cc * 32), r);
+                    tmem_ld_wait();
+                    if (!row_ok) continue;
                     float part = 0.0f;
 #pragma unroll
                     for (int v = 0; v < 8; ++v) {
@@ -231,16 +299,39 @@ objective_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
                     }
                     dsum += static_cast<double>(part);
                 }
-            }
-            // This warp has read all it needs from the accumulator: tell the MMA issuer (first CTA).
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_acc_empty[buf]), 0));
-            {
+                // This warp has read all it needs from the accumulator: tell the MMA issuer (first CTA).
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_acc_empty[buf]), 0));
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, off);
                 if (lane == 0)
                     p.partials[static_cast<size_t>(w.unit) * PARTIALS_PER_UNIT + rank * 4 + q] = dsum;
+            } else {
+                const int rl = static_cast<int>(rank) * CTA_ROWS + q * 32 + lane;      // row inside the block
+                const bool row_ok = p.s0 + rl < p.d;
+                const int ch_end = (ge.k + 1) * p.mk;                                  // channels of this group only
+                float *prow = p.P + static_cast<size_t>(rl) * p.d_out;
+#pragma unroll 1
+                for (int cc = 0; cc < TILE_N / 32; ++cc) {
+                    const int ch0 = ge.k * p.mk + ge.tj * TILE_N + cc * 32;
+                    if (ch0 >= ch_end) break;
+                    if (p.s0 + static_cast<int>(rank) * CTA_ROWS + q * 32 >= p.d) break;
+                    uint32_t r[32];
+                    tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
+                                      static_cast<uint32_t>(buf * TILE_N + cc * 32), r);
+                    tmem_ld_wait();
+                    if (!row_ok) continue;
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        if (ch0 + v * 4 < ch_end)
+                            red_add_f32x4(prow + ch0 + v * 4, __uint_as_float(r[v * 4 + 0]), __uint_as_float(r[v * 4 + 1]),
+                                          __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
+                    }
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_acc_empty[buf]), 0));
             }
             buf ^= 1;
             if (buf == 0) acc_ph ^= 1u;
