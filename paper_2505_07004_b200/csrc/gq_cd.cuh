@@ -132,9 +132,9 @@ struct CdBlockParams {
 // them owns the rows 32 t + 4 l + e (t < 8, e < 4) of the running sums
 //     Bu[r] = sum_{c != r} H[r][c] * E_c      (current E: this cycle's values for c < r, last cycle's for c > r).
 // Pass 1 adds the in-block part of last cycle's values (c > r), pass 2 walks the rows in order: the owner of
-// row i rounds W_i - Bu[i] / H_ii to the channel's codebook (ties to the smaller index), the new E_i goes
-// to its seven neighbours by shuffle and every thread adds H[i][r] * E_i to its rows r > i.  Both loops are
-// fully unrolled so that Bu stays in registers.  H[i][.] rows come through shared memory in chunks of 32.
+// row i hands W_i - Bu[i] / H_ii to its seven neighbours, the eight of them find the nearest codebook level
+// (ties to the smaller index), and every thread adds H[i][r] * E_i to its rows r > i.  H[i][.] rows come
+// through shared memory in chunks of 32.
 __global__ void __launch_bounds__(CD_THREADS, 1)
 cd_block_kernel(const CdBlockParams p)
 {
@@ -165,24 +165,32 @@ cd_block_kernel(const CdBlockParams p)
     for (int r = tid; r < CD_BLOCK; r += CD_THREADS)
         rds[r] = r < p.rows ? p.rdiag[static_cast<size_t>(k) * p.d_in + p.s0 + r] : 0.0f;
 
-    // rows [c0, c0 + CD_HCHUNK) of the block's H (columns of the block only) into buffer b; zero outside
+    // rows [c0, c0 + CD_HCHUNK) of the block's H (columns of the block only) into buffer b, zero outside the
+    // block; asynchronous copies (cp.async), completed by h_chunk_wait() before the next __syncthreads
     auto load_h_chunk = [&](int c0, int b) {
         float *dst = Hs + b * CD_HCHUNK * CD_BLOCK;
         for (int idx = tid; idx < CD_HCHUNK * CD_BLOCK / 4; idx += CD_THREADS) {
             const int rr = idx / (CD_BLOCK / 4), cc = (idx % (CD_BLOCK / 4)) * 4;
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (c0 + rr < p.rows && cc < p.rows)      // rows is a multiple of 8 (d_in % 8 == 0): whole float4 in range
-                v = *reinterpret_cast<const float4 *>(Hk + static_cast<size_t>(p.s0 + c0 + rr) * p.d_in + p.s0 + cc);
-            *reinterpret_cast<float4 *>(dst + rr * CD_BLOCK + cc) = v;
+            float *d = dst + rr * CD_BLOCK + cc;
+            if (c0 + rr < p.rows && cc < p.rows) {    // rows is a multiple of 8 (d_in % 8 == 0): whole float4 in range
+                const float *src = Hk + static_cast<size_t>(p.s0 + c0 + rr) * p.d_in + p.s0 + cc;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(
+                                 __cvta_generic_to_shared(d))), "l"(src) : "memory");
+            } else {
+                *reinterpret_cast<float4 *>(d) = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
         }
+        asm volatile("cp.async.commit_group;" ::: "memory");
     };
+    auto h_chunk_wait = [&]() { asm volatile("cp.async.wait_group 0;" ::: "memory"); };
 
-    float cb[CD_MAX_LEVELS];
-#pragma unroll
-    for (int q = 0; q < CD_MAX_LEVELS; ++q)
-        cb[q] = (q < p.m && cidx < ch_n) ? p.codebook[static_cast<size_t>(ch0 + cidx) * p.m + q] : 0.0f;
+    // codebook levels l and l + 8 of this thread's channel (the eight threads of a channel hold all sixteen)
+    static_assert(CD_MAX_LEVELS == 2 * CD_LANES, "two codebook levels per thread");
+    const float cb0 = (l < p.m && cidx < ch_n) ? p.codebook[static_cast<size_t>(ch0 + cidx) * p.m + l] : 0.0f;
+    const float cb1 = (l + 8 < p.m && cidx < ch_n) ? p.codebook[static_cast<size_t>(ch0 + cidx) * p.m + l + 8] : 0.0f;
 
     load_h_chunk(0, 0);
+    h_chunk_wait();
     __syncthreads();
 
     float Bu[8][4];
@@ -192,11 +200,13 @@ cd_block_kernel(const CdBlockParams p)
         for (int e = 0; e < 4; ++e) Bu[t][e] = Xs[(32 * t + 4 * l + e) * CD_TILE_LD + cidx];
 
     // ---- pass 1: Bu[r] += sum_{c in block, c > r} H[c][r] * E_old[c]
+    // (The 32-row bands t are unrolled so that Bu is indexed statically; the rows inside a band are a real
+    // loop - unrolling all 256 steps makes the code larger than the instruction cache and ten times slower.)
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
         if (t + 1 < 8) load_h_chunk((t + 1) * CD_HCHUNK, (t + 1) & 1);
         const float *hc = Hs + (t & 1) * CD_HCHUNK * CD_BLOCK;
-#pragma unroll
+#pragma unroll 1
         for (int ii = 0; ii < 32; ++ii) {
             const float ec = Es[(32 * t + ii) * CD_TILE_LD + cidx];
 #pragma unroll
@@ -215,38 +225,45 @@ cd_block_kernel(const CdBlockParams p)
                 }
             }
         }
+        h_chunk_wait();
         __syncthreads();
     }
 
     // ---- pass 2: the coordinates in order
     load_h_chunk(0, 0);
+    h_chunk_wait();
     __syncthreads();
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
         if (t + 1 < 8) load_h_chunk((t + 1) * CD_HCHUNK, (t + 1) & 1);
         const float *hc = Hs + (t & 1) * CD_HCHUNK * CD_BLOCK;
-#pragma unroll
+#pragma unroll 1
         for (int ii = 0; ii < 32; ++ii) {
             const int i = 32 * t + ii;
-            float e_new = 0.0f;
-            if (l == ii / 4) {                            // the owner of row i rounds it
-                const float target = Ws[i * CD_TILE_LD + cidx] - rds[i] * Bu[t][ii % 4];
-                int best = 0;
-                float bd = fabsf(target - cb[0]);
+            const int owner = ii >> 2, oe = ii & 3;
+            // the owner of row i forms the rounding target; all eight threads of the channel find the nearest
+            // codebook level together (two levels each, then a three-step minimum; ties: the smaller index)
+            const float bu = oe == 0 ? Bu[t][0] : (oe == 1 ? Bu[t][1] : (oe == 2 ? Bu[t][2] : Bu[t][3]));
+            const float w = Ws[i * CD_TILE_LD + cidx];
+            const float target = __shfl_sync(0xffffffffu, w - rds[i] * bu, owner, CD_LANES);
+            const float d0 = l < p.m ? fabsf(target - cb0) : 3.0e38f;
+            const float d1 = l + 8 < p.m ? fabsf(target - cb1) : 3.0e38f;
+            float bd = d1 < d0 ? d1 : d0;                 // equal distances keep the smaller index l
+            int best = d1 < d0 ? l + 8 : l;
+            float val = d1 < d0 ? cb1 : cb0;
 #pragma unroll
-                for (int q = 1; q < CD_MAX_LEVELS; ++q) {
-                    const float dq = fabsf(target - cb[q]);
-                    if (q < p.m && dq < bd) { bd = dq; best = q; }
-                }
-                float val = cb[0];
-#pragma unroll
-                for (int q = 1; q < CD_MAX_LEVELS; ++q) val = (best == q) ? cb[q] : val;
-                e_new = val - Ws[i * CD_TILE_LD + cidx];
+            for (int off = 1; off < CD_LANES; off <<= 1) {
+                const float od = __shfl_xor_sync(0xffffffffu, bd, off, CD_LANES);
+                const int ob = __shfl_xor_sync(0xffffffffu, best, off, CD_LANES);
+                const float ov = __shfl_xor_sync(0xffffffffu, val, off, CD_LANES);
+                if (od < bd || (od == bd && ob < best)) { bd = od; best = ob; val = ov; }
+            }
+            const float e_new = val - w;
+            if (l == owner) {
                 Es[i * CD_TILE_LD + cidx] = e_new;
                 Xs[i * CD_TILE_LD + cidx] = val;
                 Qs[i * CD_CH + cidx] = static_cast<uint8_t>(best);
             }
-            e_new = __shfl_sync(0xffffffffu, e_new, ii / 4, CD_LANES);
 #pragma unroll
             for (int tp = t; tp < 8; ++tp) {
                 const float4 h = *reinterpret_cast<const float4 *>(hc + ii * CD_BLOCK + 32 * tp + 4 * l);
@@ -263,6 +280,7 @@ cd_block_kernel(const CdBlockParams p)
                 }
             }
         }
+        h_chunk_wait();
         __syncthreads();
     }
 
