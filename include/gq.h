@@ -224,6 +224,14 @@ size_t gq_cd_workspace_bytes(int64_t d_in, int64_t d_out, int32_t g);
  */
 int32_t gq_check(void *stream, uint32_t *detail /* HOST, may be NULL */);
 
+/*
+ * Self-test of the device-side failure detection (no counterpart in the paper): launches a one-warp kernel
+ * that waits, with the pipeline kernels' own bounded wait, on a barrier nothing ever signals.  After
+ * `budget_ms` (1 .. 1000) the wait gives up, the kernel returns normally and the next gq_check() reports
+ * GQ_ERR_TIMEOUT with site id 99; the CUDA context stays usable.  Nothing is trapped, faulted or hung.
+ */
+int32_t gq_selftest_wait_timeout(int32_t budget_ms, void *stream);
+
 /* Number of kernels this library has launched from the calling process (for bookkeeping). */
 uint64_t gq_launch_count(void);
 

@@ -23,6 +23,7 @@ EXPORTS = (
     "gq_hessian_workspace_bytes", "gq_hessian_finalize", "gq_objective", "gq_objective_workspace_bytes",
     "gq_layer_objective_host", "gq_layer_host_arena_bytes", "gq_check", "gq_launch_count",
     "gq_kernel_timing_enable", "gq_kernel_timing_read", "gq_objective_noalloc", "gq_cd_cycles", "gq_cd_workspace_bytes",
+    "gq_selftest_wait_timeout",
 )
 GQ_HESSIAN_DETERMINISTIC = 1      # flag of gq_hessian_accumulate: single writer per element of H
 KERNEL_NAMES = ("saliency", "hessian", "mirror", "split_delta", "gram_dot", "reduce", "split_saliency", "cd_panel",
@@ -79,6 +80,8 @@ def lib() -> ctypes.CDLL:
         L.gq_cd_workspace_bytes.argtypes = [i64, i64, i32]
         L.gq_cd_cycles.restype = i32
         L.gq_cd_cycles.argtypes = [vp, vp, vp, vp, i32, i64, i64, vp, i32, i32, vp, sz, vp]
+        L.gq_selftest_wait_timeout.restype = i32
+        L.gq_selftest_wait_timeout.argtypes = [i32, vp]
         L.gq_kernel_timing_enable.restype = i32
         L.gq_kernel_timing_enable.argtypes = [i32]
         L.gq_kernel_timing_read.restype = i32
@@ -314,3 +317,11 @@ def gq_cd_cycles(W: torch.Tensor, W_hat: torch.Tensor, codebook: torch.Tensor, H
     if rc:
         raise GQError("gq_cd_cycles", rc)
     return W_hat, Q
+
+
+def gq_selftest_wait_timeout(budget_ms: int = 20, stream=None) -> None:
+    """Launches the kernel whose wait runs out after ``budget_ms``; the next :func:`gq_check` raises
+    ``GQ_ERR_TIMEOUT`` (site 99)."""
+    rc = lib().gq_selftest_wait_timeout(int(budget_ms), _stream_ptr(stream))
+    if rc:
+        raise GQError("gq_selftest_wait_timeout", rc)

@@ -19,7 +19,10 @@
 //              (M = 256, N = 256, K = 16) with fp32 accumulation in tensor memory
 //   epilogue   eight warps per CTA move the accumulators to H: tcgen05.ld -> swizzled staging block in
 //              shared memory -> TMA reduce-add (cp.reduce.async.bulk.tensor ... .add) of 32 x 32 fp32
-//              blocks, so H is never read by the SMs and every access to it is a full 128-byte row segment
+//              blocks, so H is never read by the SMs and every access to it is a full 128-byte row segment.
+//              When a unit is short (few k-steps, i.e. small token chunks) the time the tensor core waits
+//              for this read-out matters more than the access pattern, and the warps add their registers
+//              to H directly with red.global.add.v4.f32 instead (no staging, nothing to wait for)
 //
 // Per CTA and k-step (1024 tensor-core clocks for two groups) this moves 32 KB from L2 (half of what a
 // per-group pass over pre-scaled operands needs) and 112 KB through shared memory.
@@ -60,6 +63,9 @@ constexpr int HS_SMEM_BYTES = HS_STAGES * HS_STAGE_BYTES + HS_STAGING_BYTES + 10
 struct HessianParams {
     const __nv_bfloat16 *X;  // [n][ld_x]
     long long ld_x;
+    float *H;                // [g][d][d] (used by the register epilogue; the TMA epilogue goes through mapH)
+    int direct_epilogue;     // 1: accumulators are added to H straight from registers (red.global.add.v4.f32);
+                             // 0: through a shared-memory staging block and TMA reduce-add
     const uint2 *s2;         // [ceil(g / 2)][n]: split saliency of groups (2 q, 2 q + 1), see split_saliency_kernel
     int n;                   // tokens in this call
     int d;                   // d_in
@@ -422,6 +428,20 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                     tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                       static_cast<uint32_t>(kk * TILE_N + cc * 32), r);
                     tmem_ld_wait();
+                    if (p.direct_epilogue) {
+                        // short units: straight from registers, nothing to wait for (each lane adds eight
+                        // 16-byte pieces of its own row)
+                        const int row = row0 + lane;
+                        if (row < p.d) {
+                            float *hrow = p.H + (static_cast<size_t>(u.grp[kk]) * p.d + row) * static_cast<size_t>(p.d) + col0;
+#pragma unroll
+                            for (int v = 0; v < 8; ++v)
+                                if (col0 + v * 4 < p.d)
+                                    red_add_f32x4(hrow + v * 4, __uint_as_float(r[v * 4 + 0]), __uint_as_float(r[v * 4 + 1]),
+                                                  __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
+                        }
+                        continue;
+                    }
 #pragma unroll
                     for (int v = 0; v < 8; ++v)
                         st_shared_16(stg + static_cast<uint32_t>(lane * 128 + ((v ^ (lane & 7)) << 4)),

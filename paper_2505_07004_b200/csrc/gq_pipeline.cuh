@@ -204,6 +204,25 @@ __device__ __forceinline__ bool bounded_wait_hot(uint32_t bar, uint32_t parity, 
     }
 }
 
+// Self-test of the bounded waits: one thread waits, with the kernels' own wait routine, on a barrier that
+// nothing will ever signal.  The wait gives up after `budget_ns`, records STATUS_TIMEOUT (site 99) in the
+// status word and the kernel returns normally - the context stays usable.
+__global__ void wait_selftest_kernel(uint32_t *status, unsigned long long budget_ns)
+{
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ volatile uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0u;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const WaitCtx wc{&abort_flag, status, budget_ns};
+        (void)bounded_wait(smem_u32(&bar), 0u, wc, 99u, 0u);
+    }
+}
+
 __device__ __forceinline__ void spin_ns(unsigned long long ns)
 {
     const uint64_t t0 = global_timer_ns();

@@ -337,6 +337,35 @@ def test_full_shapes_sampled(dev, name, g, n_tokens, s_chunks):
     torch.cuda.empty_cache()
 
 
+# ------------------------------------------------------------------------------------------ failure detection
+def test_device_wait_timeout_is_reported_and_context_survives(dev):
+    """A pipeline wait that runs out of its time budget makes the kernel return (no trap, no hang), the status
+    word reports it once, and the library keeps working afterwards."""
+    libgq.gq_check()
+    libgq.gq_selftest_wait_timeout(20)
+    with pytest.raises(libgq.GQError) as e:
+        libgq.gq_check()
+    assert "GQ_ERR_TIMEOUT" in str(e.value)
+    assert e.value.detail[1] == 99                        # the site id of the self-test wait
+    libgq.gq_check()                                      # reported once, then clear
+    grad = torch.ones((8, 16), dtype=torch.bfloat16, device=dev)
+    s = libgq.gq_saliency(grad, 2)
+    libgq.gq_check()
+    assert torch.allclose(s, torch.ones_like(s))
+
+
+def test_hessian_padded_rows_and_saliency_stride(dev):
+    """ld_x > d_in and ld_s > n: views into wider buffers."""
+    n, d_in, g = 200, 264, 3
+    gen = torch.Generator(device=dev).manual_seed(9)
+    Xw = torch.randn(n, d_in + 40, generator=gen, device=dev).to(torch.bfloat16)
+    sw = torch.rand(g, n + 24, generator=gen, device=dev)
+    X, s = Xw[:, :d_in], sw[:, :n]
+    H = gpu_hessian([X], [s], d_in, g, dev)
+    H_ref = orc.hessian(synth.bf16_bits(X.contiguous()), s.contiguous().cpu().numpy().astype(np.float64))
+    check_H(H, H_ref)
+
+
 # ------------------------------------------------------------------------------------------ host path
 def test_host_pipeline_matches_device_calls(dev):
     cfg = synth.LayerConfig("host", 700, 256, 384, 256, (2,), "lognormal", 0.01, 20.0)
