@@ -147,3 +147,43 @@ def cd_naive(W, W_hat0, codebook, H, cycles: int = 1):
                 What[j, i] = cbk[j, best_q]
                 Q[j, i] = best_q
     return What.astype(np.float32), Q
+
+
+# --------------------------------------------------------------------------------------------------------
+# Codebook step and the LNQ loop (Section 4.2, Eq. 8; Algorithm 2)
+
+def one_hot(q_j: np.ndarray, m: int) -> np.ndarray:
+    """Assignment matrix P^(j) in {0,1}^{d_in x m} of one channel from its codes."""
+    P = np.zeros((q_j.shape[0], m), dtype=np.float64)
+    P[np.arange(q_j.shape[0]), q_j] = 1.0
+    return P
+
+
+def codebook_update(W, Q, H, m: int, lam: float = 1e-7) -> np.ndarray:
+    """Eq. 8 for every channel: c^(j) = (P^T H_k P + lam I)^-1 P^T H_k w_j, with the small constant lam on the
+    diagonal that the text below Eq. 8 prescribes (1e-7 in the paper).  Returns fp64 [d_out, m]."""
+    W = np.asarray(W, dtype=np.float64)
+    H = np.asarray(H, dtype=np.float64)
+    d_out, d_in = W.shape
+    mk = d_out // H.shape[0]
+    C = np.zeros((d_out, m), dtype=np.float64)
+    for j in range(d_out):
+        Hk = H[j // mk]
+        P = one_hot(np.asarray(Q[j]), m)
+        G = P.T @ Hk @ P + lam * np.eye(m)
+        r = P.T @ (Hk @ W[j])
+        C[j] = np.linalg.solve(G, r)
+    return C
+
+
+def lnq(W, Q0, H, m: int, T: int, K: int, lam: float = 1e-7, b: int = 128):
+    """Algorithm 2: T rounds of (codebook step, K CD cycles), then a final codebook step.
+    Returns (W_hat fp32 [d_out, d_in], Q int32, codebook fp32 [d_out, m])."""
+    W32 = np.ascontiguousarray(W, dtype=np.float32)
+    Q = np.asarray(Q0, dtype=np.int32).copy()
+    for _ in range(T):
+        cbk = codebook_update(W32, Q, H, m, lam).astype(np.float32)
+        What = np.take_along_axis(cbk, Q, axis=1)
+        What, Q = cd(W32, What, cbk, H, K, b)
+    cbk = codebook_update(W32, Q, H, m, lam).astype(np.float32)
+    return np.take_along_axis(cbk, Q, axis=1), Q, cbk

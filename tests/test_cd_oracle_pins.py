@@ -93,3 +93,62 @@ def test_ties_and_dead_features():
     What, Q = cdo.cd(W, np.zeros((1, 3), np.float32), cb, H, 1, 128)
     assert Q.tolist() == [[0, 1, 1]]          # exact ties go to the smaller index; dead feature: nearest to W
     assert What.tolist() == [[0.0, 1.0, 1.0]]
+
+
+# ------------------------------------------------------------------------------------------ codebook step
+def test_codebook_step_is_the_least_squares_solution():
+    """Eq. 8 against the formulation the paper gives to its solver: min_c || L^T (P c - w) ||_2 with
+    H = L L^T (library least squares), against the diagonal closed form, and against perturbations."""
+    from scipy.linalg import cholesky, lstsq
+    W, W0, cb, H = make_problem(9, 40, 6, 2, 4, n=200)
+    _, Q = cdo.round_to_codebook(W, cb)
+    C = cdo.codebook_update(W, Q, H, 4, lam=0.0)
+    mk = 3
+    for j in range(6):
+        Hk = H[j // mk].astype(np.float64)
+        L = cholesky(Hk, lower=True)
+        P = cdo.one_hot(Q[j], 4)
+        ref, *_ = lstsq(L.T @ P, L.T @ W[j].astype(np.float64))
+        assert np.allclose(C[j], ref, rtol=1e-7, atol=1e-10)
+        f_opt = cdo.channel_objective(P @ C[j] - W[j], Hk)
+        rng = np.random.default_rng(j)
+        for _ in range(5):                                   # no perturbed codebook does better
+            f = cdo.channel_objective(P @ (C[j] + 1e-3 * rng.standard_normal(4)) - W[j], Hk)
+            assert f >= f_opt
+        assert f_opt <= cdo.channel_objective(P @ cb[j].astype(np.float64) - W[j], Hk) * (1 + 1e-12)
+    # diagonal H: every level becomes the H_ii-weighted mean of the weights assigned to it
+    h = np.random.default_rng(1).random(40) + 0.1
+    Cd = cdo.codebook_update(W, Q, np.stack([np.diag(h)] * 2), 4, lam=0.0)
+    for j in range(6):
+        for q in range(4):
+            sel = Q[j] == q
+            if sel.any():
+                assert np.isclose(Cd[j, q], (h[sel] * W[j, sel]).sum() / h[sel].sum(), rtol=1e-10)
+    # a level nobody uses: lam keeps the system solvable and gives that level the value 0
+    Q1 = Q.copy()
+    Q1[Q1 == 3] = 2
+    C1 = cdo.codebook_update(W, Q1, H, 4, lam=1e-7)
+    assert np.all(C1[:, 3] == 0.0) and np.all(np.isfinite(C1))
+
+
+def test_lnq_descends():
+    """Proposition 1: the objective of every channel is non-increasing over the LNQ iterations."""
+    W, W0, cb, H = make_problem(10, 48, 8, 2, 4, n=200)
+    _, Q0 = cdo.round_to_codebook(W, cb)
+    mk = 4
+
+    def per_channel(What):
+        return np.array([cdo.channel_objective(What[j].astype(np.float64) - W[j], H[j // mk].astype(np.float64))
+                         for j in range(8)])
+
+    f_prev = per_channel(W0)
+    Q = Q0
+    for t in range(3):
+        c = cdo.codebook_update(W, Q, H, 4).astype(np.float32)
+        f_c = per_channel(np.take_along_axis(c, Q, axis=1))
+        assert np.all(f_c <= f_prev * (1 + 1e-5))            # codebook step (fp32 codebook: 1e-5 slack)
+        What, Q = cdo.cd(W, np.take_along_axis(c, Q, axis=1), c, H, 2, 16)
+        f_prev = per_channel(What)
+        assert np.all(f_prev <= f_c * (1 + 1e-12))           # CD
+    What, Qf, cf = cdo.lnq(W, Q0, H, 4, T=3, K=2, b=16)
+    assert np.all(per_channel(What) <= f_prev * (1 + 1e-5))
