@@ -225,6 +225,34 @@ size_t gq_cd_workspace_bytes(int64_t d_in, int64_t d_out, int32_t g);
 int32_t gq_check(void *stream, uint32_t *detail /* HOST, may be NULL */);
 
 /*
+ * Codebook step of the layer-wise quantiser (Section 4.2, Eq. 8; Algorithm 2 lines 4 and 14): with the
+ * assignment matrix P^(j) in {0,1}^{d_in x m} given by the codes of channel j (P_iq = 1 iff Q[j][i] == q),
+ *     codebook[j] = (P^T H_k P + lambda I)^-1 P^T H_k w_j          for every channel j of every group k,
+ * the minimiser of channel j's objective over its m codebook values for fixed codes (lambda is the small
+ * constant the paper adds to the diagonal, 1e-7 there; a level that no coordinate uses gets the value 0).
+ *
+ *   W          fp32 [d_out, d_in], 16-byte aligned
+ *   Q          uint8 [d_out, d_in], codes < m (larger values are read as m - 1)
+ *   m          1 <= m <= 16
+ *   H          fp32 [g, d_in, d_in], FULL symmetric matrices (after gq_hessian_finalize), 16-byte aligned
+ *   lambda     >= 0
+ *   codebook   fp32 [d_out, m], out
+ *   W_hat      fp32 [d_out, d_in] or NULL; out: W_hat[j][i] = codebook[j][Q[j][i]]
+ *   workspace  device scratch of at least gq_codebook_workspace_bytes(d_in, d_out, g, m) bytes, 1024-byte aligned
+ * Same shape rules as gq_objective.
+ * Arithmetic: H_k W_k^T and H_k [P^(j) ...] are formed on the tensor cores with H as three bf16 terms that
+ * sum to the fp32 value exactly (the one-hot columns are exact, W is carried to 24 bits as well), fp32
+ * accumulation; the sums over the rows of each level and the m x m Cholesky solves are fp64.
+ * Together with gq_cd_cycles and gq_objective this is Algorithm 2: repeat { gq_codebook_update (with W_hat);
+ * gq_cd_cycles } T times, then gq_codebook_update once more.
+ */
+int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t d_in, int64_t d_out,
+                           const float *H, int32_t g, double lambda, float *codebook, float *W_hat,
+                           void *workspace, size_t workspace_bytes, void *stream);
+
+size_t gq_codebook_workspace_bytes(int64_t d_in, int64_t d_out, int32_t g, int32_t m);
+
+/*
  * Self-test of the device-side failure detection (no counterpart in the paper): launches a one-warp kernel
  * that waits, with the pipeline kernels' own bounded wait, on a barrier nothing ever signals.  After
  * `budget_ms` (1 .. 1000) the wait gives up, the kernel returns normally and the next gq_check() reports
@@ -249,7 +277,10 @@ enum gq_kernel_id {
     GQ_KERNEL_CD_PANEL = 7,    /* coordinate descent: tensor-core product with the coordinates outside a block */
     GQ_KERNEL_CD_BLOCK = 8,    /* coordinate descent: the 256 coordinates of a block, in order */
     GQ_KERNEL_CD_AUX = 9,      /* coordinate descent: transposes and bf16 splits */
-    GQ_KERNEL_COUNT = 10
+    GQ_KERNEL_CB_GEMM = 10,    /* codebook step: tensor-core products H W^T and H [P ...] */
+    GQ_KERNEL_CB_FOLD = 11,    /* codebook step: sums over the rows of each level, m x m solves */
+    GQ_KERNEL_CB_AUX = 12,     /* codebook step: splits, transposes, one-hot columns, W_hat */
+    GQ_KERNEL_COUNT = 13
 };
 
 /*

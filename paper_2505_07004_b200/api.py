@@ -23,11 +23,11 @@ EXPORTS = (
     "gq_hessian_workspace_bytes", "gq_hessian_finalize", "gq_objective", "gq_objective_workspace_bytes",
     "gq_layer_objective_host", "gq_layer_host_arena_bytes", "gq_check", "gq_launch_count",
     "gq_kernel_timing_enable", "gq_kernel_timing_read", "gq_objective_noalloc", "gq_cd_cycles", "gq_cd_workspace_bytes",
-    "gq_selftest_wait_timeout",
+    "gq_selftest_wait_timeout", "gq_codebook_update", "gq_codebook_workspace_bytes",
 )
 GQ_HESSIAN_DETERMINISTIC = 1      # flag of gq_hessian_accumulate: single writer per element of H
 KERNEL_NAMES = ("saliency", "hessian", "mirror", "split_delta", "gram_dot", "reduce", "split_saliency", "cd_panel",
-                "cd_block", "cd_aux")
+                "cd_block", "cd_aux", "cb_gemm", "cb_fold", "cb_aux")
 
 
 class GQError(RuntimeError):
@@ -80,6 +80,10 @@ def lib() -> ctypes.CDLL:
         L.gq_cd_workspace_bytes.argtypes = [i64, i64, i32]
         L.gq_cd_cycles.restype = i32
         L.gq_cd_cycles.argtypes = [vp, vp, vp, vp, i32, i64, i64, vp, i32, i32, vp, sz, vp]
+        L.gq_codebook_workspace_bytes.restype = sz
+        L.gq_codebook_workspace_bytes.argtypes = [i64, i64, i32, i32]
+        L.gq_codebook_update.restype = i32
+        L.gq_codebook_update.argtypes = [vp, vp, i32, i64, i64, vp, i32, ctypes.c_double, vp, vp, vp, sz, vp]
         L.gq_selftest_wait_timeout.restype = i32
         L.gq_selftest_wait_timeout.argtypes = [i32, vp]
         L.gq_kernel_timing_enable.restype = i32
@@ -325,3 +329,36 @@ def gq_selftest_wait_timeout(budget_ms: int = 20, stream=None) -> None:
     rc = lib().gq_selftest_wait_timeout(int(budget_ms), _stream_ptr(stream))
     if rc:
         raise GQError("gq_selftest_wait_timeout", rc)
+
+
+def gq_codebook_workspace_bytes(d_in: int, d_out: int, g: int, m: int) -> int:
+    return int(lib().gq_codebook_workspace_bytes(d_in, d_out, g, m))
+
+
+def gq_codebook_update(W: torch.Tensor, Q: torch.Tensor, m: int, H: torch.Tensor, workspace: torch.Tensor,
+                       lam: float = 1e-7, codebook: Optional[torch.Tensor] = None,
+                       W_hat: Optional[torch.Tensor] = None, stream=None):
+    """Eq. 8 for every channel: the optimal codebook for fixed codes ``Q``.  Returns ``(codebook, W_hat)``;
+    ``W_hat`` (if a tensor is passed) receives ``codebook[j, Q[j, i]]``."""
+    _dev(W, torch.float32, "W")
+    _dev(Q, torch.uint8, "Q")
+    _dev(H, torch.float32, "H")
+    if W.dim() != 2 or W.shape != Q.shape or not W.is_contiguous() or not Q.is_contiguous():
+        raise ValueError("W and Q must be contiguous [d_out, d_in]")
+    d_out, d_in = W.shape
+    g = H.shape[0]
+    if tuple(H.shape) != (g, d_in, d_in) or not H.is_contiguous():
+        raise ValueError("H must be a contiguous [g, d_in, d_in] tensor")
+    if codebook is None:
+        codebook = torch.empty((d_out, m), dtype=torch.float32, device=W.device)
+    _dev(codebook, torch.float32, "codebook")
+    if W_hat is not None:
+        _dev(W_hat, torch.float32, "W_hat")
+        if W_hat.shape != W.shape or not W_hat.is_contiguous():
+            raise ValueError("W_hat must be contiguous [d_out, d_in]")
+    rc = lib().gq_codebook_update(W.data_ptr(), Q.data_ptr(), int(m), d_in, d_out, H.data_ptr(), g, float(lam),
+                                  codebook.data_ptr(), W_hat.data_ptr() if W_hat is not None else None,
+                                  workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc:
+        raise GQError("gq_codebook_update", rc)
+    return codebook, W_hat

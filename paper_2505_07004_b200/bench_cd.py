@@ -1,8 +1,9 @@
 #!/usr/bin/env python
-"""Times gq_cd_cycles (cyclic coordinate descent with fixed codebooks, Algorithm 4) on a synthetic layer.
+"""Times gq_cd_cycles (cyclic coordinate descent with fixed codebooks, Algorithm 4) and, optionally, the LNQ loop
+(Algorithm 2: gq_codebook_update + gq_cd_cycles) on a synthetic layer.
 
     python -m paper_2505_07004_b200.bench_cd [--d-in 4096] [--d-out 4096] [--g 4] [--levels 16] [--cycles 2]
-                                             [--tokens 8192] [--oracle-channels 0]
+                                             [--tokens 8192] [--oracle-channels 0] [--lnq-rounds 0]
 
 The layer's guided Hessians come from the library's own path (gq_saliency, gq_hessian_accumulate,
 gq_hessian_finalize on seeded synthetic activations and gradients), the codebooks are per-channel grids
@@ -36,6 +37,8 @@ def main():
     ap.add_argument("--cycles", type=int, default=2)
     ap.add_argument("--tokens", type=int, default=8192)
     ap.add_argument("--oracle-channels", type=int, default=0)
+    ap.add_argument("--lnq-rounds", type=int, default=0,
+                    help="also time Algorithm 2: this many rounds of (codebook step, --cycles CD cycles) + a final codebook step")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise RuntimeError("bench_cd needs a CUDA device: libgq has no CPU path")
@@ -81,6 +84,29 @@ def main():
         "kernels_ms": {k: {"ms": round(v[0], 4), "launches": v[1]} for k, v in kern.items() if v[1]},
         "objective_start": f0, "objective_end": f1,
     }
+    if args.lnq_rounds > 0:
+        cbw = libgq.alloc_workspace(libgq.gq_codebook_workspace_bytes(cfg.d_in, cfg.d_out, g, m), dev)
+        Q = (W[:, :, None] - cb[:, None, :]).abs().argmin(-1).to(torch.uint8).contiguous()
+        Wh = W0.clone()
+        cbl, _ = libgq.gq_codebook_update(W, Q, m, H, cbw, W_hat=Wh)      # warm-up
+        libgq.gq_check()
+        Wh = W0.clone()
+        traj = [f0]
+        libgq.gq_kernel_timing_enable(True)
+        e0.record()
+        for _ in range(args.lnq_rounds):
+            cbl, Wh = libgq.gq_codebook_update(W, Q, m, H, cbw, W_hat=Wh)
+            Wh, Q = libgq.gq_cd_cycles(W, Wh, cbl, H, args.cycles, ws, Q=Q)
+        cbl, Wh = libgq.gq_codebook_update(W, Q, m, H, cbw, W_hat=Wh)
+        e1.record()
+        e1.synchronize()
+        kern = libgq.gq_kernel_timing_read()
+        libgq.gq_kernel_timing_enable(False)
+        libgq.gq_check()
+        traj.append(float(libgq.gq_objective(W, Wh, H, ows).cpu()[-1]))
+        out["lnq"] = {"rounds": args.lnq_rounds, "cd_cycles_per_round": args.cycles, "ms_total": e0.elapsed_time(e1),
+                      "kernels_ms": {k: {"ms": round(v[0], 4), "launches": v[1]} for k, v in kern.items() if v[1]},
+                      "objective_start": traj[0], "objective_end": traj[1]}
     if args.oracle_channels > 0:
         from oracle import cd_oracle as cdo
         mk = cfg.d_out // g

@@ -1,0 +1,182 @@
+// Codebook step of the layer-wise quantiser (Section 4.2, Eq. 8; Algorithm 2 lines 4 and 14): for every
+// output channel j of group k, with the assignment matrix P in {0,1}^{d_in x m} given by the codes Q,
+//
+//     c^(j) = (P^T H_k P + lambda I)^-1  P^T H_k w_j .
+//
+// The two d_in^2-sized contractions run on the tensor cores (pair_gemm_kernel<MODE_FULL>):
+//     HW = H_k W_k^T                      [d_in x channels]
+//     HP = H_k [P^(j0) ... P^(j0+c-1)]    [d_in x (channels * m)]   for a slab of channels at a time
+// with H carried as three bf16 matrices whose sum is the fp32 value exactly (8 + 8 + 8 mantissa bits), the
+// one-hot columns exact in bf16 and W as three bf16 terms as well; accumulation is fp32.  The kernels here
+// prepare those operands, fold HP and HW over the rows of each level (fp64),
+//     G^(j)[q][q'] = sum_{i : Q_ij = q} HP[i][j m + q'],      r^(j)[q] = sum_{i : Q_ij = q} HW[i][j],
+// and solve the m x m systems by Cholesky in fp64.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace gq {
+
+constexpr int CB_MAX_LEVELS = 16;
+constexpr int CB_SLAB_CHANNELS = 1024;      // channels whose one-hot columns are multiplied at a time
+
+// v = t0 + t1 + t2 exactly (for finite v in bf16 range): three rounds of "round to bf16, subtract".
+__device__ __forceinline__ void split3_bf16(float v, __nv_bfloat16 &t0, __nv_bfloat16 &t1, __nv_bfloat16 &t2)
+{
+    t0 = __float2bfloat16_rn(v);
+    const float r1 = v - __bfloat162float(t0);
+    t1 = __float2bfloat16_rn(r1);
+    t2 = __float2bfloat16_rn(r1 - __bfloat162float(t1));
+}
+
+__global__ void __launch_bounds__(256)
+cb_split3_kernel(const float *__restrict__ src, long long count, __nv_bfloat16 *__restrict__ d0,
+                 __nv_bfloat16 *__restrict__ d1, __nv_bfloat16 *__restrict__ d2)
+{
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; idx < count; idx += stride) {
+        __nv_bfloat16 a, b, c;
+        split3_bf16(src[idx], a, b, c);
+        d0[idx] = a;
+        d1[idx] = b;
+        d2[idx] = c;
+    }
+}
+
+// W [d_out][d_in] -> three bf16 terms of W^T [d_in][d_out]; Q [d_out][d_in] -> Qt [d_in][d_out].  32 x 32 tiles.
+__global__ void __launch_bounds__(256)
+cb_transpose_kernel(const float *__restrict__ W, const uint8_t *__restrict__ Q, int d_in, int d_out,
+                    __nv_bfloat16 *__restrict__ W0, __nv_bfloat16 *__restrict__ W1, __nv_bfloat16 *__restrict__ W2,
+                    uint8_t *__restrict__ Qt)
+{
+    __shared__ float tw[32][33];
+    __shared__ uint8_t tq[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int i0 = blockIdx.x * 32, j0 = blockIdx.y * 32;
+    for (int r = ty; r < 32; r += 8) {
+        const int j = j0 + r, i = i0 + tx;
+        const bool ok = j < d_out && i < d_in;
+        tw[r][tx] = ok ? W[static_cast<size_t>(j) * d_in + i] : 0.0f;
+        tq[r][tx] = ok ? Q[static_cast<size_t>(j) * d_in + i] : 0;
+    }
+    __syncthreads();
+    for (int r = ty; r < 32; r += 8) {
+        const int i = i0 + r, j = j0 + tx;
+        if (i < d_in && j < d_out) {
+            const size_t o = static_cast<size_t>(i) * d_out + j;
+            __nv_bfloat16 a, b, c;
+            split3_bf16(tw[tx][r], a, b, c);
+            W0[o] = a;
+            W1[o] = b;
+            W2[o] = c;
+            Qt[o] = tq[tx][r];
+        }
+    }
+}
+
+// One-hot columns of channels [j0, j0 + nch): Pm[i][jj * m + q] = (Qt[i][j0 + jj] == q), bf16, row stride ld.
+__global__ void __launch_bounds__(256)
+cb_onehot_kernel(const uint8_t *__restrict__ Qt, int d_in, int d_out, int j0, int nch, int m,
+                 __nv_bfloat16 *__restrict__ Pm, long long ld)
+{
+    const long long cols = static_cast<long long>(nch) * m;
+    const long long total = static_cast<long long>(d_in) * cols;
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total; idx += stride) {
+        const int i = static_cast<int>(idx / cols);
+        const int c = static_cast<int>(idx - static_cast<long long>(i) * cols);
+        const int jj = c / m, q = c - jj * m;
+        const int code = Qt[static_cast<size_t>(i) * d_out + j0 + jj];
+        const bool one = (code < m ? code : m - 1) == q;
+        Pm[static_cast<size_t>(i) * ld + c] = __float2bfloat16_rn(one ? 1.0f : 0.0f);
+    }
+}
+
+// Fold over the rows of each level.  One CTA = 8 channels of the slab x 16 threads; thread (ch, q') owns column
+// q' of G^(ch) in shared memory (fp64), so no two threads ever add to the same word; thread q' = 0 also owns r.
+__global__ void __launch_bounds__(128)
+cb_fold_kernel(const float *__restrict__ HP, long long ld_hp, const float *__restrict__ HW, const uint8_t *__restrict__ Qt,
+               int d_in, int d_out, int j0, int nch, int m, double *__restrict__ G, double *__restrict__ R)
+{
+    __shared__ double Gs[8][CB_MAX_LEVELS][CB_MAX_LEVELS + 1];
+    __shared__ double Rs[8][CB_MAX_LEVELS];
+    const int ch = threadIdx.x >> 4, qp = threadIdx.x & 15;
+    const int jj = blockIdx.x * 8 + ch;
+    for (int q = 0; q < CB_MAX_LEVELS; ++q) Gs[ch][q][qp] = 0.0;
+    Rs[ch][qp] = 0.0;
+    __syncthreads();
+    if (jj < nch && qp < m) {
+        const int j = j0 + jj;
+        const float *hp = HP + static_cast<size_t>(jj) * m + qp;
+        for (int i = 0; i < d_in; ++i) {
+            int q = Qt[static_cast<size_t>(i) * d_out + j];
+            q = q < m ? q : m - 1;                       // codes are expected to be < m
+            Gs[ch][q][qp] += static_cast<double>(hp[static_cast<size_t>(i) * ld_hp]);
+            if (qp == 0) Rs[ch][q] += static_cast<double>(HW[static_cast<size_t>(i) * d_out + j]);
+        }
+    }
+    __syncthreads();
+    if (jj < nch) {
+        const int j = j0 + jj;
+        for (int q = 0; q < CB_MAX_LEVELS; ++q)
+            G[(static_cast<size_t>(j) * CB_MAX_LEVELS + q) * CB_MAX_LEVELS + qp] = (q < m && qp < m) ? Gs[ch][q][qp] : 0.0;
+        R[static_cast<size_t>(j) * CB_MAX_LEVELS + qp] = qp < m ? Rs[ch][qp] : 0.0;
+    }
+}
+
+// (G + lambda I) c = r by Cholesky, one thread per channel, fp64; G is symmetrised first (its two triangles
+// come from different sums).  A pivot that is not positive (possible only through rounding) is replaced by
+// lambda-sized regularisation so that the solve always completes.
+__global__ void __launch_bounds__(128)
+cb_solve_kernel(const double *__restrict__ G, const double *__restrict__ R, int d_out, int m, double lambda,
+                float *__restrict__ codebook)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= d_out) return;
+    double A[CB_MAX_LEVELS][CB_MAX_LEVELS];
+    double b[CB_MAX_LEVELS];
+    const double *g = G + static_cast<size_t>(j) * CB_MAX_LEVELS * CB_MAX_LEVELS;
+    for (int q = 0; q < m; ++q) {
+        for (int p = 0; p <= q; ++p) A[q][p] = 0.5 * (g[q * CB_MAX_LEVELS + p] + g[p * CB_MAX_LEVELS + q]);
+        A[q][q] += lambda;
+        b[q] = R[static_cast<size_t>(j) * CB_MAX_LEVELS + q];
+    }
+    for (int q = 0; q < m; ++q) {                 // A = L L^T, L stored in the lower triangle
+        for (int p = 0; p < q; ++p) {
+            double v = A[q][p];
+            for (int t = 0; t < p; ++t) v -= A[q][t] * A[p][t];
+            A[q][p] = v / A[p][p];
+        }
+        double d = A[q][q];
+        for (int t = 0; t < q; ++t) d -= A[q][t] * A[q][t];
+        if (!(d > 0.0)) d = lambda > 0.0 ? lambda : 1e-300;
+        A[q][q] = sqrt(d);
+    }
+    for (int q = 0; q < m; ++q) {                 // L y = b
+        double v = b[q];
+        for (int t = 0; t < q; ++t) v -= A[q][t] * b[t];
+        b[q] = v / A[q][q];
+    }
+    for (int q = m - 1; q >= 0; --q) {            // L^T c = y
+        double v = b[q];
+        for (int t = q + 1; t < m; ++t) v -= A[t][q] * b[t];
+        b[q] = v / A[q][q];
+    }
+    for (int q = 0; q < m; ++q) codebook[static_cast<size_t>(j) * m + q] = static_cast<float>(b[q]);
+}
+
+// What[j][i] = codebook[j][Q[j][i]]
+__global__ void __launch_bounds__(256)
+cb_apply_kernel(const float *__restrict__ codebook, const uint8_t *__restrict__ Q, long long count, int d_in, int m,
+                float *__restrict__ What)
+{
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; idx < count; idx += stride) {
+        const long long j = idx / d_in;
+        const int q = Q[idx];
+        What[idx] = codebook[j * m + (q < m ? q : m - 1)];
+    }
+}
+
+}  // namespace gq

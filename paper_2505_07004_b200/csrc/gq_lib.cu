@@ -16,6 +16,7 @@
 #include "gq_hessian.cuh"
 #include "gq_objective.cuh"
 #include "gq_cd.cuh"
+#include "gq_codebook.cuh"
 #include "gq_kernels.cuh"
 
 #define GQ_VERSION_NUMBER 100   /* 0.1.0 */
@@ -98,6 +99,8 @@ int32_t device_info(DeviceInfo **out)
         GQ_CUDA(cudaFuncSetAttribute(gq::pair_gemm_kernel<gq::MODE_OBJECTIVE>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, gq::OBJ_SMEM_BYTES));
         GQ_CUDA(cudaFuncSetAttribute(gq::pair_gemm_kernel<gq::MODE_PANEL>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, gq::OBJ_SMEM_BYTES));
+        GQ_CUDA(cudaFuncSetAttribute(gq::pair_gemm_kernel<gq::MODE_FULL>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, gq::OBJ_SMEM_BYTES));
         GQ_CUDA(cudaFuncSetAttribute(gq::cd_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      gq::CD_SMEM_BYTES));
@@ -259,6 +262,35 @@ ObjectiveLayout objective_layout(int64_t d_in, int64_t d_out, int32_t g)
     L.partials_off = 2 * mat;
     L.total = L.partials_off +
               round_up(static_cast<size_t>(tiles_for(d_in)) * g * gq::PARTIALS_PER_UNIT * sizeof(double), 1024);
+    return L;
+}
+
+struct CodebookLayout {
+    size_t h0, h1, h2, w0, w1, w2, qt, hw, pm, hp, gmat, rvec, total;
+    int64_t slab_channels, slab_ld;
+};
+CodebookLayout codebook_layout(int64_t d_in, int64_t d_out, int32_t g, int32_t m)
+{
+    CodebookLayout L;
+    const int64_t mk = d_out / g;
+    L.slab_channels = mk < gq::CB_SLAB_CHANNELS ? mk : gq::CB_SLAB_CHANNELS;
+    L.slab_ld = (L.slab_channels * m + 7) / 8 * 8;
+    const size_t h2 = round_up(static_cast<size_t>(g) * d_in * d_in * 2, 1024);
+    const size_t w2 = round_up(static_cast<size_t>(d_in) * d_out * 2, 1024);
+    size_t o = 0;
+    L.h0 = o; o += h2;
+    L.h1 = o; o += h2;
+    L.h2 = o; o += h2;
+    L.w0 = o; o += w2;
+    L.w1 = o; o += w2;
+    L.w2 = o; o += w2;
+    L.qt = o; o += round_up(static_cast<size_t>(d_in) * d_out, 1024);
+    L.hw = o; o += round_up(static_cast<size_t>(d_in) * d_out * 4, 1024);
+    L.pm = o; o += round_up(static_cast<size_t>(d_in) * L.slab_ld * 2, 1024);
+    L.hp = o; o += round_up(static_cast<size_t>(d_in) * L.slab_ld * 4, 1024);
+    L.gmat = o; o += round_up(static_cast<size_t>(d_out) * gq::CB_MAX_LEVELS * gq::CB_MAX_LEVELS * 8, 1024);
+    L.rvec = o; o += round_up(static_cast<size_t>(d_out) * gq::CB_MAX_LEVELS * 8, 1024);
+    L.total = o;
     return L;
 }
 
@@ -475,7 +507,8 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     const int grid = 2 * p.sched.pairs;
     {
         LaunchScope scope(GQ_KERNEL_GRAM_DOT, st);
-        gq::pair_gemm_kernel<gq::MODE_OBJECTIVE><<<grid, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(mapHi, mapLo, mapHi, mapLo, p);
+        gq::pair_gemm_kernel<gq::MODE_OBJECTIVE><<<grid, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(mapHi, mapLo, mapHi, mapLo, mapHi,
+                                                                                               mapLo, p);
     }
     GQ_CUDA(cudaGetLastError());
     {
@@ -576,7 +609,8 @@ int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, i
     p.status = di->status_ptr;
     p.wait_budget_ns = wait_budget_ns();
     const int grid = 2 * p.sched.pairs;
-    gq::pair_gemm_kernel<gq::MODE_OBJECTIVE><<<grid, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(mapHi, mapLo, mapHi, mapLo, p);
+    gq::pair_gemm_kernel<gq::MODE_OBJECTIVE><<<grid, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(mapHi, mapLo, mapHi, mapLo, mapHi,
+                                                                                               mapLo, p);
     g_launches.fetch_add(1);
     GQ_CUDA(cudaGetLastError());
     gq::reduce_partials_kernel<<<1, 1024, 0, st>>>(partials, tiles, g, gq::PARTIALS_PER_UNIT, loss_out);
@@ -676,7 +710,7 @@ int32_t gq_cd_cycles(const float *W, float *W_hat, uint8_t *Q, const float *code
                 {
                     LaunchScope scope(GQ_KERNEL_CD_PANEL, st);
                     gq::pair_gemm_kernel<gq::MODE_PANEL><<<2 * pp.sched.pairs, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(
-                        mapHhi, mapHlo, mapEhi, mapElo, pp);
+                        mapHhi, mapHlo, mapEhi, mapElo, mapEhi, mapElo, pp);
                 }
                 GQ_CUDA(cudaGetLastError());
             }
@@ -697,6 +731,139 @@ int32_t gq_cd_cycles(const float *W, float *W_hat, uint8_t *Q, const float *code
         gq::cd_finish_kernel<<<tgrid, 256, 0, st>>>(Wht, Qt, static_cast<int>(d_in), static_cast<int>(d_out), W_hat, Q);
     }
     GQ_CUDA(cudaGetLastError());
+    return GQ_OK;
+}
+
+size_t gq_codebook_workspace_bytes(int64_t d_in, int64_t d_out, int32_t g, int32_t m)
+{
+    if (m < 1 || m > gq::CB_MAX_LEVELS || check_layer_shape(d_in, d_out, g, true) != GQ_OK) return 0;
+    return codebook_layout(d_in, d_out, g, m).total;
+}
+
+int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t d_in, int64_t d_out, const float *H,
+                           int32_t g, double lambda, float *codebook, float *W_hat, void *workspace,
+                           size_t workspace_bytes, void *stream)
+{
+    if (!W || !Q || !H || !codebook || m < 1 || !(lambda >= 0.0)) return GQ_ERR_INVALID_ARG;
+    if (int32_t rc = check_layer_shape(d_in, d_out, g, true)) return rc;
+    if (m > gq::CB_MAX_LEVELS) return GQ_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned(W, 16) || !aligned(H, 16) || !aligned(codebook, 4) || (W_hat && !aligned(W_hat, 16))) return GQ_ERR_ALIGNMENT;
+    const CodebookLayout L = codebook_layout(d_in, d_out, g, m);
+    if (!workspace || workspace_bytes < L.total) return GQ_ERR_WORKSPACE;
+    if (!aligned(workspace, 1024)) return GQ_ERR_ALIGNMENT;
+    DeviceInfo *di;
+    if (int32_t rc = device_info(&di)) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    __nv_bfloat16 *H0 = reinterpret_cast<__nv_bfloat16 *>(ws + L.h0), *H1 = reinterpret_cast<__nv_bfloat16 *>(ws + L.h1),
+                  *H2 = reinterpret_cast<__nv_bfloat16 *>(ws + L.h2);
+    __nv_bfloat16 *W0 = reinterpret_cast<__nv_bfloat16 *>(ws + L.w0), *W1 = reinterpret_cast<__nv_bfloat16 *>(ws + L.w1),
+                  *W2 = reinterpret_cast<__nv_bfloat16 *>(ws + L.w2);
+    uint8_t *Qt = ws + L.qt;
+    float *HW = reinterpret_cast<float *>(ws + L.hw);
+    __nv_bfloat16 *Pm = reinterpret_cast<__nv_bfloat16 *>(ws + L.pm);
+    float *HP = reinterpret_cast<float *>(ws + L.hp);
+    double *Gm = reinterpret_cast<double *>(ws + L.gmat);
+    double *Rv = reinterpret_cast<double *>(ws + L.rvec);
+    const int64_t mk = d_out / g;
+    const long long hcount = static_cast<long long>(g) * d_in * d_in;
+    {
+        LaunchScope scope(GQ_KERNEL_CB_AUX, st);
+        gq::cb_split3_kernel<<<grid_for(hcount, 256, di->sm_count, 8), 256, 0, st>>>(H, hcount, H0, H1, H2);
+    }
+    GQ_CUDA(cudaGetLastError());
+    {
+        const dim3 tgrid(static_cast<unsigned>((d_in + 31) / 32), static_cast<unsigned>((d_out + 31) / 32));
+        LaunchScope scope(GQ_KERNEL_CB_AUX, st);
+        gq::cb_transpose_kernel<<<tgrid, 256, 0, st>>>(W, Q, static_cast<int>(d_in), static_cast<int>(d_out), W0, W1, W2, Qt);
+    }
+    GQ_CUDA(cudaGetLastError());
+    CUtensorMap mH0, mH1, mH2, mW0, mW1, mW2, mPm;
+    if (int32_t rc = make_map(&mH0, H0, d_in, d_in, g, d_in, d_in * d_in)) return rc;
+    if (int32_t rc = make_map(&mH1, H1, d_in, d_in, g, d_in, d_in * d_in)) return rc;
+    if (int32_t rc = make_map(&mH2, H2, d_in, d_in, g, d_in, d_in * d_in)) return rc;
+    if (int32_t rc = make_map(&mW0, W0, d_out, d_in, 1, d_out, d_in * d_out)) return rc;
+    if (int32_t rc = make_map(&mW1, W1, d_out, d_in, 1, d_out, d_in * d_out)) return rc;
+    if (int32_t rc = make_map(&mW2, W2, d_out, d_in, 1, d_out, d_in * d_out)) return rc;
+    if (int32_t rc = make_map(&mPm, Pm, L.slab_ld, d_in, 1, L.slab_ld, d_in * L.slab_ld)) return rc;
+
+    auto launch_full = [&](gq::PairGemmParams &pp, const CUtensorMap &b0, const CUtensorMap &b1, const CUtensorMap &b2,
+                           int kernel_id) -> int32_t {
+        pp.d = static_cast<int>(d_in);
+        pp.rows = static_cast<int>(d_in);
+        pp.g = g;
+        pp.map_grouped[0] = pp.map_grouped[1] = pp.map_grouped[2] = 1;
+        pp.map_grouped[3] = pp.map_grouped[4] = pp.map_grouped[5] = 0;
+        pp.col_tiles = (pp.cols + gq::TILE_N - 1) / gq::TILE_N;
+        const int row_blocks = static_cast<int>((d_in + gq::TILE_M - 1) / gq::TILE_M);
+        const int units = row_blocks * pp.col_tiles;
+        const int ksteps = pp.n_terms * static_cast<int>((d_in + gq::TILE_K - 1) / gq::TILE_K);
+        pp.sched = gq::plan_schedule(units, ksteps, units < di->max_pairs ? units : di->max_pairs, false);
+        pp.status = di->status_ptr;
+        pp.wait_budget_ns = wait_budget_ns();
+        {
+            LaunchScope scope(kernel_id, st);
+            gq::pair_gemm_kernel<gq::MODE_FULL><<<2 * pp.sched.pairs, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(
+                mH0, mH1, mH2, b0, b1, b2, pp);
+        }
+        GQ_CUDA(cudaGetLastError());
+        return GQ_OK;
+    };
+
+    for (int32_t k = 0; k < g; ++k) {
+        // HW[:, group k] = H_k W_k^T: terms of total order <= 2 of (H0 + H1 + H2)(W0 + W1 + W2)
+        gq::PairGemmParams pp{};
+        pp.n_terms = 6;
+        const int ta[6] = {0, 0, 1, 0, 1, 2}, tb[6] = {3, 4, 3, 5, 4, 3};
+        for (int t = 0; t < 6; ++t) { pp.term_a[t] = ta[t]; pp.term_b[t] = tb[t]; }
+        pp.full_k = k;
+        pp.col0 = static_cast<int>(k * mk);
+        pp.cols = static_cast<int>(mk);
+        pp.C = HW + k * mk;
+        pp.ldc = d_out;
+        if (int32_t rc = launch_full(pp, mW0, mW1, mW2, GQ_KERNEL_CB_GEMM)) return rc;
+        for (int64_t j0 = k * mk; j0 < (k + 1) * mk; j0 += L.slab_channels) {
+            const int nch = static_cast<int>((k + 1) * mk - j0 < L.slab_channels ? (k + 1) * mk - j0 : L.slab_channels);
+            {
+                const long long total = static_cast<long long>(d_in) * nch * m;
+                LaunchScope scope(GQ_KERNEL_CB_AUX, st);
+                gq::cb_onehot_kernel<<<grid_for(total, 256, di->sm_count, 8), 256, 0, st>>>(
+                    Qt, static_cast<int>(d_in), static_cast<int>(d_out), static_cast<int>(j0), nch, m, Pm, L.slab_ld);
+            }
+            GQ_CUDA(cudaGetLastError());
+            // HP = H_k Pm: the one-hot columns are exact in bf16, so three terms give the exact products
+            gq::PairGemmParams pq{};
+            pq.n_terms = 3;
+            pq.term_a[0] = 0; pq.term_b[0] = 3;
+            pq.term_a[1] = 1; pq.term_b[1] = 3;
+            pq.term_a[2] = 2; pq.term_b[2] = 3;
+            pq.full_k = k;
+            pq.col0 = 0;
+            pq.cols = nch * m;
+            pq.C = HP;
+            pq.ldc = L.slab_ld;
+            if (int32_t rc = launch_full(pq, mPm, mPm, mPm, GQ_KERNEL_CB_GEMM)) return rc;
+            {
+                LaunchScope scope(GQ_KERNEL_CB_FOLD, st);
+                gq::cb_fold_kernel<<<(nch + 7) / 8, 128, 0, st>>>(HP, L.slab_ld, HW, Qt, static_cast<int>(d_in),
+                                                                 static_cast<int>(d_out), static_cast<int>(j0), nch, m, Gm, Rv);
+            }
+            GQ_CUDA(cudaGetLastError());
+        }
+    }
+    {
+        LaunchScope scope(GQ_KERNEL_CB_FOLD, st);
+        gq::cb_solve_kernel<<<static_cast<unsigned>((d_out + 127) / 128), 128, 0, st>>>(Gm, Rv, static_cast<int>(d_out), m,
+                                                                                      lambda, codebook);
+    }
+    GQ_CUDA(cudaGetLastError());
+    if (W_hat) {
+        const long long count = static_cast<long long>(d_out) * d_in;
+        LaunchScope scope(GQ_KERNEL_CB_AUX, st);
+        gq::cb_apply_kernel<<<grid_for(count, 256, di->sm_count, 8), 256, 0, st>>>(codebook, Q, count, static_cast<int>(d_in),
+                                                                                 m, W_hat);
+        GQ_CUDA(cudaGetLastError());
+    }
     return GQ_OK;
 }
 

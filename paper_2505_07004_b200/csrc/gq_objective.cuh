@@ -23,6 +23,9 @@
 //                  B = E = (What - W)^T (rows = input coordinates c, columns = output channels); work unit =
 //                  (group, tile of 256 channels, piece of the contraction range); the pieces of a tile are
 //                  added into P with red.global.add.
+// MODE_FULL        C[r][col] = sum_c A[c][r] * B[c][col], a plain product of MN-major operands (used by the
+//                  LNQ codebook step: A = H_k split three ways, B = W^T or one-hot assignment columns); work
+//                  unit = (256-row block, 256-column tile), each unit stores its tile.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -38,11 +41,13 @@ constexpr int OBJ_B_BYTES = (CTA_ROWS / BOX_FEATURES) * BOX_BYTES;
 constexpr int OBJ_STAGE_BYTES = OBJ_A_BYTES + OBJ_B_BYTES;
 constexpr int OBJ_THREADS = 256;
 constexpr int OBJ_SMEM_BYTES = OBJ_STAGES * OBJ_STAGE_BYTES + 1024;   // + slack to align the ring to 1024 B
-constexpr int MAX_TERMS = 3;
+constexpr int MAX_TERMS = 6;
+constexpr int MAX_MAPS = 6;
 constexpr int PARTIALS_PER_UNIT = 8;                   // one fp64 per (CTA of the pair, epilogue warp)
 
 constexpr int MODE_OBJECTIVE = 0;
 constexpr int MODE_PANEL = 1;
+constexpr int MODE_FULL = 2;
 
 struct PairGemmParams {
     int d;                   // number of features (d_in)
@@ -51,9 +56,9 @@ struct PairGemmParams {
     int nj;                  // ceil(d / 256): tile blocks per side
     int raster;              // edge (in tiles) of the super-blocks of the tile order
     int n_terms;
-    int term_a[MAX_TERMS];   // which of the four tensor maps feeds A / B in each term
+    int term_a[MAX_TERMS];   // which of the six tensor maps feeds A / B in each term
     int term_b[MAX_TERMS];
-    int map_grouped[4];      // 1: the map's third coordinate is the group index; 0: always 0
+    int map_grouped[MAX_MAPS];   // 1: the map's third coordinate is the group index; 0: always 0
     Schedule sched;          // units = (number of upper-triangular 256 x 256 tiles) * g,
                              // ksteps = n_terms * ceil(rows / 64)
     const float *H;          // MODE_OBJECTIVE: [g][d][d], only a <= b is read
@@ -67,6 +72,12 @@ struct PairGemmParams {
     int mk;                  // channels per group
     int d_out;
     float *P;                // [256][d_out]
+    // MODE_FULL: C[r][col - col0] = sum over all `rows` contraction rows, r < d, col0 <= col < col0 + cols
+    int full_k;              // group index given to the grouped maps
+    int col0, cols;          // B columns of this launch
+    int col_tiles;           // ceil(cols / 256)
+    float *C;                // output, row stride ldc (floats), written (not added)
+    long long ldc;
     uint32_t *status;        // device status word (4 x u32)
     unsigned long long wait_budget_ns;
 };
@@ -91,6 +102,16 @@ __device__ __forceinline__ bool item_geom(const PairGemmParams &p, const WorkIte
         ge.ks1 = w.ks1;
         return true;
     }
+    if (MODE == MODE_FULL) {
+        ge.ti = w.unit / p.col_tiles;
+        ge.tj = w.unit % p.col_tiles;
+        ge.k = p.full_k;
+        ge.a0 = ge.ti * TILE_M + static_cast<int>(rank) * CTA_ROWS;
+        ge.b0 = p.col0 + ge.tj * TILE_N + static_cast<int>(rank) * CTA_ROWS;
+        ge.ks0 = w.ks0;
+        ge.ks1 = w.ks1;
+        return true;
+    }
     const int piece = w.unit % p.pieces;
     const int t = (w.unit / p.pieces) % p.ch_tiles;
     ge.k = w.unit / (p.pieces * p.ch_tiles);
@@ -108,7 +129,7 @@ __device__ __forceinline__ bool item_geom(const PairGemmParams &p, const WorkIte
 template <int MODE>
 __device__ __forceinline__ void kstep_coords(const PairGemmParams &p, int ks, int kblocks, int &term, int &row)
 {
-    if (MODE == MODE_OBJECTIVE) {
+    if (MODE != MODE_PANEL) {
         term = ks / kblocks;
         row = (ks - term * kblocks) * TILE_K;
     } else {
@@ -122,6 +143,7 @@ template <int MODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(OBJ_THREADS, 1)
 pair_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1,
                  const __grid_constant__ CUtensorMap map2, const __grid_constant__ CUtensorMap map3,
+                 const __grid_constant__ CUtensorMap map4, const __grid_constant__ CUtensorMap map5,
                  const PairGemmParams p)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -155,6 +177,8 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
         prefetch_tensormap(&map1);
         prefetch_tensormap(&map2);
         prefetch_tensormap(&map3);
+        prefetch_tensormap(&map4);
+        prefetch_tensormap(&map5);
     }
     if (warp == 2) {
         tmem_alloc(smem_u32(&tmem_base_smem), TMEM_COLS);
@@ -178,7 +202,7 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
         for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
             ItemGeom ge;
             if (!item_geom<MODE>(p, w, rank, ge)) continue;
-            const void *maps[4] = {&map0, &map1, &map2, &map3};
+            const void *maps[MAX_MAPS] = {&map0, &map1, &map2, &map3, &map4, &map5};
             for (int ks = ge.ks0; ks < ge.ks1; ++ks) {
                 int term, row;
                 kstep_coords<MODE>(p, ks, kblocks, term, row);
@@ -307,6 +331,30 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
                 for (int off = 16; off > 0; off >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, off);
                 if (lane == 0)
                     p.partials[static_cast<size_t>(w.unit) * PARTIALS_PER_UNIT + rank * 4 + q] = dsum;
+            } else if (MODE == MODE_FULL) {
+                const int row0 = ge.ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + q * 32;
+                const int row = row0 + lane;
+                float *crow = p.C + static_cast<size_t>(row < p.d ? row : 0) * p.ldc;
+#pragma unroll 1
+                for (int cc = 0; cc < TILE_N / 32; ++cc) {
+                    const int c0 = ge.tj * TILE_N + cc * 32;                           // column relative to col0
+                    if (c0 >= p.cols || row0 >= p.d) break;
+                    uint32_t r[32];
+                    tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
+                                      static_cast<uint32_t>(buf * TILE_N + cc * 32), r);
+                    tmem_ld_wait();
+                    if (row >= p.d) continue;
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        if (c0 + v * 4 < p.cols)
+                            *reinterpret_cast<float4 *>(crow + c0 + v * 4) =
+                                make_float4(__uint_as_float(r[v * 4 + 0]), __uint_as_float(r[v * 4 + 1]),
+                                            __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
+                    }
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_acc_empty[buf]), 0));
             } else {
                 const int rl = static_cast<int>(rank) * CTA_ROWS + q * 32 + lane;      // row inside the block
                 const bool row_ok = p.s0 + rl < p.d;
