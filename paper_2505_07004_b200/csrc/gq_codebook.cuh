@@ -93,8 +93,10 @@ cb_onehot_kernel(const uint8_t *__restrict__ Qt, int d_in, int d_out, int j0, in
     }
 }
 
-// Fold over the rows of each level.  One CTA = 8 channels of the slab x 16 threads; thread (ch, q') owns column
-// q' of G^(ch) in shared memory (fp64), so no two threads ever add to the same word; thread q' = 0 also owns r.
+// Fold over the rows of each level.  One CTA = 8 channels of the slab x 16 threads x one of gridDim.y row
+// ranges; thread (ch, q') owns column q' of G^(ch) in shared memory (fp64), so no two threads of a CTA ever add
+// to the same word; thread q' = 0 also owns r.  The row ranges are combined with fp64 atomic adds (the order
+// of at most gridDim.y fp64 partial sums is the only thing that can vary from run to run).
 __global__ void __launch_bounds__(128)
 cb_fold_kernel(const float *__restrict__ HP, long long ld_hp, const float *__restrict__ HW, const uint8_t *__restrict__ Qt,
                int d_in, int d_out, int j0, int nch, int m, double *__restrict__ G, double *__restrict__ R)
@@ -109,19 +111,35 @@ cb_fold_kernel(const float *__restrict__ HP, long long ld_hp, const float *__res
     if (jj < nch && qp < m) {
         const int j = j0 + jj;
         const float *hp = HP + static_cast<size_t>(jj) * m + qp;
-        for (int i = 0; i < d_in; ++i) {
-            int q = Qt[static_cast<size_t>(i) * d_out + j];
-            q = q < m ? q : m - 1;                       // codes are expected to be < m
-            Gs[ch][q][qp] += static_cast<double>(hp[static_cast<size_t>(i) * ld_hp]);
-            if (qp == 0) Rs[ch][q] += static_cast<double>(HW[static_cast<size_t>(i) * d_out + j]);
+        constexpr int BATCH = 8;                         // independent loads in flight per thread
+        const int rows_per = (d_in + static_cast<int>(gridDim.y) - 1) / static_cast<int>(gridDim.y);
+        const int i_begin = static_cast<int>(blockIdx.y) * rows_per;
+        const int i_end = i_begin + rows_per < d_in ? i_begin + rows_per : d_in;
+        for (int i0 = i_begin; i0 < i_end; i0 += BATCH) {
+            int q[BATCH];
+            float v[BATCH], w[BATCH];
+#pragma unroll
+            for (int t = 0; t < BATCH; ++t) {
+                const int i = i0 + t;
+                const bool ok = i < i_end;
+                q[t] = ok ? Qt[static_cast<size_t>(i) * d_out + j] : 0;
+                v[t] = ok ? hp[static_cast<size_t>(i) * ld_hp] : 0.0f;
+                w[t] = (ok && qp == 0) ? HW[static_cast<size_t>(i) * d_out + j] : 0.0f;
+            }
+#pragma unroll
+            for (int t = 0; t < BATCH; ++t) {
+                const int qq = q[t] < m ? q[t] : m - 1;  // codes are expected to be < m
+                Gs[ch][qq][qp] += static_cast<double>(v[t]);
+                if (qp == 0) Rs[ch][qq] += static_cast<double>(w[t]);
+            }
         }
     }
     __syncthreads();
-    if (jj < nch) {
+    if (jj < nch && qp < m) {                        // G and R were zeroed by the host; row ranges add up
         const int j = j0 + jj;
-        for (int q = 0; q < CB_MAX_LEVELS; ++q)
-            G[(static_cast<size_t>(j) * CB_MAX_LEVELS + q) * CB_MAX_LEVELS + qp] = (q < m && qp < m) ? Gs[ch][q][qp] : 0.0;
-        R[static_cast<size_t>(j) * CB_MAX_LEVELS + qp] = qp < m ? Rs[ch][qp] : 0.0;
+        for (int q = 0; q < m; ++q)
+            atomicAdd(&G[(static_cast<size_t>(j) * CB_MAX_LEVELS + q) * CB_MAX_LEVELS + qp], Gs[ch][q][qp]);
+        atomicAdd(&R[static_cast<size_t>(j) * CB_MAX_LEVELS + qp], Rs[ch][qp]);
     }
 }
 

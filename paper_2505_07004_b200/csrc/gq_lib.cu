@@ -810,6 +810,8 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
         return GQ_OK;
     };
 
+    GQ_CUDA(cudaMemsetAsync(Gm, 0, static_cast<size_t>(d_out) * gq::CB_MAX_LEVELS * gq::CB_MAX_LEVELS * sizeof(double), st));
+    GQ_CUDA(cudaMemsetAsync(Rv, 0, static_cast<size_t>(d_out) * gq::CB_MAX_LEVELS * sizeof(double), st));
     for (int32_t k = 0; k < g; ++k) {
         // HW[:, group k] = H_k W_k^T: terms of total order <= 2 of (H0 + H1 + H2)(W0 + W1 + W2)
         gq::PairGemmParams pp{};
@@ -845,7 +847,7 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
             if (int32_t rc = launch_full(pq, mPm, mPm, mPm, GQ_KERNEL_CB_GEMM)) return rc;
             {
                 LaunchScope scope(GQ_KERNEL_CB_FOLD, st);
-                gq::cb_fold_kernel<<<(nch + 7) / 8, 128, 0, st>>>(HP, L.slab_ld, HW, Qt, static_cast<int>(d_in),
+                gq::cb_fold_kernel<<<dim3((nch + 7) / 8, 8), 128, 0, st>>>(HP, L.slab_ld, HW, Qt, static_cast<int>(d_in),
                                                                  static_cast<int>(d_out), static_cast<int>(j0), nch, m, Gm, Rv);
             }
             GQ_CUDA(cudaGetLastError());
