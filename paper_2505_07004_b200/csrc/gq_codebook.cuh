@@ -6,9 +6,11 @@
 // The two d_in^2-sized contractions run on the tensor cores (pair_gemm_kernel<MODE_FULL>):
 //     HW = H_k W_k^T                      [d_in x channels]
 //     HP = H_k [P^(j0) ... P^(j0+c-1)]    [d_in x (channels * m)]   for a slab of channels at a time
-// with H carried as three bf16 matrices whose sum is the fp32 value exactly (8 + 8 + 8 mantissa bits), the
-// one-hot columns exact in bf16 and W as three bf16 terms as well; accumulation is fp32.  The kernels here
-// prepare those operands, fold HP and HW over the rows of each level (fp64),
+// with H split into three bf16 matrices whose sum is the fp32 value exactly (8 + 8 + 8 mantissa bits) and W
+// likewise; accumulation is fp32.  HW takes every product of total order <= 2 (six terms).  HP, where the
+// one-hot columns are exact in bf16, takes the two leading terms of H: what it drops is below 2^-16 of each
+// entry, the size of the fp32 accumulation error of these 4096-long sums, and HP is 16 x the work of HW.
+// The kernels here prepare those operands, fold HP and HW over the rows of each level (fp64),
 //     G^(j)[q][q'] = sum_{i : Q_ij = q} HP[i][j m + q'],      r^(j)[q] = sum_{i : Q_ij = q} HW[i][j],
 // and solve the m x m systems by Cholesky in fp64.
 #pragma once

@@ -833,12 +833,11 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
                     Qt, static_cast<int>(d_in), static_cast<int>(d_out), static_cast<int>(j0), nch, m, Pm, L.slab_ld);
             }
             GQ_CUDA(cudaGetLastError());
-            // HP = H_k Pm: the one-hot columns are exact in bf16, so three terms give the exact products
+            // HP = H_k Pm: the one-hot columns are exact in bf16; the two leading terms of H carry 16 mantissa bits
             gq::PairGemmParams pq{};
-            pq.n_terms = 3;
+            pq.n_terms = 2;
             pq.term_a[0] = 0; pq.term_b[0] = 3;
             pq.term_a[1] = 1; pq.term_b[1] = 3;
-            pq.term_a[2] = 2; pq.term_b[2] = 3;
             pq.full_k = k;
             pq.col0 = 0;
             pq.cols = nch * m;
