@@ -78,20 +78,32 @@ cb_transpose_kernel(const float *__restrict__ W, const uint8_t *__restrict__ Q, 
 }
 
 // One-hot columns of channels [j0, j0 + nch): Pm[i][jj * m + q] = (Qt[i][j0 + jj] == q), bf16, row stride ld.
+// One thread writes the m columns of one (row, channel); with m = 16 and ld a multiple of 8 that is two
+// 16-byte stores, and consecutive threads write consecutive 32-byte pieces.
 __global__ void __launch_bounds__(256)
 cb_onehot_kernel(const uint8_t *__restrict__ Qt, int d_in, int d_out, int j0, int nch, int m,
                  __nv_bfloat16 *__restrict__ Pm, long long ld)
 {
-    const long long cols = static_cast<long long>(nch) * m;
-    const long long total = static_cast<long long>(d_in) * cols;
+    const long long total = static_cast<long long>(d_in) * nch;
     const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    const bool wide = m == 16 && (ld & 7) == 0;
     for (long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total; idx += stride) {
-        const int i = static_cast<int>(idx / cols);
-        const int c = static_cast<int>(idx - static_cast<long long>(i) * cols);
-        const int jj = c / m, q = c - jj * m;
-        const int code = Qt[static_cast<size_t>(i) * d_out + j0 + jj];
-        const bool one = (code < m ? code : m - 1) == q;
-        Pm[static_cast<size_t>(i) * ld + c] = __float2bfloat16_rn(one ? 1.0f : 0.0f);
+        const int i = static_cast<int>(idx / nch);
+        const int jj = static_cast<int>(idx - static_cast<long long>(i) * nch);
+        int code = Qt[static_cast<size_t>(i) * d_out + j0 + jj];
+        code = code < m ? code : m - 1;
+        __nv_bfloat16 *dst = Pm + static_cast<size_t>(i) * ld + static_cast<size_t>(jj) * m;
+        if (wide) {
+            uint32_t w[8];
+#pragma unroll
+            for (int t = 0; t < 8; ++t)            // bf16 1.0 = 0x3F80 in the low or the high half of word t
+                w[t] = (code >> 1) == t ? ((code & 1) ? 0x3F800000u : 0x00003F80u) : 0u;
+            uint4 *d4 = reinterpret_cast<uint4 *>(dst);
+            d4[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            d4[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        } else {
+            for (int q = 0; q < m; ++q) dst[q] = __float2bfloat16_rn(q == code ? 1.0f : 0.0f);
+        }
     }
 }
 

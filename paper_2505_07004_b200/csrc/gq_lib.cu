@@ -827,7 +827,7 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
         for (int64_t j0 = k * mk; j0 < (k + 1) * mk; j0 += L.slab_channels) {
             const int nch = static_cast<int>((k + 1) * mk - j0 < L.slab_channels ? (k + 1) * mk - j0 : L.slab_channels);
             {
-                const long long total = static_cast<long long>(d_in) * nch * m;
+                const long long total = static_cast<long long>(d_in) * nch;
                 LaunchScope scope(GQ_KERNEL_CB_AUX, st);
                 gq::cb_onehot_kernel<<<grid_for(total, 256, di->sm_count, 8), 256, 0, st>>>(
                     Qt, static_cast<int>(d_in), static_cast<int>(d_out), static_cast<int>(j0), nch, m, Pm, L.slab_ld);
