@@ -129,3 +129,68 @@ def test_lnq_loop_descends_like_the_oracle(dev):
     print("LNQ objective per group: start %s, GPU %s, oracle %s" % (f[0].reshape(g, mk).sum(1), tg, to))
     assert np.all(np.abs(tg - to) <= 2e-2 * to)
     assert np.all(tg < 0.9 * f[0].reshape(g, mk).sum(1))
+
+
+def test_full_size_layer_sampled_channels(dev):
+    """The layer size the timing script uses (d_in = d_out = 4096, 4 groups, 16 levels), whole layer on the GPU,
+    oracle on sampled channels (channels are independent given H_k and the codes): codebook step, then one CD
+    cycle, then the codebook step on the new codes.  Inputs are drawn on the device with torch and the same
+    bits are handed to the oracle."""
+    d_in = d_out = 4096
+    g, m, n = 4, 16, 8192
+    mk = d_out // g
+    gen = torch.Generator(device=dev).manual_seed(31)
+    X = torch.randn(n, d_in, device=dev, generator=gen) * torch.exp(0.7 * torch.randn(d_in, device=dev, generator=gen))
+    sal = torch.rand(g, n, device=dev, generator=gen) * torch.exp(torch.randn(g, n, device=dev, generator=gen))
+    old = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = False
+    Hd = torch.stack([(X * sal[k][:, None]).T @ X for k in range(g)])
+    torch.backends.cuda.matmul.allow_tf32 = old
+    Hd = ((Hd + Hd.transpose(1, 2)) / 2).contiguous()
+    del X, sal
+    Wd = 0.02 * torch.randn(d_out, d_in, device=dev, generator=gen)
+    lo, hi = Wd.min(1, keepdim=True).values, Wd.max(1, keepdim=True).values
+    cb0 = lo + (hi - lo) * (torch.arange(m, device=dev)[None, :] + 0.5) / m
+    Q0 = ((Wd - lo) / (hi - lo) * m).floor().clamp_(0, m - 1).to(torch.uint8)          # a valid starting assignment
+    sel = np.concatenate([k * mk + np.array([0, 1, 517, mk - 1]) for k in range(g)])
+    W, H = Wd.cpu().numpy(), Hd.cpu().numpy()
+
+    cbw = libgq.alloc_workspace(libgq.gq_codebook_workspace_bytes(d_in, d_out, g, m), dev)
+    cdw = libgq.alloc_workspace(libgq.gq_cd_workspace_bytes(d_in, d_out, g), dev)
+    What = torch.empty_like(Wd)
+    cb1, What = libgq.gq_codebook_update(Wd, Q0, m, Hd, cbw, W_hat=What)
+    cb1_h, What1_h = cb1.cpu().numpy(), What.cpu().numpy()
+    What2, Q2 = libgq.gq_cd_cycles(Wd, What, cb1, Hd, 1, cdw, Q=Q0.clone())
+    cb3, What3 = libgq.gq_codebook_update(Wd, Q2, m, Hd, cbw, W_hat=torch.empty_like(Wd))
+    libgq.gq_check()
+    Q0_h, Q2_h, What2_h = Q0.cpu().numpy().astype(np.int32), Q2.cpu().numpy().astype(np.int32), What2.cpu().numpy()
+    cb3_h = cb3.cpu().numpy()
+
+    n_tie = 0
+    for j in sel:
+        Hk = H[j // mk][None].astype(np.float64)
+        # codebook step on the starting codes
+        c_o = cdo.codebook_update(W[j:j + 1], Q0_h[j:j + 1], Hk, m)[0]
+        assert np.abs(cb1_h[j] - c_o).max() <= C_RTOL * np.abs(c_o).max()
+        assert np.array_equal(What1_h[j], cb1_h[j][Q0_h[j]])
+        # one CD cycle from the GPU's own codebook and starting point
+        Wo, Qo = cdo.cd(W[j:j + 1], What1_h[j:j + 1], cb1_h[j:j + 1], Hk, 1, 128)
+        assert np.array_equal(What2_h[j], cb1_h[j][Q2_h[j]])
+        f0 = cdo.channel_objective(What1_h[j].astype(np.float64) - W[j], Hk[0])
+        fg = cdo.channel_objective(What2_h[j].astype(np.float64) - W[j], Hk[0])
+        fo = cdo.channel_objective(Wo[0].astype(np.float64) - W[j], Hk[0])
+        assert fg <= f0 * (1 + 1e-6)
+        if not np.array_equal(Q2_h[j], Qo[0]):
+            i = int(np.nonzero(Q2_h[j] != Qo[0])[0][0])
+            state = What1_h[j].astype(np.float64).copy()
+            state[:i] = Wo[0, :i]
+            t, mag = cdo.coordinate_target(W[j], state, Hk[0], i)
+            da, db = abs(t - float(cb1_h[j, Q2_h[j, i]])), abs(t - float(cb1_h[j, Qo[0, i]]))
+            assert abs(da - db) <= 2e-4 * mag, "channel %d coordinate %d is no near-tie" % (j, i)
+            assert abs(fg - fo) <= 2e-2 * fo
+            n_tie += 1
+        # codebook step on the GPU's new codes
+        c_o = cdo.codebook_update(W[j:j + 1], Q2_h[j:j + 1], Hk, m)[0]
+        assert np.abs(cb3_h[j] - c_o).max() <= C_RTOL * np.abs(c_o).max()
+    print("sampled channels on a near-tie path: %d of %d" % (n_tie, len(sel)))
+    assert n_tie <= len(sel) // 2
