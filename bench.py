@@ -253,7 +253,9 @@ def run_ours(args, cfg, g):
             libgq.gq_layer_objective_host(Xh, Gh, cfg.chunk, g, 1.0, Wh, Whh, arena, loss_host=loss_h)
         torch.cuda.synchronize()
         e2e_s = time.perf_counter() - t0
-        if abs(loss_h[g].item() - loss_host[g]) > 1e-9 * abs(loss_host[g]):
+        # same arithmetic on both paths; the units that were cut along the token axis are added to H in an
+        # order that varies from launch to launch, hence agreement to fp32 summation order only
+        if abs(loss_h[g].item() - loss_host[g]) > 1e-6 * abs(loss_host[g]):
             raise RuntimeError("host-buffer path and device path disagree: %r vs %r" % (loss_h[g].item(), loss_host[g]))
         h2d = Xh.numel() * 2 + Gh.numel() * 2 + Wh.numel() * 4 + Whh.numel() * 4
         d2h = (g + 1) * 8
@@ -320,7 +322,7 @@ def main():
     ap.add_argument("--workload", default="c1_7b_attn", choices=sorted(synth.CONFIGS))
     ap.add_argument("--g", type=int, default=0, help="override the number of groups (sweep config)")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--cpu-tokens", type=int, default=768)
+    ap.add_argument("--cpu-tokens", type=int, default=4096)
     ap.add_argument("--cpu-channels", type=int, default=128)
     ap.add_argument("--ref-tokens", type=int, default=256)
     ap.add_argument("--ref-channels", type=int, default=64)
