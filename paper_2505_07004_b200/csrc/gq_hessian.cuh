@@ -63,9 +63,6 @@ constexpr int HS_SMEM_BYTES = HS_STAGES * HS_STAGE_BYTES + HS_STAGING_BYTES + 10
 struct HessianParams {
     const __nv_bfloat16 *X;  // [n][ld_x]
     long long ld_x;
-    float *H;                // [g][d][d] (used by the register epilogue; the TMA epilogue goes through mapH)
-    int direct_epilogue;     // 1: accumulators are added to H straight from registers (red.global.add.v4.f32);
-                             // 0: through a shared-memory staging block and TMA reduce-add
     const uint2 *s2;         // [ceil(g / 2)][n]: split saliency of groups (2 q, 2 q + 1), see split_saliency_kernel
     int n;                   // tokens in this call
     int d;                   // d_in
@@ -428,20 +425,8 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                     tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                       static_cast<uint32_t>(kk * TILE_N + cc * 32), r);
                     tmem_ld_wait();
-                    if (p.direct_epilogue) {
-                        // short units: straight from registers, nothing to wait for (each lane adds eight
-                        // 16-byte pieces of its own row)
-                        const int row = row0 + lane;
-                        if (row < p.d) {
-                            float *hrow = p.H + (static_cast<size_t>(u.grp[kk]) * p.d + row) * static_cast<size_t>(p.d) + col0;
-#pragma unroll
-                            for (int v = 0; v < 8; ++v)
-                                if (col0 + v * 4 < p.d)
-                                    red_add_f32x4(hrow + v * 4, __uint_as_float(r[v * 4 + 0]), __uint_as_float(r[v * 4 + 1]),
-                                                  __uint_as_float(r[v * 4 + 2]), __uint_as_float(r[v * 4 + 3]));
-                        }
-                        continue;
-                    }
+                    if (lane == 0) bulk_wait_group_read0();   // the copy engine has read the previous staging block
+                    __syncwarp();
 #pragma unroll
                     for (int v = 0; v < 8; ++v)
                         st_shared_16(stg + static_cast<uint32_t>(lane * 128 + ((v ^ (lane & 7)) << 4)),
@@ -451,9 +436,7 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                     if (lane == 0) {
                         tma_reduce_add_3d(&mapH, stg, col0, row0, u.grp[kk]);
                         bulk_commit_group();
-                        bulk_wait_group_read0();      // staging block reusable once the copy engine has read it
                     }
-                    __syncwarp();
                 }
             }
             // This warp has read all it needs from tensor memory: tell the MMA issuer (first CTA).
@@ -462,6 +445,7 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
             if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_acc_empty), 0));
             acc_ph ^= 1u;
         }
+        if (lane == 0) bulk_wait_group_read0();       // shared memory must outlive the last reduce-add's read
     }
 
     __syncwarp();

@@ -239,11 +239,6 @@ int32_t check_layer_shape(int64_t d_in, int64_t d_out, int32_t g, bool need_out)
     return GQ_OK;
 }
 
-// Units of at most 64 k-steps (chunks of up to 4096 tokens) use the register epilogue of the Hessian kernel:
-// measured on the 70B MLP shape (4096-token chunks) 7.3 -> 6.9-7.1 ms per launch, while 8192-token chunks are
-// about 2 % faster with the TMA epilogue.
-bool ksteps_per_unit_short(int64_t n) { return n <= 64 * gq::TILE_K; }
-
 // Scratch of gq_hessian_accumulate: the split saliency words, 8 bytes per (pair of groups, token).
 size_t hessian_ws_bytes(int64_t n_max, int64_t, int32_t g)
 {
@@ -408,8 +403,6 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
     p.X = static_cast<const __nv_bfloat16 *>(X);
     p.ld_x = ld_x;
     p.s2 = static_cast<const uint2 *>(workspace);
-    p.H = H;
-    p.direct_epilogue = ksteps_per_unit_short(n) ? 1 : 0;
     p.n = static_cast<int>(n);
     p.d = static_cast<int>(d_in);
     p.g = g;
