@@ -112,6 +112,35 @@ size_t gq_hessian_workspace_bytes(int64_t n_max, int64_t d_in, int32_t g, uint32
 int32_t gq_hessian_finalize(float *H, int64_t d_in, int32_t g, void *stream);
 
 /*
+ * Token-sharded accumulation over several GPUs: H_k is a sum over tokens (Algorithm 1, line 4), so every GPU
+ * may run gq_hessian_accumulate on its own share of the tokens and the partial matrices are then added.
+ * These two calls do that exchange with plain loads from the other GPUs' memory (peer access enabled by the
+ * caller, e.g. through CUDA IPC or symmetric memory); no kernel waits for another GPU, the CALLER provides
+ * the synchronisation:
+ *     every rank:  accumulate its chunks;  barrier (all partial matrices complete)
+ *     every rank:  gq_hessian_reduce_share(...);  barrier (all shares reduced)
+ *     every rank:  gq_hessian_gather_shares(...); barrier (nobody still reads this rank's H)
+ *     every rank:  gq_hessian_finalize(own H, ...)
+ * The upper triangle is exchanged in 128 x 128 blocks; rank r owns blocks [r B / R, (r + 1) B / R) of the
+ * B = g nb (nb + 1) / 2 blocks (nb = ceil(d_in / 128)), numbered group after group and, inside a group, block
+ * column after block column.  reduce_share adds rank r's blocks over all R matrices in rank order (the result
+ * does not depend on which GPU forms it) and stores them in H_ranks[rank]; gather_shares copies the other
+ * ranks' blocks from their owners' matrices into H_ranks[rank].  Afterwards every rank holds the same upper
+ * triangle, bit for bit.
+ *
+ *   H_ranks    HOST array of `ranks` DEVICE pointers: the [g, d_in, d_in] fp32 matrix of rank 0 .. ranks-1
+ *              as addressable from the calling GPU (H_ranks[rank] is the caller's own), 16-byte aligned
+ *   ranks      1 <= ranks <= 16 (1: both calls are no-ops)
+ *   rank       0 <= rank < ranks
+ * The kernels run on `stream` of the current device.  Passing the same set of matrices and every rank in turn
+ * from one GPU is valid as well (all "ranks" in one address space).
+ */
+int32_t gq_hessian_reduce_share(float *const *H_ranks, int32_t ranks, int32_t rank, int64_t d_in, int32_t g,
+                                void *stream);
+int32_t gq_hessian_gather_shares(float *const *H_ranks, int32_t ranks, int32_t rank, int64_t d_in, int32_t g,
+                                 void *stream);
+
+/*
  * Objective, Eq. 7:
  *     loss_out[k] = sum_{j in J_k} (w_j - what_j)^T H_k (w_j - what_j),  k < g
  *     loss_out[g] = sum_k loss_out[k]
@@ -280,7 +309,8 @@ enum gq_kernel_id {
     GQ_KERNEL_CB_GEMM = 10,    /* codebook step: tensor-core products H W^T and H [P ...] */
     GQ_KERNEL_CB_FOLD = 11,    /* codebook step: sums over the rows of each level, m x m solves */
     GQ_KERNEL_CB_AUX = 12,     /* codebook step: splits, transposes, one-hot columns, W_hat */
-    GQ_KERNEL_COUNT = 13
+    GQ_KERNEL_EXCHANGE = 13,   /* token-sharded accumulation: reduce / gather of blocks of H over peer memory */
+    GQ_KERNEL_COUNT = 14
 };
 
 /*

@@ -24,10 +24,11 @@ EXPORTS = (
     "gq_layer_objective_host", "gq_layer_host_arena_bytes", "gq_check", "gq_launch_count",
     "gq_kernel_timing_enable", "gq_kernel_timing_read", "gq_objective_noalloc", "gq_cd_cycles", "gq_cd_workspace_bytes",
     "gq_selftest_wait_timeout", "gq_codebook_update", "gq_codebook_workspace_bytes",
+    "gq_hessian_reduce_share", "gq_hessian_gather_shares",
 )
 GQ_HESSIAN_DETERMINISTIC = 1      # flag of gq_hessian_accumulate: single writer per element of H
 KERNEL_NAMES = ("saliency", "hessian", "mirror", "split_delta", "gram_dot", "reduce", "split_saliency", "cd_panel",
-                "cd_block", "cd_aux", "cb_gemm", "cb_fold", "cb_aux")
+                "cd_block", "cd_aux", "cb_gemm", "cb_fold", "cb_aux", "exchange")
 
 
 class GQError(RuntimeError):
@@ -64,6 +65,9 @@ def lib() -> ctypes.CDLL:
         L.gq_hessian_accumulate.argtypes = [vp, i64, i64, i64, vp, i64, i32, vp, u32, vp, sz, vp]
         L.gq_hessian_finalize.restype = i32
         L.gq_hessian_finalize.argtypes = [vp, i64, i32, vp]
+        for f in (L.gq_hessian_reduce_share, L.gq_hessian_gather_shares):
+            f.restype = i32
+            f.argtypes = [ctypes.POINTER(ctypes.c_void_p), i32, i32, i64, i32, vp]
         L.gq_objective_workspace_bytes.restype = sz
         L.gq_objective_workspace_bytes.argtypes = [i64, i64, i32]
         L.gq_objective.restype = i32
@@ -181,6 +185,36 @@ def gq_hessian_finalize(H: torch.Tensor, stream=None) -> torch.Tensor:
     if rc:
         raise GQError("gq_hessian_finalize", rc)
     return H
+
+
+def _rank_pointers(H_ranks, d_in: int, g: int):
+    ptrs = []
+    for h in H_ranks:
+        if isinstance(h, torch.Tensor):
+            _dev(h, torch.float32, "H_ranks[i]")
+            if tuple(h.shape) != (g, d_in, d_in) or not h.is_contiguous():
+                raise ValueError("every H must be a contiguous [g, d_in, d_in] tensor")
+            ptrs.append(h.data_ptr())
+        else:
+            ptrs.append(int(h))           # a peer's device pointer as mapped into this process
+    return (ctypes.c_void_p * len(ptrs))(*ptrs)
+
+
+def gq_hessian_reduce_share(H_ranks, rank: int, d_in: int, g: int, stream=None) -> None:
+    """Token-sharded accumulation, step 1: add rank ``rank``'s blocks of the upper triangle over all ranks'
+    matrices (tensors of this process, or peers' device pointers as integers) into ``H_ranks[rank]``."""
+    arr = _rank_pointers(H_ranks, d_in, g)
+    rc = lib().gq_hessian_reduce_share(arr, len(arr), rank, d_in, g, _stream_ptr(stream))
+    if rc:
+        raise GQError("gq_hessian_reduce_share", rc)
+
+
+def gq_hessian_gather_shares(H_ranks, rank: int, d_in: int, g: int, stream=None) -> None:
+    """Token-sharded accumulation, step 2: copy the other ranks' reduced blocks into ``H_ranks[rank]``."""
+    arr = _rank_pointers(H_ranks, d_in, g)
+    rc = lib().gq_hessian_gather_shares(arr, len(arr), rank, d_in, g, _stream_ptr(stream))
+    if rc:
+        raise GQError("gq_hessian_gather_shares", rc)
 
 
 def gq_objective_workspace_bytes(d_in: int, d_out: int, g: int) -> int:

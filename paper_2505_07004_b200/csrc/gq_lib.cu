@@ -17,6 +17,7 @@
 #include "gq_objective.cuh"
 #include "gq_cd.cuh"
 #include "gq_codebook.cuh"
+#include "gq_exchange.cuh"
 #include "gq_kernels.cuh"
 
 #define GQ_VERSION_NUMBER 100   /* 0.1.0 */
@@ -440,6 +441,52 @@ int32_t gq_hessian_finalize(float *H, int64_t d_in, int32_t g, void *stream)
     }
     GQ_CUDA(cudaGetLastError());
     return GQ_OK;
+}
+
+static int32_t hessian_exchange(float *const *H_ranks, int32_t ranks, int32_t rank, int64_t d_in, int32_t g,
+                                void *stream, bool reduce)
+{
+    if (!H_ranks || ranks < 1 || ranks > gq::EX_MAX_RANKS || rank < 0 || rank >= ranks) return GQ_ERR_INVALID_ARG;
+    if (int32_t rc = check_layer_shape(d_in, 0, g, false)) return rc;
+    gq::ExchangeParams p{};
+    for (int32_t r = 0; r < ranks; ++r) {
+        if (!H_ranks[r]) return GQ_ERR_INVALID_ARG;
+        if (!aligned(H_ranks[r], 16)) return GQ_ERR_ALIGNMENT;
+        p.H[r] = H_ranks[r];
+    }
+    if (ranks == 1) return GQ_OK;
+    p.ranks = ranks;
+    p.rank = rank;
+    p.d = static_cast<int>(d_in);
+    p.g = g;
+    p.nb = static_cast<int>((d_in + gq::EX_BLOCK - 1) / gq::EX_BLOCK);
+    p.blocks = static_cast<long long>(g) * p.nb * (p.nb + 1) / 2;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    long long first = 0, count = p.blocks;
+    if (reduce) {
+        first = gq::exchange_share_begin(p.blocks, ranks, rank);
+        count = gq::exchange_share_begin(p.blocks, ranks, rank + 1) - first;
+    }
+    if (count <= 0) return GQ_OK;
+    {
+        LaunchScope scope(GQ_KERNEL_EXCHANGE, st);
+        if (reduce)
+            gq::exchange_kernel<true><<<static_cast<unsigned>(count), 256, 0, st>>>(p, first);
+        else
+            gq::exchange_kernel<false><<<static_cast<unsigned>(count), 256, 0, st>>>(p, first);
+    }
+    GQ_CUDA(cudaGetLastError());
+    return GQ_OK;
+}
+
+int32_t gq_hessian_reduce_share(float *const *H_ranks, int32_t ranks, int32_t rank, int64_t d_in, int32_t g, void *stream)
+{
+    return hessian_exchange(H_ranks, ranks, rank, d_in, g, stream, true);
+}
+
+int32_t gq_hessian_gather_shares(float *const *H_ranks, int32_t ranks, int32_t rank, int64_t d_in, int32_t g, void *stream)
+{
+    return hessian_exchange(H_ranks, ranks, rank, d_in, g, stream, false);
 }
 
 size_t gq_objective_workspace_bytes(int64_t d_in, int64_t d_out, int32_t g)

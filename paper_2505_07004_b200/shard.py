@@ -1,6 +1,12 @@
-"""Multi-GPU plumbing: the path shards over independent layers, one per rank, with no data-path
-collective (the paper computes Hessians of different layers / groups on different GPUs, Section 3.2 and
-Appendix C).  The only communication is the reduction of timings and of per-rank scalar results."""
+"""Multi-GPU plumbing.
+
+Default: the path shards over independent layers, one per rank, with no data-path collective (the paper
+computes Hessians of different layers / groups on different GPUs, Section 3.2 and Appendix C); the only
+communication is the reduction of timings and of per-rank scalar results.
+
+Token sharding of ONE layer (H_k is a sum over tokens, Algorithm 1 line 4): every rank accumulates the chunks
+`chunks_for_rank` gives it into its own H, then `exchange_hessian` adds the partial matrices with the library's
+reduce / gather kernels over peer memory, the ranks meeting at host barriers in between."""
 from __future__ import annotations
 
 from typing import Sequence
@@ -35,3 +41,39 @@ def gather_scalars(value: float, device="cpu") -> list:
 def whole_job_throughput(units_per_rank: int, steps: int, max_seconds: float, world: int) -> float:
     """Units all ranks processed divided by the slowest rank's time."""
     return float(units_per_rank) * world * steps / max_seconds
+
+
+def chunks_for_rank(n_chunks: int, rank: int, world: int) -> list:
+    """Token chunks of one layer that rank `rank` accumulates (round-robin: every chunk exactly once)."""
+    return list(range(int(rank), int(n_chunks), int(world)))
+
+
+def allocate_symmetric_hessian(g: int, d_in: int, device, group=None):
+    """H of this rank in memory every rank of `group` can address, zeroed, and all ranks' pointers to it
+    (index = rank) as this process sees them."""
+    import torch.distributed._symmetric_memory as symm_mem
+    H = symm_mem.empty((g, d_in, d_in), dtype=torch.float32, device=device)
+    H.zero_()
+    handle = symm_mem.rendezvous(H, group=group if group is not None else dist.group.WORLD)
+    return H, [int(p) for p in handle.buffer_ptrs]
+
+
+def exchange_hessian(H: torch.Tensor, rank_ptrs: Sequence, rank: int, group=None) -> torch.Tensor:
+    """After every rank has accumulated its chunks into its H: make every rank's H the full sum and complete
+    it (finalize).  `rank_ptrs[r]` is rank r's H as addressable from this GPU (`rank_ptrs[rank]` is `H`)."""
+    from . import api
+    g, d_in = int(H.shape[0]), int(H.shape[1])
+
+    def meet():
+        torch.cuda.current_stream().synchronize()
+        if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+            dist.barrier(group)
+
+    if len(rank_ptrs) > 1:
+        meet()                                            # all partial matrices are complete
+        api.gq_hessian_reduce_share(rank_ptrs, rank, d_in, g)
+        meet()                                            # all shares are reduced
+        api.gq_hessian_gather_shares(rank_ptrs, rank, d_in, g)
+        meet()                                            # nobody reads this rank's H any more
+    api.gq_hessian_finalize(H)
+    return H

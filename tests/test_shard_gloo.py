@@ -44,3 +44,49 @@ def test_two_rank_timing_reduction_and_distinct_layers(tmp_path):
 def test_single_process_fallbacks():
     assert shard.max_over_ranks([1.5, 2.5]) == [1.5, 2.5]
     assert shard.gather_scalars(3.0) == [3.0]
+
+
+def _token_worker(rank, world, port, out_dir):
+    """Token sharding of one layer: every rank sums the oracle's partial Hessians of its chunks; adding the
+    partial matrices over the ranks (here: gloo all-reduce, on the GPUs: the library's exchange kernels) must
+    give the Hessian of all tokens."""
+    import numpy as np
+    from oracle import gq_oracle as orc
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        cfg = synth.LayerConfig("t", 5 * 32 + 7, 32, 24, 16, (2,), "lognormal", 0.05, 20.0)
+        syn = synth.LayerSynth(cfg, "cpu", seed=3)                      # the same layer on every rank
+        H = np.zeros((2, cfg.d_in, cfg.d_in))
+        mine = shard.chunks_for_rank(cfg.n_chunks, rank, world)
+        for c in mine:
+            xb, gb = synth.bf16_bits(syn.x_chunk(c)), synth.bf16_bits(syn.grad_chunk(c))
+            orc.hessian(xb, orc.saliency(gb, 2, 1.0), H)
+        t = torch.from_numpy(H)
+        dist.all_reduce(t)
+        torch.save({"H": t, "mine": mine}, os.path.join(out_dir, "t%d.pt" % rank))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_rank_token_sharding_adds_up(tmp_path):
+    import numpy as np
+    from oracle import gq_oracle as orc
+    world, port = 2, _free_port()
+    mp.spawn(_token_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    r = [torch.load(os.path.join(tmp_path, "t%d.pt" % i)) for i in range(world)]
+    assert sorted(r[0]["mine"] + r[1]["mine"]) == list(range(6))
+    cfg = synth.LayerConfig("t", 5 * 32 + 7, 32, 24, 16, (2,), "lognormal", 0.05, 20.0)
+    syn = synth.LayerSynth(cfg, "cpu", seed=3)
+    xb = np.concatenate([synth.bf16_bits(syn.x_chunk(c)) for c in range(cfg.n_chunks)])
+    gb = np.concatenate([synth.bf16_bits(syn.grad_chunk(c)) for c in range(cfg.n_chunks)])
+    H_all = orc.hessian(xb, orc.saliency(gb, 2, 1.0))
+    for i in range(world):
+        assert np.allclose(r[i]["H"].numpy(), H_all, rtol=1e-12, atol=1e-14 * np.abs(H_all).max())
+
+
+def test_chunks_for_rank_partitions():
+    for n_chunks in (0, 1, 5, 16):
+        for world in (1, 2, 3, 8):
+            got = sorted(c for r in range(world) for c in shard.chunks_for_rank(n_chunks, r, world))
+            assert got == list(range(n_chunks))
