@@ -269,9 +269,11 @@ int32_t gq_check(void *stream, uint32_t *detail /* HOST, may be NULL */);
  *   W_hat      fp32 [d_out, d_in] or NULL; out: W_hat[j][i] = codebook[j][Q[j][i]]
  *   workspace  device scratch of at least gq_codebook_workspace_bytes(d_in, d_out, g, m) bytes, 1024-byte aligned
  * Same shape rules as gq_objective.
- * Arithmetic: H_k W_k^T and H_k [P^(j) ...] are formed on the tensor cores with H as three bf16 terms that
- * sum to the fp32 value exactly (the one-hot columns are exact, W is carried to 24 bits as well), fp32
- * accumulation; the sums over the rows of each level and the m x m Cholesky solves are fp64.
+ * Arithmetic: H_k W_k^T and H_k [P^(j) ...] are formed on the tensor cores, fp32 accumulation.  H and W are
+ * split into three bf16 terms each that sum to the fp32 value exactly; H_k W_k^T takes the six products of
+ * total order <= 2, H_k [P^(j) ...] (one-hot columns, exact in bf16) the two leading terms of H (16 mantissa
+ * bits; what is dropped is of the size of the fp32 accumulation error).  The sums over the rows of each level
+ * and the m x m Cholesky solves are fp64.
  * Together with gq_cd_cycles and gq_objective this is Algorithm 2: repeat { gq_codebook_update (with W_hat);
  * gq_cd_cycles } T times, then gq_codebook_update once more.
  */
@@ -280,6 +282,27 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
                            void *workspace, size_t workspace_bytes, void *stream);
 
 size_t gq_codebook_workspace_bytes(int64_t d_in, int64_t d_out, int32_t g, int32_t m);
+
+/*
+ * The layer-wise non-uniform quantiser, Algorithm 2, as one call: starting from the assignment Q,
+ *     repeat T times { codebook step (Eq. 8) ; K cycles of coordinate descent (Eq. 10) } ; codebook step
+ * i.e. exactly the sequence of gq_codebook_update and gq_cd_cycles calls described above, enqueued on `stream`
+ * without any host synchronisation in between.
+ *
+ *   W          fp32 [d_out, d_in], 16-byte aligned
+ *   Q          uint8 [d_out, d_in], in: the initial assignment (codes < m), out: the final one
+ *   m          1 <= m <= 16;   T >= 0 rounds;   K >= 0 cycles per round;   lambda >= 0 (the paper: 1e-7)
+ *   H          fp32 [g, d_in, d_in], full symmetric matrices (after gq_hessian_finalize), 16-byte aligned
+ *   codebook   fp32 [d_out, m], out
+ *   W_hat      fp32 [d_out, d_in], out: codebook[j][Q[j][i]], 16-byte aligned
+ *   workspace  device scratch of at least gq_lnq_workspace_bytes(d_in, d_out, g, m) bytes, 1024-byte aligned
+ * No step increases any channel's objective (Proposition 1 and the optimality of Eq. 8), up to rounding.
+ */
+int32_t gq_lnq(const float *W, uint8_t *Q, int32_t m, int64_t d_in, int64_t d_out, const float *H, int32_t g,
+               int32_t T, int32_t K, double lambda, float *codebook, float *W_hat, void *workspace,
+               size_t workspace_bytes, void *stream);
+
+size_t gq_lnq_workspace_bytes(int64_t d_in, int64_t d_out, int32_t g, int32_t m);
 
 /*
  * Self-test of the device-side failure detection (no counterpart in the paper): launches a one-warp kernel

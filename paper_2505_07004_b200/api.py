@@ -24,7 +24,7 @@ EXPORTS = (
     "gq_layer_objective_host", "gq_layer_host_arena_bytes", "gq_check", "gq_launch_count",
     "gq_kernel_timing_enable", "gq_kernel_timing_read", "gq_objective_noalloc", "gq_cd_cycles", "gq_cd_workspace_bytes",
     "gq_selftest_wait_timeout", "gq_codebook_update", "gq_codebook_workspace_bytes",
-    "gq_hessian_reduce_share", "gq_hessian_gather_shares",
+    "gq_hessian_reduce_share", "gq_hessian_gather_shares", "gq_lnq", "gq_lnq_workspace_bytes",
 )
 GQ_HESSIAN_DETERMINISTIC = 1      # flag of gq_hessian_accumulate: single writer per element of H
 KERNEL_NAMES = ("saliency", "hessian", "mirror", "split_delta", "gram_dot", "reduce", "split_saliency", "cd_panel",
@@ -88,6 +88,10 @@ def lib() -> ctypes.CDLL:
         L.gq_codebook_workspace_bytes.argtypes = [i64, i64, i32, i32]
         L.gq_codebook_update.restype = i32
         L.gq_codebook_update.argtypes = [vp, vp, i32, i64, i64, vp, i32, ctypes.c_double, vp, vp, vp, sz, vp]
+        L.gq_lnq_workspace_bytes.restype = sz
+        L.gq_lnq_workspace_bytes.argtypes = [i64, i64, i32, i32]
+        L.gq_lnq.restype = i32
+        L.gq_lnq.argtypes = [vp, vp, i32, i64, i64, vp, i32, i32, i32, ctypes.c_double, vp, vp, vp, sz, vp]
         L.gq_selftest_wait_timeout.restype = i32
         L.gq_selftest_wait_timeout.argtypes = [i32, vp]
         L.gq_kernel_timing_enable.restype = i32
@@ -367,6 +371,33 @@ def gq_selftest_wait_timeout(budget_ms: int = 20, stream=None) -> None:
 
 def gq_codebook_workspace_bytes(d_in: int, d_out: int, g: int, m: int) -> int:
     return int(lib().gq_codebook_workspace_bytes(d_in, d_out, g, m))
+
+
+def gq_lnq_workspace_bytes(d_in: int, d_out: int, g: int, m: int) -> int:
+    return int(lib().gq_lnq_workspace_bytes(d_in, d_out, g, m))
+
+
+def gq_lnq(W: torch.Tensor, Q: torch.Tensor, m: int, H: torch.Tensor, T: int, K: int, workspace: torch.Tensor,
+           lam: float = 1e-7, stream=None):
+    """Algorithm 2 in one call: ``T`` rounds of (codebook step, ``K`` CD cycles) and a final codebook step,
+    starting from the assignment ``Q`` (uint8, updated in place).  Returns ``(W_hat, Q, codebook)``."""
+    _dev(W, torch.float32, "W")
+    _dev(Q, torch.uint8, "Q")
+    _dev(H, torch.float32, "H")
+    if W.dim() != 2 or W.shape != Q.shape or not W.is_contiguous() or not Q.is_contiguous():
+        raise ValueError("W and Q must be contiguous [d_out, d_in]")
+    d_out, d_in = W.shape
+    g = H.shape[0]
+    if tuple(H.shape) != (g, d_in, d_in) or not H.is_contiguous():
+        raise ValueError("H must be a contiguous [g, d_in, d_in] tensor")
+    codebook = torch.empty((d_out, max(int(m), 1)), dtype=torch.float32, device=W.device)
+    W_hat = torch.empty_like(W)
+    rc = lib().gq_lnq(W.data_ptr(), Q.data_ptr(), int(m), d_in, d_out, H.data_ptr(), g, int(T), int(K), float(lam),
+                  codebook.data_ptr(), W_hat.data_ptr(), workspace.data_ptr(),
+                  workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc:
+        raise GQError("gq_lnq", rc)
+    return W_hat, Q, codebook
 
 
 def gq_codebook_update(W: torch.Tensor, Q: torch.Tensor, m: int, H: torch.Tensor, workspace: torch.Tensor,

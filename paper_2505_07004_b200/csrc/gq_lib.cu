@@ -908,6 +908,36 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
     return GQ_OK;
 }
 
+size_t gq_lnq_workspace_bytes(int64_t d_in, int64_t d_out, int32_t g, int32_t m)
+{
+    const size_t cb = gq_codebook_workspace_bytes(d_in, d_out, g, m);
+    const size_t cd = gq_cd_workspace_bytes(d_in, d_out, g);
+    if (cb == 0 || cd == 0) return 0;
+    return cb > cd ? cb : cd;                     // the two steps alternate: one region serves both
+}
+
+int32_t gq_lnq(const float *W, uint8_t *Q, int32_t m, int64_t d_in, int64_t d_out, const float *H, int32_t g,
+               int32_t T, int32_t K, double lambda, float *codebook, float *W_hat, void *workspace,
+               size_t workspace_bytes, void *stream)
+{
+    if (!W || !Q || !H || !codebook || !W_hat || T < 0 || K < 0) return GQ_ERR_INVALID_ARG;
+    const size_t need = gq_lnq_workspace_bytes(d_in, d_out, g, m);
+    if (need == 0) {
+        if (int32_t rc = check_layer_shape(d_in, d_out, g, true)) return rc;
+        return (m < 1) ? GQ_ERR_INVALID_ARG : GQ_ERR_UNSUPPORTED_SHAPE;
+    }
+    if (!workspace || workspace_bytes < need) return GQ_ERR_WORKSPACE;
+    for (int32_t t = 0; t < T; ++t) {
+        if (int32_t rc = gq_codebook_update(W, Q, m, d_in, d_out, H, g, lambda, codebook, W_hat, workspace,
+                                            workspace_bytes, stream))
+            return rc;
+        if (K == 0) continue;
+        if (int32_t rc = gq_cd_cycles(W, W_hat, Q, codebook, m, d_in, d_out, H, g, K, workspace, workspace_bytes, stream))
+            return rc;
+    }
+    return gq_codebook_update(W, Q, m, d_in, d_out, H, g, lambda, codebook, W_hat, workspace, workspace_bytes, stream);
+}
+
 int32_t gq_selftest_wait_timeout(int32_t budget_ms, void *stream)
 {
     if (budget_ms < 1 || budget_ms > 1000) return GQ_ERR_INVALID_ARG;

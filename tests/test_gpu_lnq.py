@@ -194,3 +194,40 @@ def test_full_size_layer_sampled_channels(dev):
         assert np.abs(cb3_h[j] - c_o).max() <= C_RTOL * np.abs(c_o).max()
     print("sampled channels on a near-tie path: %d of %d" % (n_tie, len(sel)))
     assert n_tie <= len(sel) // 2
+
+
+def test_gq_lnq_is_the_sequence_of_its_steps(dev):
+    """gq_lnq (Algorithm 2 as one call) must give bit for bit what the separate calls give, and land where the
+    oracle's LNQ lands (objective per group within 2 %, see test_lnq_loop_descends_like_the_oracle)."""
+    d_in, d_out, g, m, T, K = 640, 256, 2, 8, 2, 2
+    W, W0, Q0, cb0, H = make_problem(21, d_in, d_out, g, m)
+    Wd, Hd = torch.from_numpy(W).to(dev), torch.from_numpy(H).to(dev)
+    ws = libgq.alloc_workspace(libgq.gq_lnq_workspace_bytes(d_in, d_out, g, m), dev)
+    assert ws.numel() == max(libgq.gq_codebook_workspace_bytes(d_in, d_out, g, m), libgq.gq_cd_workspace_bytes(d_in, d_out, g))
+    What1, Q1, cb1 = libgq.gq_lnq(Wd, torch.from_numpy(Q0.astype(np.uint8)).to(dev), m, Hd, T, K, ws)
+    libgq.gq_check()
+    Q = torch.from_numpy(Q0.astype(np.uint8)).to(dev)
+    What = torch.empty_like(Wd)
+    for _ in range(T):
+        cb, What = libgq.gq_codebook_update(Wd, Q, m, Hd, ws, W_hat=What)
+        What, Q = libgq.gq_cd_cycles(Wd, What, cb, Hd, K, ws, Q=Q)
+    cb, What = libgq.gq_codebook_update(Wd, Q, m, Hd, ws, W_hat=What)
+    libgq.gq_check()
+    assert torch.equal(Q1, Q) and torch.equal(cb1, cb) and torch.equal(What1, What)
+    What_o, Q_o, cb_o = cdo.lnq(W, Q0, H, m, T=T, K=K)
+    mk = d_out // g
+    tg = per_channel_objective(W, What1.cpu().numpy(), H).reshape(g, mk).sum(1)
+    to = per_channel_objective(W, What_o, H).reshape(g, mk).sum(1)
+    assert np.all(np.abs(tg - to) <= 2e-2 * to)
+    # K = 0: only codebook steps, the assignment is untouched
+    What0, Qk, cbk = libgq.gq_lnq(Wd, torch.from_numpy(Q0.astype(np.uint8)).to(dev), m, Hd, 3, 0, ws)
+    assert np.array_equal(Qk.cpu().numpy(), Q0.astype(np.uint8))
+    cb_first, _ = libgq.gq_codebook_update(Wd, Qk, m, Hd, ws)
+    assert torch.equal(cbk, cb_first)
+    with pytest.raises(libgq.GQError) as e:
+        libgq.gq_lnq(Wd, Qk, m, Hd, 1, 1, ws[:4096])
+    assert "GQ_ERR_WORKSPACE" in str(e.value)
+    with pytest.raises(libgq.GQError):
+        libgq.gq_lnq(Wd, Qk, 17, Hd, 1, 1, ws)
+    with pytest.raises(libgq.GQError):
+        libgq.gq_lnq(Wd, Qk, m, Hd, -1, 1, ws)
