@@ -142,6 +142,16 @@ def run_reference(args, cfg, g):
     from oracle import gq_oracle as orc
     orc.build()
     tokens, cpg = args.ref_tokens, args.ref_channels
+    if tokens <= 0:
+        # Size the per-step sample so that the whole run (warm-up + steps) takes about two minutes of oracle
+        # time: one untimed calibration pass on 64 tokens and 16 channels per group, cost taken as linear in both.
+        t0 = time.perf_counter()
+        oracle_sample(cfg, g, 64, 16)
+        t_cal = max(time.perf_counter() - t0, 1e-3)
+        per_step = 120.0 / max(1, args.steps + args.warmup)
+        scale = per_step / t_cal
+        tokens = int(min(1024, max(32, 64 * scale)) // 32 * 32)
+        cpg = int(min(64, max(8, 16 * scale)) // 8 * 8)
     for _ in range(args.warmup):
         oracle_sample(cfg, g, tokens, cpg)
     t0 = time.perf_counter()
@@ -324,7 +334,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-tokens", type=int, default=4096)
     ap.add_argument("--cpu-channels", type=int, default=128)
-    ap.add_argument("--ref-tokens", type=int, default=256)
+    ap.add_argument("--ref-tokens", type=int, default=0,
+                    help="tokens per step of the reference arm (0: sized so that the run takes about two minutes)")
     ap.add_argument("--ref-channels", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
