@@ -304,6 +304,12 @@ def run_ours(args, cfg, g):
                          "flops_per_launch": flops_per_launch, "ms_per_launch": ga_ms / max(1, ga_n)},
             "saliency_hbm": {"achieved_gbs": (sal_bytes / (sal_ms / max(1, sal_n) * 1e-3) / 1e9) if sal_n else None,
                              "peak_gbs": peaks["hbm_gbs"]},
+            "objective": (lambda ms: {
+                "ms_per_call": ms,
+                "tflops_dense_equivalent": 2.0 * cfg.d_in ** 2 * cfg.d_out / (ms * 1e-3) / 1e12,
+                "gbs_algorithmic": (2.0 * g * cfg.d_in * (cfg.d_in + 1) + 8.0 * cfg.d_in * cfg.d_out) / (ms * 1e-3) / 1e9,
+            })((kern["split_delta"][0] + kern["gram_dot"][0] + kern["reduce"][0]) / max(1, kern["gram_dot"][1]))
+            if kern["gram_dot"][1] else None,
             "kernels": kernels,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "api": "gq_layer_objective_host (pinned host buffers)"},
