@@ -231,3 +231,40 @@ def test_gq_lnq_is_the_sequence_of_its_steps(dev):
         libgq.gq_lnq(Wd, Qk, 17, Hd, 1, 1, ws)
     with pytest.raises(libgq.GQError):
         libgq.gq_lnq(Wd, Qk, m, Hd, -1, 1, ws)
+
+
+def test_whole_pipeline_guided_hessian_to_quantised_layer(dev):
+    """Everything through the library: saliency -> guided Hessians -> finalize -> LNQ -> objective.  The
+    objective the library reports for the quantised layer must match the oracle's evaluation (Eq. 7) on the
+    oracle's own Hessians, and LNQ must have lowered it below nearest-level rounding to a uniform grid."""
+    from oracle import gq_oracle as orc
+    from paper_2505_07004_b200 import synth
+    cfg = synth.LayerConfig("p", 3000, 1024, 512, 256, (2,), "lognormal", 0.02, 20.0)
+    syn = synth.LayerSynth(cfg, dev, seed=9)
+    g, m = 2, 8
+    H = torch.zeros(g, cfg.d_in, cfg.d_in, device=dev)
+    ws = libgq.alloc_workspace(libgq.gq_hessian_workspace_bytes(cfg.chunk, cfg.d_in, g), dev)
+    xb, gb = [], []
+    for c in range(cfg.n_chunks):
+        x, gr = syn.x_chunk(c), syn.grad_chunk(c)
+        xb.append(synth.bf16_bits(x))
+        gb.append(synth.bf16_bits(gr))
+        libgq.gq_hessian_accumulate(x, libgq.gq_saliency(gr, g, 1e3), H, ws)
+    libgq.gq_hessian_finalize(H)
+    W, _ = syn.weights()
+    lo, hi = W.min(1, keepdim=True).values, W.max(1, keepdim=True).values
+    Q0 = ((W - lo) / (hi - lo) * m).floor().clamp_(0, m - 1).to(torch.uint8)
+    W_grid = lo + (hi - lo) * (Q0.float() + 0.5) / m
+    ows = libgq.alloc_workspace(libgq.gq_objective_workspace_bytes(cfg.d_in, cfg.d_out, g), dev)
+    f_grid = libgq.gq_objective(W, W_grid.contiguous(), H, ows).cpu().numpy()
+    lws = libgq.alloc_workspace(libgq.gq_lnq_workspace_bytes(cfg.d_in, cfg.d_out, g, m), dev)
+    What, Q, cb = libgq.gq_lnq(W, Q0.clone(), m, H, 2, 2, lws)
+    f_lnq = libgq.gq_objective(W, What, H, ows).cpu().numpy()
+    libgq.gq_check()
+    assert torch.equal(What, torch.gather(cb, 1, Q.long()))
+    assert np.all(f_lnq[:g] < 0.5 * f_grid[:g])
+    # oracle: its own saliency and Hessians from the same bits, its own objective of the GPU's W_hat
+    s_o = orc.saliency(np.concatenate(gb), g, 1e3)
+    H_o = orc.hessian(np.concatenate(xb), s_o)
+    f_o = orc.objective(W.cpu().numpy(), What.cpu().numpy(), H_o)
+    assert np.all(np.abs(f_lnq - f_o) <= 1e-3 * np.abs(f_o)), (f_lnq, f_o)
