@@ -18,6 +18,7 @@
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <math_constants.h>
 #include <stdint.h>
 
 namespace gq {
@@ -29,7 +30,7 @@ constexpr int CD_THREADS = CD_CH * CD_LANES;
 constexpr int CD_MAX_LEVELS = 16;       // codebook entries per channel (m = 2^b, b <= 4)
 constexpr int CD_TILE_LD = CD_CH + 1;   // padded row of the [CD_BLOCK][CD_CH] shared-memory tiles
 constexpr int CD_HCHUNK = 32;           // rows of the block's Hessian staged at a time
-constexpr int CD_SMEM_BYTES = (3 * CD_BLOCK * CD_TILE_LD + 2 * CD_HCHUNK * CD_BLOCK + CD_BLOCK) * 4 + CD_BLOCK * CD_CH;
+constexpr int CD_SMEM_BYTES = (3 * CD_BLOCK * CD_TILE_LD + 2 * CD_HCHUNK * CD_BLOCK + CD_BLOCK + 2 * CD_CH * CD_MAX_LEVELS) * 4;
 
 __device__ __forceinline__ void split_bf16(float v, __nv_bfloat16 &hi, __nv_bfloat16 &lo)
 {
@@ -129,12 +130,17 @@ struct CdBlockParams {
 };
 
 // One block of coordinates for CD_CH channels of one group.  Eight threads share a channel; thread l of
-// them owns the rows 32 t + 4 l + e (t < 8, e < 4) of the running sums
+// them owns the rows 32 t + 4 l + e (band t < 8, e < 4) of the running sums
 //     Bu[r] = sum_{c != r} H[r][c] * E_c      (current E: this cycle's values for c < r, last cycle's for c > r).
-// Pass 1 adds the in-block part of last cycle's values (c > r), pass 2 walks the rows in order: the owner of
-// row i hands W_i - Bu[i] / H_ii to its seven neighbours, the eight of them find the nearest codebook level
-// (ties to the smaller index), and every thread adds H[i][r] * E_i to its rows r > i.  H[i][.] rows come
-// through shared memory in chunks of 32.
+// Pass 1 adds the in-block part of last cycle's values (c > r).  Pass 2 walks the rows in order; per row i:
+//   * the owner hands the rounding target W_i - Bu[i] / H_ii to the channel's threads (one shuffle);
+//   * Round_j: the channel's levels are kept sorted, thread l holding the thresholds between the sorted levels
+//     2l, 2l+1 and 2l+1, 2l+2 (their midpoints, lowered by one ulp where the upper level has the smaller
+//     original index, so that an exact tie goes to the smaller index); the nearest level is at sorted position
+//     #{q : target > thr_q}: two compares and two warp votes per thread, one table read;
+//   * every thread adds H[i][r] * E_i to those of its rows that come after i.
+// H[i][.] rows come through shared memory in chunks of 32 (= one band).  The codes are recovered at the end as
+// the first level, in the codebook's given order, that equals the chosen value.
 __global__ void __launch_bounds__(CD_THREADS, 1)
 cd_block_kernel(const CdBlockParams p)
 {
@@ -144,13 +150,15 @@ cd_block_kernel(const CdBlockParams p)
     float *Xs = Es + CD_BLOCK * CD_TILE_LD;              // first P (pulled sums), then What of the block
     float *Hs = Xs + CD_BLOCK * CD_TILE_LD;              // [2][CD_HCHUNK][CD_BLOCK]
     float *rds = Hs + 2 * CD_HCHUNK * CD_BLOCK;          // [CD_BLOCK]
-    uint8_t *Qs = reinterpret_cast<uint8_t *>(rds + CD_BLOCK);   // [CD_BLOCK][CD_CH]
+    float *cbs = rds + CD_BLOCK;                         // [CD_CH][CD_MAX_LEVELS] codebooks in their given order
+    float *srt = cbs + CD_CH * CD_MAX_LEVELS;            // [CD_CH][CD_MAX_LEVELS] the same, sorted
 
     const int tid = threadIdx.x;
     const int k = blockIdx.x / p.slices;
     const int ch0 = k * p.mk + (blockIdx.x % p.slices) * CD_CH;          // first channel of this CTA
     const int ch_n = min(CD_CH, (k + 1) * p.mk - ch0);                   // valid channels
     const int cidx = tid / CD_LANES, l = tid % CD_LANES;
+    const int group_shift = 8 * ((tid >> 3) & 3);                       // where this channel's eight threads sit in a warp vote
     const float *Hk = p.H + static_cast<size_t>(k) * p.d_in * p.d_in;
 
     // ---- tiles in: 32 channels x 256 coordinates, coalesced over channels
@@ -184,10 +192,39 @@ cd_block_kernel(const CdBlockParams p)
     };
     auto h_chunk_wait = [&]() { asm volatile("cp.async.wait_group 0;" ::: "memory"); };
 
-    // codebook levels l and l + 8 of this thread's channel (the eight threads of a channel hold all sixteen)
+    // ---- the channel's levels: given order (cbs), sorted (srt), this thread's two thresholds
     static_assert(CD_MAX_LEVELS == 2 * CD_LANES, "two codebook levels per thread");
-    const float cb0 = (l < p.m && cidx < ch_n) ? p.codebook[static_cast<size_t>(ch0 + cidx) * p.m + l] : 0.0f;
-    const float cb1 = (l + 8 < p.m && cidx < ch_n) ? p.codebook[static_cast<size_t>(ch0 + cidx) * p.m + l + 8] : 0.0f;
+    float thr_a = CUDART_INF_F, thr_b = CUDART_INF_F;
+    {
+        const bool chan = cidx < ch_n;
+        const float v0 = (l < p.m && chan) ? p.codebook[static_cast<size_t>(ch0 + cidx) * p.m + l] : CUDART_INF_F;
+        const float v1 = (l + 8 < p.m && chan) ? p.codebook[static_cast<size_t>(ch0 + cidx) * p.m + l + 8] : CUDART_INF_F;
+        int rank0 = 0, rank1 = 0;                        // positions of (v0, l) and (v1, l + 8) among the 16 pairs
+#pragma unroll
+        for (int r = 0; r < CD_MAX_LEVELS; ++r) {
+            const float vr = __shfl_sync(0xffffffffu, r < 8 ? v0 : v1, r & 7, CD_LANES);
+            rank0 += (vr < v0 || (vr == v0 && r < l)) ? 1 : 0;
+            rank1 += (vr < v1 || (vr == v1 && r < l + 8)) ? 1 : 0;
+        }
+        int *sidx = reinterpret_cast<int *>(Hs);         // [CD_CH][CD_MAX_LEVELS] original index by sorted position
+        float *mc = cbs + cidx * CD_MAX_LEVELS, *ms = srt + cidx * CD_MAX_LEVELS;
+        int *mi = sidx + cidx * CD_MAX_LEVELS;
+        mc[l] = v0;
+        mc[l + 8] = v1;
+        ms[rank0] = v0;
+        mi[rank0] = l;
+        ms[rank1] = v1;
+        mi[rank1] = l + 8;
+        __syncwarp();
+        auto threshold = [&](int q) {                    // between sorted levels q and q + 1
+            const float mid = 0.5f * (ms[q] + ms[q + 1]);
+            return (mi[q] < mi[q + 1] || !(fabsf(mid) < CUDART_INF_F)) ? mid : nextafterf(mid, -CUDART_INF_F);
+        };
+        thr_a = threshold(2 * l);
+        if (2 * l + 2 < CD_MAX_LEVELS) thr_b = threshold(2 * l + 1);
+    }
+    const float *my_levels = srt + cidx * CD_MAX_LEVELS;
+    __syncthreads();                                     // sidx (in the H buffer) has been read by everybody
 
     load_h_chunk(0, 0);
     h_chunk_wait();
@@ -238,45 +275,42 @@ cd_block_kernel(const CdBlockParams p)
         if (t + 1 < 8) load_h_chunk((t + 1) * CD_HCHUNK, (t + 1) & 1);
         const float *hc = Hs + (t & 1) * CD_HCHUNK * CD_BLOCK;
 #pragma unroll 1
-        for (int ii = 0; ii < 32; ++ii) {
-            const int i = 32 * t + ii;
-            const int owner = ii >> 2, oe = ii & 3;
-            // the owner of row i forms the rounding target; all eight threads of the channel find the nearest
-            // codebook level together (two levels each, then a three-step minimum; ties: the smaller index)
-            const float bu = oe == 0 ? Bu[t][0] : (oe == 1 ? Bu[t][1] : (oe == 2 ? Bu[t][2] : Bu[t][3]));
-            const float w = Ws[i * CD_TILE_LD + cidx];
-            const float target = __shfl_sync(0xffffffffu, w - rds[i] * bu, owner, CD_LANES);
-            const float d0 = l < p.m ? fabsf(target - cb0) : 3.0e38f;
-            const float d1 = l + 8 < p.m ? fabsf(target - cb1) : 3.0e38f;
-            float bd = d1 < d0 ? d1 : d0;                 // equal distances keep the smaller index l
-            int best = d1 < d0 ? l + 8 : l;
-            float val = d1 < d0 ? cb1 : cb0;
+        for (int i4 = 0; i4 < 32; i4 += 4) {
+            const int owner = i4 >> 2;                    // the thread that owns rows 32 t + i4 .. + 3
+            const bool after = l > owner, mine = l == owner;
+            const float4 h4[4] = {*reinterpret_cast<const float4 *>(hc + (i4 + 0) * CD_BLOCK + 32 * t + 4 * l),
+                                  *reinterpret_cast<const float4 *>(hc + (i4 + 1) * CD_BLOCK + 32 * t + 4 * l),
+                                  *reinterpret_cast<const float4 *>(hc + (i4 + 2) * CD_BLOCK + 32 * t + 4 * l),
+                                  *reinterpret_cast<const float4 *>(hc + (i4 + 3) * CD_BLOCK + 32 * t + 4 * l)};
 #pragma unroll
-            for (int off = 1; off < CD_LANES; off <<= 1) {
-                const float od = __shfl_xor_sync(0xffffffffu, bd, off, CD_LANES);
-                const int ob = __shfl_xor_sync(0xffffffffu, best, off, CD_LANES);
-                const float ov = __shfl_xor_sync(0xffffffffu, val, off, CD_LANES);
-                if (od < bd || (od == bd && ob < best)) { bd = od; best = ob; val = ov; }
-            }
-            const float e_new = val - w;
-            if (l == owner) {
-                Es[i * CD_TILE_LD + cidx] = e_new;
-                Xs[i * CD_TILE_LD + cidx] = val;
-                Qs[i * CD_CH + cidx] = static_cast<uint8_t>(best);
-            }
+            for (int oe = 0; oe < 4; ++oe) {
+                const int i = 32 * t + i4 + oe;
+                const float w = Ws[i * CD_TILE_LD + cidx];
+                const float target = __shfl_sync(0xffffffffu, w - rds[i] * Bu[t][oe], owner, CD_LANES);
+                // the thresholds ascend, so the number of thresholds below the target is the level's position
+                const unsigned below_a = __ballot_sync(0xffffffffu, target > thr_a);
+                const unsigned below_b = __ballot_sync(0xffffffffu, target > thr_b);
+                const int pos = __popc((below_a >> group_shift) & 0xffu) + __popc((below_b >> group_shift) & 0xffu);
+                const float val = my_levels[pos];
+                const float e_new = val - w;
+                if (mine) {
+                    Es[i * CD_TILE_LD + cidx] = e_new;
+                    Xs[i * CD_TILE_LD + cidx] = val;
+                }
+                // same band: only rows after i (a zero factor instead of a branch)
+                const float4 h = h4[oe];
+                const float e_after = after ? e_new : 0.0f, e_from = (after || mine) ? e_new : 0.0f;
+                Bu[t][0] = fmaf(h.x, 0 > oe ? e_from : e_after, Bu[t][0]);
+                Bu[t][1] = fmaf(h.y, 1 > oe ? e_from : e_after, Bu[t][1]);
+                Bu[t][2] = fmaf(h.z, 2 > oe ? e_from : e_after, Bu[t][2]);
+                Bu[t][3] = fmaf(h.w, 3 > oe ? e_from : e_after, Bu[t][3]);
 #pragma unroll
-            for (int tp = t; tp < 8; ++tp) {
-                const float4 h = *reinterpret_cast<const float4 *>(hc + ii * CD_BLOCK + 32 * tp + 4 * l);
-                if (tp > t) {
-                    Bu[tp][0] = fmaf(h.x, e_new, Bu[tp][0]);
-                    Bu[tp][1] = fmaf(h.y, e_new, Bu[tp][1]);
-                    Bu[tp][2] = fmaf(h.z, e_new, Bu[tp][2]);
-                    Bu[tp][3] = fmaf(h.w, e_new, Bu[tp][3]);
-                } else {                                  // same band: only rows after i
-                    if (4 * l + 0 > ii) Bu[tp][0] = fmaf(h.x, e_new, Bu[tp][0]);
-                    if (4 * l + 1 > ii) Bu[tp][1] = fmaf(h.y, e_new, Bu[tp][1]);
-                    if (4 * l + 2 > ii) Bu[tp][2] = fmaf(h.z, e_new, Bu[tp][2]);
-                    if (4 * l + 3 > ii) Bu[tp][3] = fmaf(h.w, e_new, Bu[tp][3]);
+                for (int tp = t + 1; tp < 8; ++tp) {      // later bands: all rows
+                    const float4 hh = *reinterpret_cast<const float4 *>(hc + (i4 + oe) * CD_BLOCK + 32 * tp + 4 * l);
+                    Bu[tp][0] = fmaf(hh.x, e_new, Bu[tp][0]);
+                    Bu[tp][1] = fmaf(hh.y, e_new, Bu[tp][1]);
+                    Bu[tp][2] = fmaf(hh.z, e_new, Bu[tp][2]);
+                    Bu[tp][3] = fmaf(hh.w, e_new, Bu[tp][3]);
                 }
             }
         }
@@ -290,9 +324,14 @@ cd_block_kernel(const CdBlockParams p)
         if (r < p.rows && c < ch_n) {
             const size_t o = static_cast<size_t>(p.s0 + r) * p.d_out + ch0 + c;
             const float e = Es[r * CD_TILE_LD + c];
+            const float val = Xs[r * CD_TILE_LD + c];
+            int code = 0;                                 // first level, in the given order, with this value
+#pragma unroll
+            for (int q = CD_MAX_LEVELS - 1; q >= 0; --q)
+                if (cbs[c * CD_MAX_LEVELS + q] == val) code = q;
             p.Et[o] = e;
-            p.Wht[o] = Xs[r * CD_TILE_LD + c];
-            p.Qt[o] = Qs[r * CD_CH + c];
+            p.Wht[o] = val;
+            p.Qt[o] = static_cast<uint8_t>(code);
             __nv_bfloat16 hi, lo;
             split_bf16(e, hi, lo);
             p.Ehi[o] = hi;
