@@ -269,11 +269,10 @@ int32_t gq_check(void *stream, uint32_t *detail /* HOST, may be NULL */);
  *   W_hat      fp32 [d_out, d_in] or NULL; out: W_hat[j][i] = codebook[j][Q[j][i]]
  *   workspace  device scratch of at least gq_codebook_workspace_bytes(d_in, d_out, g, m) bytes, 1024-byte aligned
  * Same shape rules as gq_objective.
- * Arithmetic: H_k W_k^T and H_k [P^(j) ...] are formed on the tensor cores, fp32 accumulation.  H and W are
- * split into three bf16 terms each that sum to the fp32 value exactly; H_k W_k^T takes the six products of
- * total order <= 2, H_k [P^(j) ...] (one-hot columns, exact in bf16) the two leading terms of H (16 mantissa
- * bits; what is dropped is of the size of the fp32 accumulation error).  The sums over the rows of each level
- * and the m x m Cholesky solves are fp64.
+ * Arithmetic: H_k W_k^T and H_k [P^(j) ...] are formed on the tensor cores, fp32 accumulation, from bf16
+ * hi + lo splits of H and W (16 significant bits per factor; what is dropped is of the size of the fp32
+ * accumulation error; the one-hot columns are exact).  The sums over the rows of each level and the m x m
+ * Cholesky solves are fp64.
  * Together with gq_cd_cycles and gq_objective this is Algorithm 2: repeat { gq_codebook_update (with W_hat);
  * gq_cd_cycles } T times, then gq_codebook_update once more.
  */

@@ -6,10 +6,11 @@
 // The two d_in^2-sized contractions run on the tensor cores (pair_gemm_kernel<MODE_FULL>):
 //     HW = H_k W_k^T                      [d_in x channels]
 //     HP = H_k [P^(j0) ... P^(j0+c-1)]    [d_in x (channels * m)]   for a slab of channels at a time
-// with H split into three bf16 matrices whose sum is the fp32 value exactly (8 + 8 + 8 mantissa bits) and W
-// likewise; accumulation is fp32.  HW takes every product of total order <= 2 (six terms).  HP, where the
-// one-hot columns are exact in bf16, takes the two leading terms of H: what it drops is below 2^-16 of each
-// entry, the size of the fp32 accumulation error of these 4096-long sums, and HP is 16 x the work of HW.
+// with H and W as bf16 hi + lo pairs (16 significant bits, what is dropped is below 2^-16 of each entry: the
+// size of the fp32 accumulation error of these 4096-long sums); accumulation is fp32.  HW takes
+// hi hi + hi lo + lo hi; HP, where the one-hot columns are exact in bf16, the two terms of H.  (Three-way
+// splits that reproduce the fp32 values exactly were measured to change the codebooks by less than the
+// difference to the fp64 oracle that remains either way.)
 // The kernels here prepare those operands, fold HP and HW over the rows of each level (fp64),
 //     G^(j)[q][q'] = sum_{i : Q_ij = q} HP[i][j m + q'],      r^(j)[q] = sum_{i : Q_ij = q} HW[i][j],
 // and solve the m x m systems by Cholesky in fp64.
@@ -23,34 +24,30 @@ namespace gq {
 constexpr int CB_MAX_LEVELS = 16;
 constexpr int CB_SLAB_CHANNELS = 1024;      // channels whose one-hot columns are multiplied at a time
 
-// v = t0 + t1 + t2 exactly (for finite v in bf16 range): three rounds of "round to bf16, subtract".
-__device__ __forceinline__ void split3_bf16(float v, __nv_bfloat16 &t0, __nv_bfloat16 &t1, __nv_bfloat16 &t2)
+// v = t0 + t1 up to 2^-17 |v|: round to bf16, round the remainder to bf16.
+__device__ __forceinline__ void split2_bf16(float v, __nv_bfloat16 &t0, __nv_bfloat16 &t1)
 {
     t0 = __float2bfloat16_rn(v);
-    const float r1 = v - __bfloat162float(t0);
-    t1 = __float2bfloat16_rn(r1);
-    t2 = __float2bfloat16_rn(r1 - __bfloat162float(t1));
+    t1 = __float2bfloat16_rn(v - __bfloat162float(t0));
 }
 
 __global__ void __launch_bounds__(256)
-cb_split3_kernel(const float *__restrict__ src, long long count, __nv_bfloat16 *__restrict__ d0,
-                 __nv_bfloat16 *__restrict__ d1, __nv_bfloat16 *__restrict__ d2)
+cb_split2_kernel(const float *__restrict__ src, long long count, __nv_bfloat16 *__restrict__ d0,
+                 __nv_bfloat16 *__restrict__ d1)
 {
     const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
     for (long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; idx < count; idx += stride) {
-        __nv_bfloat16 a, b, c;
-        split3_bf16(src[idx], a, b, c);
+        __nv_bfloat16 a, b;
+        split2_bf16(src[idx], a, b);
         d0[idx] = a;
         d1[idx] = b;
-        d2[idx] = c;
     }
 }
 
-// W [d_out][d_in] -> three bf16 terms of W^T [d_in][d_out]; Q [d_out][d_in] -> Qt [d_in][d_out].  32 x 32 tiles.
+// W [d_out][d_in] -> bf16 hi + lo of W^T [d_in][d_out]; Q [d_out][d_in] -> Qt [d_in][d_out].  32 x 32 tiles.
 __global__ void __launch_bounds__(256)
 cb_transpose_kernel(const float *__restrict__ W, const uint8_t *__restrict__ Q, int d_in, int d_out,
-                    __nv_bfloat16 *__restrict__ W0, __nv_bfloat16 *__restrict__ W1, __nv_bfloat16 *__restrict__ W2,
-                    uint8_t *__restrict__ Qt)
+                    __nv_bfloat16 *__restrict__ W0, __nv_bfloat16 *__restrict__ W1, uint8_t *__restrict__ Qt)
 {
     __shared__ float tw[32][33];
     __shared__ uint8_t tq[32][33];
@@ -67,11 +64,10 @@ cb_transpose_kernel(const float *__restrict__ W, const uint8_t *__restrict__ Q, 
         const int i = i0 + r, j = j0 + tx;
         if (i < d_in && j < d_out) {
             const size_t o = static_cast<size_t>(i) * d_out + j;
-            __nv_bfloat16 a, b, c;
-            split3_bf16(tw[tx][r], a, b, c);
+            __nv_bfloat16 a, b;
+            split2_bf16(tw[tx][r], a, b);
             W0[o] = a;
             W1[o] = b;
-            W2[o] = c;
             Qt[o] = tq[tx][r];
         }
     }

@@ -262,7 +262,7 @@ ObjectiveLayout objective_layout(int64_t d_in, int64_t d_out, int32_t g)
 }
 
 struct CodebookLayout {
-    size_t h0, h1, h2, w0, w1, w2, qt, hw, pm, hp, gmat, rvec, total;
+    size_t h0, h1, w0, w1, qt, hw, pm, hp, gmat, rvec, total;
     int64_t slab_channels, slab_ld;
 };
 CodebookLayout codebook_layout(int64_t d_in, int64_t d_out, int32_t g, int32_t m)
@@ -276,10 +276,8 @@ CodebookLayout codebook_layout(int64_t d_in, int64_t d_out, int32_t g, int32_t m
     size_t o = 0;
     L.h0 = o; o += h2;
     L.h1 = o; o += h2;
-    L.h2 = o; o += h2;
     L.w0 = o; o += w2;
     L.w1 = o; o += w2;
-    L.w2 = o; o += w2;
     L.qt = o; o += round_up(static_cast<size_t>(d_in) * d_out, 1024);
     L.hw = o; o += round_up(static_cast<size_t>(d_in) * d_out * 4, 1024);
     L.pm = o; o += round_up(static_cast<size_t>(d_in) * L.slab_ld * 2, 1024);
@@ -795,10 +793,8 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
     if (int32_t rc = device_info(&di)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint8_t *ws = static_cast<uint8_t *>(workspace);
-    __nv_bfloat16 *H0 = reinterpret_cast<__nv_bfloat16 *>(ws + L.h0), *H1 = reinterpret_cast<__nv_bfloat16 *>(ws + L.h1),
-                  *H2 = reinterpret_cast<__nv_bfloat16 *>(ws + L.h2);
-    __nv_bfloat16 *W0 = reinterpret_cast<__nv_bfloat16 *>(ws + L.w0), *W1 = reinterpret_cast<__nv_bfloat16 *>(ws + L.w1),
-                  *W2 = reinterpret_cast<__nv_bfloat16 *>(ws + L.w2);
+    __nv_bfloat16 *H0 = reinterpret_cast<__nv_bfloat16 *>(ws + L.h0), *H1 = reinterpret_cast<__nv_bfloat16 *>(ws + L.h1);
+    __nv_bfloat16 *W0 = reinterpret_cast<__nv_bfloat16 *>(ws + L.w0), *W1 = reinterpret_cast<__nv_bfloat16 *>(ws + L.w1);
     uint8_t *Qt = ws + L.qt;
     float *HW = reinterpret_cast<float *>(ws + L.hw);
     __nv_bfloat16 *Pm = reinterpret_cast<__nv_bfloat16 *>(ws + L.pm);
@@ -809,22 +805,20 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
     const long long hcount = static_cast<long long>(g) * d_in * d_in;
     {
         LaunchScope scope(GQ_KERNEL_CB_AUX, st);
-        gq::cb_split3_kernel<<<grid_for(hcount, 256, di->sm_count, 8), 256, 0, st>>>(H, hcount, H0, H1, H2);
+        gq::cb_split2_kernel<<<grid_for(hcount, 256, di->sm_count, 8), 256, 0, st>>>(H, hcount, H0, H1);
     }
     GQ_CUDA(cudaGetLastError());
     {
         const dim3 tgrid(static_cast<unsigned>((d_in + 31) / 32), static_cast<unsigned>((d_out + 31) / 32));
         LaunchScope scope(GQ_KERNEL_CB_AUX, st);
-        gq::cb_transpose_kernel<<<tgrid, 256, 0, st>>>(W, Q, static_cast<int>(d_in), static_cast<int>(d_out), W0, W1, W2, Qt);
+        gq::cb_transpose_kernel<<<tgrid, 256, 0, st>>>(W, Q, static_cast<int>(d_in), static_cast<int>(d_out), W0, W1, Qt);
     }
     GQ_CUDA(cudaGetLastError());
-    CUtensorMap mH0, mH1, mH2, mW0, mW1, mW2, mPm;
+    CUtensorMap mH0, mH1, mW0, mW1, mPm;
     if (int32_t rc = make_map(&mH0, H0, d_in, d_in, g, d_in, d_in * d_in)) return rc;
     if (int32_t rc = make_map(&mH1, H1, d_in, d_in, g, d_in, d_in * d_in)) return rc;
-    if (int32_t rc = make_map(&mH2, H2, d_in, d_in, g, d_in, d_in * d_in)) return rc;
     if (int32_t rc = make_map(&mW0, W0, d_out, d_in, 1, d_out, d_in * d_out)) return rc;
     if (int32_t rc = make_map(&mW1, W1, d_out, d_in, 1, d_out, d_in * d_out)) return rc;
-    if (int32_t rc = make_map(&mW2, W2, d_out, d_in, 1, d_out, d_in * d_out)) return rc;
     if (int32_t rc = make_map(&mPm, Pm, L.slab_ld, d_in, 1, L.slab_ld, d_in * L.slab_ld)) return rc;
 
     auto launch_full = [&](gq::PairGemmParams &pp, const CUtensorMap &b0, const CUtensorMap &b1, const CUtensorMap &b2,
@@ -844,7 +838,7 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
         {
             LaunchScope scope(kernel_id, st);
             gq::pair_gemm_kernel<gq::MODE_FULL><<<2 * pp.sched.pairs, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(
-                mH0, mH1, mH2, b0, b1, b2, pp);
+                mH0, mH1, mH1, b0, b1, b2, pp);
         }
         GQ_CUDA(cudaGetLastError());
         return GQ_OK;
@@ -853,17 +847,17 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
     GQ_CUDA(cudaMemsetAsync(Gm, 0, static_cast<size_t>(d_out) * gq::CB_MAX_LEVELS * gq::CB_MAX_LEVELS * sizeof(double), st));
     GQ_CUDA(cudaMemsetAsync(Rv, 0, static_cast<size_t>(d_out) * gq::CB_MAX_LEVELS * sizeof(double), st));
     for (int32_t k = 0; k < g; ++k) {
-        // HW[:, group k] = H_k W_k^T: terms of total order <= 2 of (H0 + H1 + H2)(W0 + W1 + W2)
+        // HW[:, group k] = H_k W_k^T: H0 W0 + H0 W1 + H1 W0 (hi + lo splits, 16 significant bits per factor)
         gq::PairGemmParams pp{};
-        pp.n_terms = 6;
-        const int ta[6] = {0, 0, 1, 0, 1, 2}, tb[6] = {3, 4, 3, 5, 4, 3};
-        for (int t = 0; t < 6; ++t) { pp.term_a[t] = ta[t]; pp.term_b[t] = tb[t]; }
+        pp.n_terms = 3;
+        const int ta[3] = {0, 0, 1}, tb[3] = {3, 4, 3};
+        for (int t = 0; t < 3; ++t) { pp.term_a[t] = ta[t]; pp.term_b[t] = tb[t]; }
         pp.full_k = k;
         pp.col0 = static_cast<int>(k * mk);
         pp.cols = static_cast<int>(mk);
         pp.C = HW + k * mk;
         pp.ldc = d_out;
-        if (int32_t rc = launch_full(pp, mW0, mW1, mW2, GQ_KERNEL_CB_GEMM)) return rc;
+        if (int32_t rc = launch_full(pp, mW0, mW1, mW1, GQ_KERNEL_CB_GEMM)) return rc;
         for (int64_t j0 = k * mk; j0 < (k + 1) * mk; j0 += L.slab_channels) {
             const int nch = static_cast<int>((k + 1) * mk - j0 < L.slab_channels ? (k + 1) * mk - j0 : L.slab_channels);
             {
