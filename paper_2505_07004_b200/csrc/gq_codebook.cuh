@@ -103,20 +103,23 @@ cb_onehot_kernel(const uint8_t *__restrict__ Qt, int d_in, int d_out, int j0, in
     }
 }
 
-// Fold over the rows of each level.  One CTA = 8 channels of the slab x 16 threads x one of gridDim.y row
-// ranges; thread (ch, q') owns column q' of G^(ch) in shared memory (fp64), so no two threads of a CTA ever add
-// to the same word; thread q' = 0 also owns r.  The row ranges are combined with fp64 atomic adds (the order
-// of at most gridDim.y fp64 partial sums is the only thing that can vary from run to run).
-__global__ void __launch_bounds__(128)
+// Fold over the rows of each level.  One CTA = CB_FOLD_CH channels of the slab x 16 threads x one of gridDim.y
+// row ranges; thread (ch, q') owns column q' of G^(ch) in shared memory, so no two threads of a CTA ever add
+// to the same word; thread q' = 0 also owns r.  Within a row range (a few hundred rows, a few dozen per level)
+// the sums are fp32 and use shared-memory reductions whose results are not read back, so that nothing in the
+// row loop waits for an addition; the row ranges are combined in fp64 with atomic adds (the order of at most
+// gridDim.y fp64 partial sums is the only thing that can vary from run to run).
+constexpr int CB_FOLD_CH = 16;
+__global__ void __launch_bounds__(CB_FOLD_CH * 16)
 cb_fold_kernel(const float *__restrict__ HP, long long ld_hp, const float *__restrict__ HW, const uint8_t *__restrict__ Qt,
                int d_in, int d_out, int j0, int nch, int m, double *__restrict__ G, double *__restrict__ R)
 {
-    __shared__ double Gs[8][CB_MAX_LEVELS][CB_MAX_LEVELS + 1];
-    __shared__ double Rs[8][CB_MAX_LEVELS];
+    __shared__ float Gs[CB_FOLD_CH][CB_MAX_LEVELS][CB_MAX_LEVELS + 1];
+    __shared__ float Rs[CB_FOLD_CH][CB_MAX_LEVELS];
     const int ch = threadIdx.x >> 4, qp = threadIdx.x & 15;
-    const int jj = blockIdx.x * 8 + ch;
-    for (int q = 0; q < CB_MAX_LEVELS; ++q) Gs[ch][q][qp] = 0.0;
-    Rs[ch][qp] = 0.0;
+    const int jj = blockIdx.x * CB_FOLD_CH + ch;
+    for (int q = 0; q < CB_MAX_LEVELS; ++q) Gs[ch][q][qp] = 0.0f;
+    Rs[ch][qp] = 0.0f;
     __syncthreads();
     if (jj < nch && qp < m) {
         const int j = j0 + jj;
@@ -139,8 +142,8 @@ cb_fold_kernel(const float *__restrict__ HP, long long ld_hp, const float *__res
 #pragma unroll
             for (int t = 0; t < BATCH; ++t) {
                 const int qq = q[t] < m ? q[t] : m - 1;  // codes are expected to be < m
-                Gs[ch][qq][qp] += static_cast<double>(v[t]);
-                if (qp == 0) Rs[ch][qq] += static_cast<double>(w[t]);
+                atomicAdd(&Gs[ch][qq][qp], v[t]);
+                if (qp == 0) atomicAdd(&Rs[ch][qq], w[t]);
             }
         }
     }
@@ -148,8 +151,88 @@ cb_fold_kernel(const float *__restrict__ HP, long long ld_hp, const float *__res
     if (jj < nch && qp < m) {                        // G and R were zeroed by the host; row ranges add up
         const int j = j0 + jj;
         for (int q = 0; q < m; ++q)
-            atomicAdd(&G[(static_cast<size_t>(j) * CB_MAX_LEVELS + q) * CB_MAX_LEVELS + qp], Gs[ch][q][qp]);
-        atomicAdd(&R[static_cast<size_t>(j) * CB_MAX_LEVELS + qp], Rs[ch][qp]);
+            atomicAdd(&G[(static_cast<size_t>(j) * CB_MAX_LEVELS + q) * CB_MAX_LEVELS + qp], static_cast<double>(Gs[ch][q][qp]));
+        atomicAdd(&R[static_cast<size_t>(j) * CB_MAX_LEVELS + qp], static_cast<double>(Rs[ch][qp]));
+    }
+}
+
+// The same fold for m a multiple of 4 (the usual 2-, 3- and 4-bit codebooks have m = 4, 8, 16): a thread takes
+// four neighbouring columns q' of one channel with one 16-byte load per row, so the row loop spends its
+// instructions on the data rather than on addresses (the one-column form above is issue-bound).  One CTA =
+// CB_FOLD4_CH channels x 4 threads.
+constexpr int CB_FOLD4_CH = 32;
+__global__ void __launch_bounds__(CB_FOLD4_CH * 4)
+cb_fold4_kernel(const float *__restrict__ HP, long long ld_hp, const float *__restrict__ HW, const uint8_t *__restrict__ Qt,
+                int d_in, int d_out, int j0, int nch, int m, double *__restrict__ G, double *__restrict__ R)
+{
+    __shared__ float Gs[CB_FOLD4_CH][CB_MAX_LEVELS][CB_MAX_LEVELS + 1];
+    __shared__ float Rs[CB_FOLD4_CH][CB_MAX_LEVELS];
+    const int ch = threadIdx.x >> 2, q4 = (threadIdx.x & 3) * 4;
+    const int jj = blockIdx.x * CB_FOLD4_CH + ch;
+    for (int q = 0; q < CB_MAX_LEVELS; ++q)
+        for (int e = 0; e < 4; ++e) Gs[ch][q][q4 + e] = 0.0f;
+    for (int e = 0; e < 4; ++e) Rs[ch][q4 + e] = 0.0f;
+    __syncthreads();
+    const bool active = jj < nch && q4 < m;
+    if (active) {
+        const int j = j0 + jj;
+        constexpr int BATCH = 8;                         // independent loads in flight per thread
+        const int rows_per = (d_in + static_cast<int>(gridDim.y) - 1) / static_cast<int>(gridDim.y);
+        const int i_begin = static_cast<int>(blockIdx.y) * rows_per;
+        const int i_end = i_begin + rows_per < d_in ? i_begin + rows_per : d_in;
+        const float *hp = HP + static_cast<size_t>(i_begin) * ld_hp + static_cast<size_t>(jj) * m + q4;
+        const uint8_t *qt = Qt + static_cast<size_t>(i_begin) * d_out + j;
+        const float *hw = HW + static_cast<size_t>(i_begin) * d_out + j;
+        float *gbase = &Gs[ch][0][q4];
+        int i0 = i_begin;
+        for (; i0 + BATCH <= i_end; i0 += BATCH) {       // whole batches: no row predicates
+            int q[BATCH];
+            float4 v[BATCH];
+            float w[BATCH];
+#pragma unroll
+            for (int t = 0; t < BATCH; ++t) {
+                q[t] = qt[static_cast<size_t>(t) * d_out];
+                v[t] = *reinterpret_cast<const float4 *>(hp + static_cast<size_t>(t) * ld_hp);
+                w[t] = q4 == 0 ? hw[static_cast<size_t>(t) * d_out] : 0.0f;
+            }
+#pragma unroll
+            for (int t = 0; t < BATCH; ++t) {
+                const int qq = q[t] < m ? q[t] : m - 1;  // codes are expected to be < m
+                float *gp = gbase + qq * (CB_MAX_LEVELS + 1);
+                atomicAdd(gp + 0, v[t].x);
+                atomicAdd(gp + 1, v[t].y);
+                atomicAdd(gp + 2, v[t].z);
+                atomicAdd(gp + 3, v[t].w);
+                if (q4 == 0) atomicAdd(&Rs[ch][qq], w[t]);
+            }
+            hp += static_cast<size_t>(BATCH) * ld_hp;
+            qt += static_cast<size_t>(BATCH) * d_out;
+            hw += static_cast<size_t>(BATCH) * d_out;
+        }
+        for (; i0 < i_end; ++i0) {                       // ragged end of the row range
+            const int qr = *qt;
+            const int qq = qr < m ? qr : m - 1;
+            const float4 v = *reinterpret_cast<const float4 *>(hp);
+            float *gp = gbase + qq * (CB_MAX_LEVELS + 1);
+            atomicAdd(gp + 0, v.x);
+            atomicAdd(gp + 1, v.y);
+            atomicAdd(gp + 2, v.z);
+            atomicAdd(gp + 3, v.w);
+            if (q4 == 0) atomicAdd(&Rs[ch][qq], *hw);
+            hp += ld_hp;
+            qt += d_out;
+            hw += d_out;
+        }
+    }
+    __syncthreads();
+    if (active) {                                    // G and R were zeroed by the host; row ranges add up
+        const int j = j0 + jj;
+        for (int q = 0; q < m; ++q)
+            for (int e = 0; e < 4; ++e)
+                atomicAdd(&G[(static_cast<size_t>(j) * CB_MAX_LEVELS + q) * CB_MAX_LEVELS + q4 + e],
+                          static_cast<double>(Gs[ch][q][q4 + e]));
+        for (int e = 0; e < 4; ++e)
+            atomicAdd(&R[static_cast<size_t>(j) * CB_MAX_LEVELS + q4 + e], static_cast<double>(Rs[ch][q4 + e]));
     }
 }
 

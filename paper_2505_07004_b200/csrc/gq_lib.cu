@@ -880,8 +880,12 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
             if (int32_t rc = launch_full(pq, mPm, mPm, mPm, GQ_KERNEL_CB_GEMM)) return rc;
             {
                 LaunchScope scope(GQ_KERNEL_CB_FOLD, st);
-                gq::cb_fold_kernel<<<dim3((nch + 7) / 8, 8), 128, 0, st>>>(HP, L.slab_ld, HW, Qt, static_cast<int>(d_in),
-                                                                 static_cast<int>(d_out), static_cast<int>(j0), nch, m, Gm, Rv);
+                if (m % 4 == 0)
+                    gq::cb_fold4_kernel<<<dim3((nch + gq::CB_FOLD4_CH - 1) / gq::CB_FOLD4_CH, 16), gq::CB_FOLD4_CH * 4, 0, st>>>(
+                        HP, L.slab_ld, HW, Qt, static_cast<int>(d_in), static_cast<int>(d_out), static_cast<int>(j0), nch, m, Gm, Rv);
+                else
+                    gq::cb_fold_kernel<<<dim3((nch + gq::CB_FOLD_CH - 1) / gq::CB_FOLD_CH, 16), gq::CB_FOLD_CH * 16, 0, st>>>(
+                        HP, L.slab_ld, HW, Qt, static_cast<int>(d_in), static_cast<int>(d_out), static_cast<int>(j0), nch, m, Gm, Rv);
             }
             GQ_CUDA(cudaGetLastError());
         }
