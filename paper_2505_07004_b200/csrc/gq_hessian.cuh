@@ -207,7 +207,7 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
     __shared__ __align__(8) uint64_t bar_full[HS_STAGES];    // first CTA: B bytes of both CTAs + all scaler warps
     __shared__ __align__(8) uint64_t bar_empty[HS_STAGES];   // both CTAs: signalled by the MMA commits
     __shared__ __align__(8) uint64_t bar_acc_full;           // both CTAs: signalled by the MMA commit
-    __shared__ __align__(8) uint64_t bar_acc_empty;          // first CTA: 16 epilogue warps arrive
+    __shared__ __align__(8) uint64_t bar_acc_empty[HS_GROUPS];   // first CTA, one per accumulator: 16 epilogue warps arrive
     __shared__ __align__(8) uint64_t bar_drain;
     __shared__ uint32_t tmem_base_smem;
     __shared__ volatile uint32_t abort_flag;
@@ -225,7 +225,7 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
             mbar_init(smem_u32(&bar_empty[s]), 1);
         }
         mbar_init(smem_u32(&bar_acc_full), 1);
-        mbar_init(smem_u32(&bar_acc_empty), 2 * HS_EPI_WARPS);
+        for (int kk = 0; kk < HS_GROUPS; ++kk) mbar_init(smem_u32(&bar_acc_empty[kk]), 2 * HS_EPI_WARPS);
         mbar_init(smem_u32(&bar_drain), 1);
         abort_flag = 0u;
         fence_mbar_init();
@@ -286,24 +286,48 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
         WorkItem w;
         for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
             const UnitDesc u = decode_unit(p, w.unit);
-            if (!bounded_wait_hot(smem_u32(&bar_acc_empty), acc_ph ^ 1u, wc, 2u, w.unit)) { ok = false; break; }
+            // The epilogue empties accumulator 0 first.  The first k-steps of the new unit (as many as the ring
+            // holds) are therefore issued for accumulator 0 as soon as it is free, while accumulator 1 is still
+            // being read out, then for accumulator 1; a stage is released after both.
+            auto issue = [&](int kk, int stage_idx, int ks) {
+                if (!u.use[kk]) return;
+                const uint32_t stage = ring + stage_idx * HS_STAGE_BYTES;
+                const uint32_t sa = stage + u.a_slot(kk) * HS_SLOT_BYTES;
+                const uint32_t sb = stage + u.b_slot(kk) * HS_SLOT_BYTES;
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(kk * TILE_N);
+#pragma unroll
+                for (int k16 = 0; k16 < TILE_K / 16; ++k16) {
+                    const uint64_t adesc = umma_smem_desc_mn_sw128(sa + k16 * 16 * 128, BOX_BYTES, 1024);
+                    const uint64_t bdesc = umma_smem_desc_mn_sw128(sb + k16 * 16 * 128, BOX_BYTES, 1024);
+                    umma_bf16(d_tmem, adesc, bdesc, idesc, (ks != w.ks0 || k16 != 0) ? 1u : 0u);
+                }
+            };
+            const int n_head = (w.ks1 - w.ks0 < HS_STAGES) ? (w.ks1 - w.ks0) : HS_STAGES;
+            if (!bounded_wait_hot(smem_u32(&bar_acc_empty[0]), acc_ph ^ 1u, wc, 2u, w.unit)) { ok = false; break; }
             tc_fence_after_sync();
-            for (int ks = w.ks0; ks < w.ks1; ++ks) {
+            {
+                int s_h = s;
+                uint32_t ph_h = ph;
+                for (int q = 0; q < n_head; ++q) {
+                    if (!bounded_wait_hot(smem_u32(&bar_full[s_h]), ph_h, wc, 3u, w.unit)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    issue(0, s_h, w.ks0 + q);
+                    if (++s_h == HS_STAGES) { s_h = 0; ph_h ^= 1u; }
+                }
+            }
+            if (!ok) break;
+            if (!bounded_wait_hot(smem_u32(&bar_acc_empty[1]), acc_ph ^ 1u, wc, 2u, w.unit)) { ok = false; break; }
+            tc_fence_after_sync();
+            for (int q = 0; q < n_head; ++q) {
+                issue(1, s, w.ks0 + q);
+                umma_commit_pair(smem_u32(&bar_empty[s]));
+                if (++s == HS_STAGES) { s = 0; ph ^= 1u; }
+            }
+            for (int ks = w.ks0 + n_head; ks < w.ks1; ++ks) {
                 if (!bounded_wait_hot(smem_u32(&bar_full[s]), ph, wc, 3u, w.unit)) { ok = false; break; }
                 tc_fence_after_sync();
-                const uint32_t stage = ring + s * HS_STAGE_BYTES;
-                for (int kk = 0; kk < HS_GROUPS; ++kk) {
-                    if (!u.use[kk]) continue;
-                    const uint32_t sa = stage + u.a_slot(kk) * HS_SLOT_BYTES;
-                    const uint32_t sb = stage + u.b_slot(kk) * HS_SLOT_BYTES;
-                    const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(kk * TILE_N);
-#pragma unroll
-                    for (int k16 = 0; k16 < TILE_K / 16; ++k16) {
-                        const uint64_t adesc = umma_smem_desc_mn_sw128(sa + k16 * 16 * 128, BOX_BYTES, 1024);
-                        const uint64_t bdesc = umma_smem_desc_mn_sw128(sb + k16 * 16 * 128, BOX_BYTES, 1024);
-                        umma_bf16(d_tmem, adesc, bdesc, idesc, (ks != w.ks0 || k16 != 0) ? 1u : 0u);
-                    }
-                }
+                issue(0, s, ks);
+                issue(1, s, ks);
                 umma_commit_pair(smem_u32(&bar_empty[s]));
                 if (++s == HS_STAGES) { s = 0; ph ^= 1u; }
             }
@@ -414,9 +438,8 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
             tc_fence_after_sync();
             const int row0 = u.ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + q * 32;
             for (int kk = 0; kk < HS_GROUPS; ++kk) {
-                if (!u.use[kk]) continue;
 #pragma unroll 1
-                for (int c4 = 0; c4 < 4; ++c4) {
+                for (int c4 = 0; u.use[kk] && c4 < 4; ++c4) {
                     const int cc = half * 4 + c4;
                     const int col0 = u.tj[kk] * TILE_N + cc * 32;
                     if (col0 >= p.d || row0 >= p.d) break;      // outside the matrix
@@ -438,11 +461,11 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                         bulk_commit_group();
                     }
                 }
+                // This warp has read all it needs from accumulator kk: tell the MMA issuer (first CTA).
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_acc_empty[kk]), 0));
             }
-            // This warp has read all it needs from tensor memory: tell the MMA issuer (first CTA).
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_acc_empty), 0));
             acc_ph ^= 1u;
         }
         if (lane == 0) bulk_wait_group_read0();       // shared memory must outlive the last reduce-add's read
