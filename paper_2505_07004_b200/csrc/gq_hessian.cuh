@@ -249,6 +249,7 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
         uint32_t issued = 0;
         bool ok = true;
         WorkItem w;
+        const uint64_t pol_x = l2_policy_evict_last();      // X is re-read by many units: keep it in L2
         for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
             const UnitDesc u = decode_unit(p, w.unit);
             const int n_b = u.wide ? (u.use[0] ? 1 : 0) + (u.use[1] ? 1 : 0) : 1;      // B blocks per stage
@@ -263,7 +264,7 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                     const int b0 = u.tj[kk] * TILE_N + static_cast<int>(rank) * CTA_ROWS;
 #pragma unroll
                     for (int q = 0; q < CTA_ROWS / BOX_FEATURES; ++q)
-                        tma_load_3d_pair(sb + q * BOX_BYTES, &mapX, full, b0 + q * BOX_FEATURES, ks * TILE_K, 0);
+                        tma_load_3d_pair_hint(sb + q * BOX_BYTES, &mapX, full, b0 + q * BOX_FEATURES, ks * TILE_K, 0, pol_x);
                 }
                 ++issued;
                 if (++s == HS_STAGES) { s = 0; ph ^= 1u; }
@@ -426,6 +427,7 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
         const int q = warp & 3;                         // TMEM lane quarter this warp may access
         const int half = ew >> 2;                       // which 128 of the 256 accumulator columns
         const uint32_t stg = staging + static_cast<uint32_t>(ew) * 4096u;
+        const uint64_t pol_h = l2_policy_evict_first();     // H is touched once per launch: it should not displace X
         uint32_t acc_ph = 0;
         bool ok = true;
         WorkItem w;
@@ -457,7 +459,7 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        tma_reduce_add_3d(&mapH, stg, col0, row0, u.grp[kk]);
+                        tma_reduce_add_3d_hint(&mapH, stg, col0, row0, u.grp[kk], pol_h);
                         bulk_commit_group();
                     }
                 }
