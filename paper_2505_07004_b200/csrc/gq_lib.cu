@@ -67,6 +67,7 @@ struct DeviceInfo {
     bool ready = false;
     int sm_count = 0;
     int max_pairs = 0;          // CTA pairs (clusters of two) of a tensor-core kernel that can be resident at once
+    int saliency_blocks = 1;    // CTAs of saliency_kernel that fit on one SM (its grid-stride grid is sized to fit)
     uint32_t *status_ptr = nullptr;
 };
 DeviceInfo g_dev[kMaxDevices];
@@ -128,6 +129,14 @@ int32_t device_info(DeviceInfo **out)
             if (clusters > di.sm_count / 2) clusters = di.sm_count / 2;
             if (clusters < 1) clusters = 1;
             di.max_pairs = clusters;
+        }
+        {
+            int blocks = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, gq::saliency_kernel, 256, 0) != cudaSuccess || blocks < 1) {
+                (void)cudaGetLastError();
+                blocks = 4;
+            }
+            di.saliency_blocks = blocks;
         }
         if (!g_encode) {
             void *fn = nullptr;
@@ -351,7 +360,7 @@ int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad,
     if (int32_t rc = device_info(&di)) return rc;
     const int m = static_cast<int>(d_out / g);
     const float coef = grad_scale * grad_scale / static_cast<float>(m);
-    const int grid = grid_for(n * g * 32, 256, di->sm_count, 8);
+    const int grid = grid_for(n * g * 32, 256, di->sm_count, di->saliency_blocks);    // one resident wave
     {
         LaunchScope scope(GQ_KERNEL_SALIENCY, static_cast<cudaStream_t>(stream));
         gq::saliency_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
