@@ -324,7 +324,23 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
                 umma_commit_pair(smem_u32(&bar_empty[s]));
                 if (++s == HS_STAGES) { s = 0; ph ^= 1u; }
             }
-            for (int ks = w.ks0 + n_head; ks < w.ks1; ++ks) {
+            int ks = w.ks0 + n_head;
+            for (; ks + 1 < w.ks1; ks += 2) {             // two k-steps at a time: eight MMAs in a row per accumulator
+                const int s2 = (s + 1 == HS_STAGES) ? 0 : s + 1;
+                const uint32_t ph2 = (s + 1 == HS_STAGES) ? (ph ^ 1u) : ph;
+                if (!bounded_wait_hot(smem_u32(&bar_full[s]), ph, wc, 3u, w.unit)) { ok = false; break; }
+                if (!bounded_wait_hot(smem_u32(&bar_full[s2]), ph2, wc, 3u, w.unit)) { ok = false; break; }
+                tc_fence_after_sync();
+                issue(0, s, ks);
+                issue(0, s2, ks + 1);
+                issue(1, s, ks);
+                umma_commit_pair(smem_u32(&bar_empty[s]));
+                issue(1, s2, ks + 1);
+                umma_commit_pair(smem_u32(&bar_empty[s2]));
+                s = (s2 + 1 == HS_STAGES) ? 0 : s2 + 1;
+                ph = (s2 + 1 == HS_STAGES) ? (ph2 ^ 1u) : ph2;
+            }
+            for (; ok && ks < w.ks1; ++ks) {
                 if (!bounded_wait_hot(smem_u32(&bar_full[s]), ph, wc, 3u, w.unit)) { ok = false; break; }
                 tc_fence_after_sync();
                 issue(0, s, ks);
