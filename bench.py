@@ -40,7 +40,7 @@ METRIC = "guided_hessian_tokens_per_s"
 UNIT = "tokens/s"
 # DRAM bytes per launch of the dominant kernel from the committed ncu capture (profiles/), scaled to
 # one launch of the default workload; None until a capture exists for the current kernel.
-NCU_TRAFFIC_BYTES = {"c1_7b_attn": 346.79e6}      # profiles/hessian_kernel_c1_7b_attn.md
+NCU_TRAFFIC_BYTES = {"c1_7b_attn": 343.36e6}      # profiles/hessian_kernel_c1_7b_attn.md
 
 
 def load_peaks():
