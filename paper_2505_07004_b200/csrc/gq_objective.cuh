@@ -285,40 +285,54 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
         for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
             ItemGeom ge;
             if (!item_geom<MODE>(p, w, rank, ge)) continue;
-            ok = bounded_wait(smem_u32(&bar_acc_full[buf]), acc_ph, wc, 4u, w.unit);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after_sync();
             if (MODE == MODE_OBJECTIVE) {
+                // The H values this warp needs do not depend on the accumulator: the first block's are requested
+                // before the wait for the MMAs, every other block's while the block before it is being used.
                 const int ti = ge.ti, tj = ge.tj, k = ge.k;
                 const int row0 = ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + q * 32;
                 const int row = row0 + lane;
                 const bool row_ok = row < p.d;
                 const float *hrow = p.H + (static_cast<size_t>(k) * p.d + (row_ok ? row : 0)) * static_cast<size_t>(p.d);
-                double dsum = 0.0;
-#pragma unroll 1
-                for (int cc = 0; cc < TILE_N / 32; ++cc) {
+                auto block_active = [&](int cc) {
                     const int col0 = tj * TILE_N + cc * 32;
-                    if (col0 >= p.d) break;                    // right of the matrix
-                    if (col0 + 32 <= row0) continue;           // 32 x 32 block strictly below the diagonal
-                    if (row0 >= p.d) break;                    // below the matrix
+                    return col0 < p.d && row0 < p.d && col0 + 32 > row0;      // inside the matrix, not below the diagonal
+                };
+                auto load_block = [&](int cc, float4 (&h)[8]) {
+                    const int col0 = tj * TILE_N + cc * 32;
+                    const bool act = row_ok && block_active(cc);
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        const int c = col0 + v * 4;
+                        h[v] = (act && c < p.d && c + 3 >= row) ? __ldg(reinterpret_cast<const float4 *>(hrow + c))
+                                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                };
+                float4 hq[2][8];
+                load_block(0, hq[0]);
+                ok = bounded_wait(smem_u32(&bar_acc_full[buf]), acc_ph, wc, 4u, w.unit);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after_sync();
+                double dsum = 0.0;
+#pragma unroll
+                for (int cc = 0; cc < TILE_N / 32; ++cc) {
+                    if (cc + 1 < TILE_N / 32) load_block(cc + 1, hq[(cc + 1) & 1]);
+                    if (!block_active(cc)) continue;           // uniform over the warp
+                    const int col0 = tj * TILE_N + cc * 32;
                     uint32_t r[32];
                     tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                       static_cast<uint32_t>(buf * TILE_N + cc * 32), r);
                     tmem_ld_wait();
-                    if (!row_ok) continue;
                     float part = 0.0f;
 #pragma unroll
                     for (int v = 0; v < 8; ++v) {
                         const int c = col0 + v * 4;
-                        if (c < p.d && c + 3 >= row) {
-                            const float4 h = __ldg(reinterpret_cast<const float4 *>(hrow + c));
-                            const float hv[4] = {h.x, h.y, h.z, h.w};
+                        const float4 h = hq[cc & 1][v];        // zero where it was not loaded
+                        const float hv[4] = {h.x, h.y, h.z, h.w};
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const float wgt = (c + e > row) ? 2.0f : ((c + e == row) ? 1.0f : 0.0f);
-                                part = fmaf(wgt * __uint_as_float(r[v * 4 + e]), hv[e], part);
-                            }
+                        for (int e = 0; e < 4; ++e) {
+                            const float wgt = (c + e > row) ? 2.0f : ((c + e == row) ? 1.0f : 0.0f);
+                            part = fmaf(wgt * __uint_as_float(r[v * 4 + e]), hv[e], part);
                         }
                     }
                     dsum += static_cast<double>(part);
@@ -331,6 +345,15 @@ pair_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
                 for (int off = 16; off > 0; off >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, off);
                 if (lane == 0)
                     p.partials[static_cast<size_t>(w.unit) * PARTIALS_PER_UNIT + rank * 4 + q] = dsum;
+                buf ^= 1;
+                if (buf == 0) acc_ph ^= 1u;
+                continue;
+            }
+            ok = bounded_wait(smem_u32(&bar_acc_full[buf]), acc_ph, wc, 4u, w.unit);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            if (MODE == MODE_OBJECTIVE) {
             } else if (MODE == MODE_FULL) {
                 const int row0 = ge.ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + q * 32;
                 const int row = row0 + lane;
