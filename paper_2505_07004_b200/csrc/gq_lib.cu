@@ -18,6 +18,7 @@
 #include "gq_cd.cuh"
 #include "gq_codebook.cuh"
 #include "gq_exchange.cuh"
+#include "gq_wide_gemm.cuh"
 #include "gq_kernels.cuh"
 
 #define GQ_VERSION_NUMBER 100   /* 0.1.0 */
@@ -104,6 +105,7 @@ int32_t device_info(DeviceInfo **out)
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, gq::OBJ_SMEM_BYTES));
         GQ_CUDA(cudaFuncSetAttribute(gq::pair_gemm_kernel<gq::MODE_FULL>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, gq::OBJ_SMEM_BYTES));
+        GQ_CUDA(cudaFuncSetAttribute(gq::wide_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gq::WG_SMEM_BYTES));
         GQ_CUDA(cudaFuncSetAttribute(gq::cd_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      gq::CD_SMEM_BYTES));
         GQ_CUDA(cudaFuncSetAttribute(gq::hessian_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -831,7 +833,7 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
     if (int32_t rc = make_map(&mPm, Pm, L.slab_ld, d_in, 1, L.slab_ld, d_in * L.slab_ld)) return rc;
 
     auto launch_full = [&](gq::PairGemmParams &pp, const CUtensorMap &b0, const CUtensorMap &b1, const CUtensorMap &b2,
-                           int kernel_id) -> int32_t {
+                           int kernel_id, bool wide) -> int32_t {
         pp.d = static_cast<int>(d_in);
         pp.rows = static_cast<int>(d_in);
         pp.g = g;
@@ -839,15 +841,19 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
         pp.map_grouped[3] = pp.map_grouped[4] = pp.map_grouped[5] = 0;
         pp.col_tiles = (pp.cols + gq::TILE_N - 1) / gq::TILE_N;
         const int row_blocks = static_cast<int>((d_in + gq::TILE_M - 1) / gq::TILE_M);
-        const int units = row_blocks * pp.col_tiles;
+        // wide: a unit is a row block times two neighbouring column tiles (gq_wide_gemm.cuh)
+        const int units = row_blocks * (wide ? (pp.col_tiles + 1) / 2 : pp.col_tiles);
         const int ksteps = pp.n_terms * static_cast<int>((d_in + gq::TILE_K - 1) / gq::TILE_K);
         pp.sched = gq::plan_schedule(units, ksteps, units < di->max_pairs ? units : di->max_pairs, false);
         pp.status = di->status_ptr;
         pp.wait_budget_ns = wait_budget_ns();
         {
             LaunchScope scope(kernel_id, st);
-            gq::pair_gemm_kernel<gq::MODE_FULL><<<2 * pp.sched.pairs, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(
-                mH0, mH1, mH1, b0, b1, b2, pp);
+            if (wide)
+                gq::wide_gemm_kernel<<<2 * pp.sched.pairs, gq::WG_THREADS, gq::WG_SMEM_BYTES, st>>>(mH0, mH1, mH1, b0, b1, b2, pp);
+            else
+                gq::pair_gemm_kernel<gq::MODE_FULL><<<2 * pp.sched.pairs, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(
+                    mH0, mH1, mH1, b0, b1, b2, pp);
         }
         GQ_CUDA(cudaGetLastError());
         return GQ_OK;
@@ -866,7 +872,7 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
         pp.cols = static_cast<int>(mk);
         pp.C = HW + k * mk;
         pp.ldc = d_out;
-        if (int32_t rc = launch_full(pp, mW0, mW1, mW1, GQ_KERNEL_CB_GEMM)) return rc;
+        if (int32_t rc = launch_full(pp, mW0, mW1, mW1, GQ_KERNEL_CB_GEMM, false)) return rc;
         for (int64_t j0 = k * mk; j0 < (k + 1) * mk; j0 += L.slab_channels) {
             const int nch = static_cast<int>((k + 1) * mk - j0 < L.slab_channels ? (k + 1) * mk - j0 : L.slab_channels);
             {
@@ -886,7 +892,7 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
             pq.cols = nch * m;
             pq.C = HP;
             pq.ldc = L.slab_ld;
-            if (int32_t rc = launch_full(pq, mPm, mPm, mPm, GQ_KERNEL_CB_GEMM)) return rc;
+            if (int32_t rc = launch_full(pq, mPm, mPm, mPm, GQ_KERNEL_CB_GEMM, pq.cols > 2 * gq::TILE_N)) return rc;
             {
                 LaunchScope scope(GQ_KERNEL_CB_FOLD, st);
                 if (m % 4 == 0)

@@ -61,6 +61,8 @@ def gpu_codebook(dev, W, Q, m, H, lam=1e-7):
     (2, 520, 48, 2, 16),        # 24 channels per group
     (3, 1032, 256, 1, 2),
     (4, 768, 2304, 2, 16),      # 1152 channels per group: two slabs of one-hot columns (1024 + 128)
+    (5, 520, 192, 2, 8),        # 768 one-hot columns per group: three column tiles, the wide product's odd last tile
+    (6, 264, 208, 2, 8),        # 832 columns: four column tiles, the last one ragged
 ])
 def test_codebook_update_matches_oracle(dev, seed, d_in, d_out, g, m):
     W, W0, Q0, cb0, H = make_problem(seed, d_in, d_out, g, m)
