@@ -96,16 +96,6 @@ struct UnitDesc {
     __device__ int scaled_groups() const { return wide ? 1 : 2; }
 };
 
-// Slot t of the enumeration of (row block i, column-block pair q) with i <= 2q + 1, pairs outermost.
-__device__ __forceinline__ void colpair_of_slot(int t, int &i, int &q)
-{
-    int qq = static_cast<int>((sqrtf(4.0f * static_cast<float>(t) + 1.0f) - 1.0f) * 0.5f);
-    while (qq * qq + qq > t) --qq;
-    while ((qq + 1) * (qq + 1) + (qq + 1) <= t) ++qq;
-    q = qq;
-    i = t - qq * qq - qq;
-}
-
 struct HessianParams;
 __device__ __forceinline__ UnitDesc decode_unit(const HessianParams &p, int unit);
 

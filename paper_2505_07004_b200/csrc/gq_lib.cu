@@ -105,7 +105,8 @@ int32_t device_info(DeviceInfo **out)
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, gq::OBJ_SMEM_BYTES));
         GQ_CUDA(cudaFuncSetAttribute(gq::pair_gemm_kernel<gq::MODE_FULL>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, gq::OBJ_SMEM_BYTES));
-        GQ_CUDA(cudaFuncSetAttribute(gq::wide_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gq::WG_SMEM_BYTES));
+        GQ_CUDA(cudaFuncSetAttribute(gq::wide_gemm_kernel<gq::WG_FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, gq::WG_SMEM_BYTES));
+        GQ_CUDA(cudaFuncSetAttribute(gq::wide_gemm_kernel<gq::WG_OBJECTIVE>, cudaFuncAttributeMaxDynamicSharedMemorySize, gq::WG_SMEM_BYTES));
         GQ_CUDA(cudaFuncSetAttribute(gq::cd_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      gq::CD_SMEM_BYTES));
         GQ_CUDA(cudaFuncSetAttribute(gq::hessian_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -268,7 +269,7 @@ ObjectiveLayout objective_layout(int64_t d_in, int64_t d_out, int32_t g)
     L.lo_off = mat;
     L.partials_off = 2 * mat;
     L.total = L.partials_off +
-              round_up(static_cast<size_t>(tiles_for(d_in)) * g * gq::PARTIALS_PER_UNIT * sizeof(double), 1024);
+              round_up(static_cast<size_t>(tiles_for(d_in)) * g * gq::WG_PARTIALS_PER_UNIT * sizeof(double), 1024);
     return L;
 }
 
@@ -545,8 +546,9 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     p.term_a[2] = 1; p.term_b[2] = 0;
     p.map_grouped[0] = 1;
     p.map_grouped[1] = 1;
-    const int tiles = tiles_for(d_in);
-    const int units = tiles * g;
+    // units: (row block, pair of neighbouring column tiles, group) over the upper triangle (gq_wide_gemm.cuh)
+    const int slots = colpair_slots_for(d_in);
+    const int units = slots * g;
     const int ksteps = 3 * static_cast<int>((m + gq::TILE_K - 1) / gq::TILE_K);
     p.sched = gq::plan_schedule(units, ksteps, units < di->max_pairs ? units : di->max_pairs, false);
     p.H = H;
@@ -556,13 +558,13 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     const int grid = 2 * p.sched.pairs;
     {
         LaunchScope scope(GQ_KERNEL_GRAM_DOT, st);
-        gq::pair_gemm_kernel<gq::MODE_OBJECTIVE><<<grid, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(mapHi, mapLo, mapHi, mapLo, mapHi,
-                                                                                               mapLo, p);
+        gq::wide_gemm_kernel<gq::WG_OBJECTIVE><<<grid, gq::WG_THREADS, gq::WG_SMEM_BYTES, st>>>(mapHi, mapLo, mapHi, mapLo, mapHi,
+                                                                                           mapLo, p);
     }
     GQ_CUDA(cudaGetLastError());
     {
         LaunchScope scope(GQ_KERNEL_REDUCE, st);
-        gq::reduce_partials_kernel<<<1, 1024, 0, st>>>(partials, tiles, g, gq::PARTIALS_PER_UNIT, loss_out);
+        gq::reduce_partials_kernel<<<1, 1024, 0, st>>>(partials, slots, g, gq::WG_PARTIALS_PER_UNIT, loss_out);
     }
     GQ_CUDA(cudaGetLastError());
     return GQ_OK;
@@ -850,7 +852,7 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
         {
             LaunchScope scope(kernel_id, st);
             if (wide)
-                gq::wide_gemm_kernel<<<2 * pp.sched.pairs, gq::WG_THREADS, gq::WG_SMEM_BYTES, st>>>(mH0, mH1, mH1, b0, b1, b2, pp);
+                gq::wide_gemm_kernel<gq::WG_FULL><<<2 * pp.sched.pairs, gq::WG_THREADS, gq::WG_SMEM_BYTES, st>>>(mH0, mH1, mH1, b0, b1, b2, pp);
             else
                 gq::pair_gemm_kernel<gq::MODE_FULL><<<2 * pp.sched.pairs, gq::OBJ_THREADS, gq::OBJ_SMEM_BYTES, st>>>(
                     mH0, mH1, mH1, b0, b1, b2, pp);

@@ -117,6 +117,16 @@ __host__ __device__ inline void tile_of_slot_blocked(int t, int nj, int R, int &
     }
 }
 
+// Slot t of the enumeration of (row block i, column-block pair q) with i <= 2q + 1, pairs outermost.
+__device__ __forceinline__ void colpair_of_slot(int t, int &i, int &q)
+{
+    int qq = static_cast<int>((sqrtf(4.0f * static_cast<float>(t) + 1.0f) - 1.0f) * 0.5f);
+    while (qq * qq + qq > t) --qq;
+    while ((qq + 1) * (qq + 1) + (qq + 1) <= t) ++qq;
+    q = qq;
+    i = t - qq * qq - qq;
+}
+
 struct WorkItem {
     int unit;      // (tile slot) * g + group
     int ks0, ks1;  // k-step range [ks0, ks1) of the unit's `ksteps`

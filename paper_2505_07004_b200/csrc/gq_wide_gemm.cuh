@@ -9,6 +9,11 @@
 // hidden behind the next unit except for its first k-steps (same scheme as in gq_hessian.cuh), which the long
 // contraction (all of d_in, two terms) makes affordable.
 //
+// The objective (Eq. 7) runs the same way (WG_OBJECTIVE): a unit is (row block i, pair of column tiles 2q and
+// 2q + 1, group) over the upper triangle, A = B = Delta of the group (bf16 hi + lo, three terms), and the
+// epilogue contracts both accumulators with H_k as pair_gemm_kernel<MODE_OBJECTIVE> does, one fp64 partial per
+// (unit, CTA, epilogue warp), whole units only, so the result is reproducible.
+//
 // Roles: warp 0 (one lane) TMA producer, warp 1 (one lane, first CTA) MMA issuer, warp 2 TMEM allocation,
 // warps 4..11 epilogue (tcgen05.ld, plain 16-byte stores; whole units only, one writer per element).
 // Every mbarrier wait is bounded (gq_pipeline.cuh).
@@ -28,10 +33,22 @@ constexpr int WG_STAGE_BYTES = 3 * WG_SLOT_BYTES;                         // [B0
 constexpr int WG_EPI_WARPS = 8;
 constexpr int WG_THREADS = 32 * (4 + WG_EPI_WARPS);
 constexpr int WG_SMEM_BYTES = WG_STAGES * WG_STAGE_BYTES + 1024;
+constexpr int WG_FULL = 0;
+constexpr int WG_OBJECTIVE = 1;
+constexpr int WG_PARTIALS_PER_UNIT = 2 * WG_EPI_WARPS;        // one fp64 per (CTA of the pair, epilogue warp)
 
-// Uses the MODE_FULL fields of PairGemmParams (d, rows, n_terms, term_a/b, map_grouped, full_k, col0, cols,
-// col_tiles, C, ldc, sched, status, wait_budget_ns); units = row blocks * ceil(col_tiles / 2),
-// sched.ksteps = n_terms * ceil(rows / 64).
+struct WideUnit {
+    int ti;          // row block
+    int tj[2];       // column tile of accumulator 0 / 1
+    bool use[2];
+    int k;           // third coordinate of the grouped maps
+};
+
+// WG_FULL uses the MODE_FULL fields of PairGemmParams (d, rows, n_terms, term_a/b, map_grouped, full_k, col0,
+// cols, col_tiles, C, ldc), units = row blocks * ceil(col_tiles / 2); WG_OBJECTIVE the MODE_OBJECTIVE fields
+// (d, rows, g, nj, H, partials with WG_PARTIALS_PER_UNIT slots per unit), units = column-pair slots * g.
+// sched.ksteps = n_terms * ceil(rows / 64) in both.
+template <int WMODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(WG_THREADS, 1)
 wide_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1,
                  const __grid_constant__ CUtensorMap map2, const __grid_constant__ CUtensorMap map3,
@@ -82,12 +99,28 @@ wide_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
     const int kblocks = (p.rows + TILE_K - 1) / TILE_K;
     const int col_pairs = (p.col_tiles + 1) / 2;
 
-    // unit -> row block, first column tile, whether the second column tile exists
-    auto decode = [&](int unit, int &ti, int &tj0, bool &two) {
-        ti = unit / col_pairs;
-        tj0 = 2 * (unit - ti * col_pairs);
-        two = tj0 + 1 < p.col_tiles;
+    auto decode = [&](int unit) {
+        WideUnit u;
+        if (WMODE == WG_FULL) {
+            u.ti = unit / col_pairs;
+            u.tj[0] = 2 * (unit - u.ti * col_pairs);
+            u.tj[1] = u.tj[0] + 1;
+            u.use[0] = true;
+            u.use[1] = u.tj[1] < p.col_tiles;
+            u.k = p.full_k;
+        } else {
+            int i, q;
+            colpair_of_slot(unit / p.g, i, q);
+            u.ti = i;
+            u.tj[0] = 2 * q;
+            u.tj[1] = 2 * q + 1;
+            u.use[0] = 2 * q >= i;               // tile (i, 2q) touches the upper triangle
+            u.use[1] = 2 * q + 1 < p.nj;
+            u.k = unit % p.g;
+        }
+        return u;
     };
+    const int col_base = (WMODE == WG_FULL) ? p.col0 : 0;
 
     if (warp == 0 && lane == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -98,29 +131,29 @@ wide_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
         WorkItem w;
         const void *maps[MAX_MAPS] = {&map0, &map1, &map2, &map3, &map4, &map5};
         for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
-            int ti, tj0;
-            bool two;
-            decode(w.unit, ti, tj0, two);
-            const int a0 = ti * TILE_M + static_cast<int>(rank) * CTA_ROWS;
-            const int b0 = p.col0 + tj0 * TILE_N + static_cast<int>(rank) * CTA_ROWS;
+            const WideUnit u = decode(w.unit);
+            const int a0 = u.ti * TILE_M + static_cast<int>(rank) * CTA_ROWS;
+            const int n_ops = 1 + (u.use[0] ? 1 : 0) + (u.use[1] ? 1 : 0);
             for (int ks = w.ks0; ks < w.ks1; ++ks) {
                 const int term = ks / kblocks;
                 const int row = (ks - term * kblocks) * TILE_K;
                 const int ma = p.term_a[term], mb = p.term_b[term];
-                const int ka = p.map_grouped[ma] ? p.full_k : 0;
-                const int kb = p.map_grouped[mb] ? p.full_k : 0;
+                const int ka = p.map_grouped[ma] ? u.k : 0;
+                const int kb = p.map_grouped[mb] ? u.k : 0;
                 if (!bounded_wait(smem_u32(&bar_empty[s]), ph ^ 1u, wc, 1u, w.unit)) { ok = false; break; }
                 const uint32_t full_local = smem_u32(&bar_full[s]);
-                if (rank == 0) mbar_arrive_expect_tx(full_local, 2 * (two ? 3 : 2) * WG_SLOT_BYTES);   // both CTAs' bytes
+                if (rank == 0) mbar_arrive_expect_tx(full_local, 2 * n_ops * WG_SLOT_BYTES);   // both CTAs' bytes
                 const uint32_t full = map_to_cta(full_local, 0);
                 const uint32_t stage = ring + s * WG_STAGE_BYTES;
 #pragma unroll
                 for (int q = 0; q < CTA_ROWS / BOX_FEATURES; ++q) {
                     tma_load_3d_pair(stage + WG_SLOT_BYTES + q * BOX_BYTES, maps[ma], full, a0 + q * BOX_FEATURES, row, ka);
-                    tma_load_3d_pair(stage + q * BOX_BYTES, maps[mb], full, b0 + q * BOX_FEATURES, row, kb);
-                    if (two)
-                        tma_load_3d_pair(stage + 2 * WG_SLOT_BYTES + q * BOX_BYTES, maps[mb], full,
-                                         b0 + TILE_N + q * BOX_FEATURES, row, kb);
+#pragma unroll
+                    for (int kk = 0; kk < 2; ++kk)
+                        if (u.use[kk])
+                            tma_load_3d_pair(stage + (kk ? 2 * WG_SLOT_BYTES : 0) + q * BOX_BYTES, maps[mb], full,
+                                             col_base + u.tj[kk] * TILE_N + static_cast<int>(rank) * CTA_ROWS + q * BOX_FEATURES,
+                                             row, kb);
                 }
                 ++issued;
                 if (++s == WG_STAGES) { s = 0; ph ^= 1u; }
@@ -142,11 +175,9 @@ wide_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
         bool ok = true;
         WorkItem w;
         for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
-            int ti, tj0;
-            bool two;
-            decode(w.unit, ti, tj0, two);
+            const WideUnit u = decode(w.unit);
             auto issue = [&](int kk, int stage_idx, int ks) {
-                if (kk == 1 && !two) return;
+                if (!u.use[kk]) return;
                 const uint32_t stage = ring + stage_idx * WG_STAGE_BYTES;
                 const uint32_t sa = stage + WG_SLOT_BYTES;
                 const uint32_t sb = stage + (kk ? 2 * WG_SLOT_BYTES : 0);
@@ -224,22 +255,86 @@ wide_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
         bool ok = true;
         WorkItem w;
         for (int it = 0; ok && work_item(p.sched, pair, it, w); ++it) {
-            int ti, tj0;
-            bool two;
-            decode(w.unit, ti, tj0, two);
+            const WideUnit u = decode(w.unit);
+            const int row0 = u.ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + q * 32;
+            const int row = row0 + lane;
+            if (WMODE == WG_OBJECTIVE) {
+                // sum_{a <= b} (2 - [a == b]) D[a][b] H_k[a][b] over this warp's four 32 x 32 blocks of each
+                // accumulator.  The H values do not depend on the accumulators: the first block's are requested
+                // before the wait for the MMAs, every other block's while the block before it is being used.
+                const bool row_ok = row < p.d;
+                const float *hrow = p.H + (static_cast<size_t>(u.k) * p.d + (row_ok ? row : 0)) * static_cast<size_t>(p.d);
+                auto block_col0 = [&](int b) { return u.tj[b >> 2] * TILE_N + (half * 4 + (b & 3)) * 32; };
+                auto block_active = [&](int b) {                 // uniform over the warp
+                    const int col0 = block_col0(b);
+                    return u.use[b >> 2] && col0 < p.d && row0 < p.d && col0 + 32 > row0;
+                };
+                auto load_block = [&](int b, float4 (&h)[8]) {
+                    const int col0 = block_col0(b);
+                    const bool act = row_ok && block_active(b);
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        const int c = col0 + v * 4;
+                        h[v] = (act && c < p.d && c + 3 >= row) ? __ldg(reinterpret_cast<const float4 *>(hrow + c))
+                                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                };
+                float4 hq[2][8];
+                load_block(0, hq[0]);
+                if (lane == 0) ok = bounded_wait(smem_u32(&bar_acc_full), acc_ph, wc, 4u, w.unit);
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                (void)mbar_try_wait(smem_u32(&bar_acc_full), acc_ph);     // every lane observes the completed phase
+                tc_fence_after_sync();
+                double dsum = 0.0;
+#pragma unroll
+                for (int b = 0; b < 8; ++b) {
+                    if (b + 1 < 8) load_block(b + 1, hq[(b + 1) & 1]);
+                    if (block_active(b)) {
+                        const int col0 = block_col0(b);
+                        uint32_t r[32];
+                        tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
+                                          static_cast<uint32_t>((b >> 2) * TILE_N + (half * 4 + (b & 3)) * 32), r);
+                        tmem_ld_wait();
+                        float part = 0.0f;
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            const int c = col0 + v * 4;
+                            const float4 h = hq[b & 1][v];         // zero where it was not loaded
+                            const float hv[4] = {h.x, h.y, h.z, h.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float wgt = (c + e > row) ? 2.0f : ((c + e == row) ? 1.0f : 0.0f);
+                                part = fmaf(wgt * __uint_as_float(r[v * 4 + e]), hv[e], part);
+                            }
+                        }
+                        dsum += static_cast<double>(part);
+                    }
+                    if ((b & 3) == 3) {
+                        // This warp has read all it needs from accumulator b / 4: tell the MMA issuer (first CTA).
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_acc_empty[b >> 2]), 0));
+                    }
+                }
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, off);
+                if (lane == 0)
+                    p.partials[static_cast<size_t>(w.unit) * WG_PARTIALS_PER_UNIT + rank * WG_EPI_WARPS + ew] = dsum;
+                acc_ph ^= 1u;
+                continue;
+            }
             if (lane == 0) ok = bounded_wait(smem_u32(&bar_acc_full), acc_ph, wc, 4u, w.unit);
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             (void)mbar_try_wait(smem_u32(&bar_acc_full), acc_ph);     // every lane observes the completed phase
             tc_fence_after_sync();
-            const int row0 = ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + q * 32;
-            const int row = row0 + lane;
             float *crow = p.C + static_cast<size_t>(row < p.d ? row : 0) * p.ldc;
             for (int kk = 0; kk < 2; ++kk) {
 #pragma unroll 1
-                for (int c4 = 0; (kk == 0 || two) && c4 < 4; ++c4) {
+                for (int c4 = 0; u.use[kk] && c4 < 4; ++c4) {
                     const int cc = half * 4 + c4;
-                    const int c0 = (tj0 + kk) * TILE_N + cc * 32;          // column relative to col0
+                    const int c0 = u.tj[kk] * TILE_N + cc * 32;            // column relative to col0
                     if (c0 >= p.cols || row0 >= p.d) break;
                     uint32_t r[32];
                     tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) +

@@ -48,9 +48,9 @@ def test_workspace_sizes(L):
     assert L.gq_hessian_workspace_bytes(1, 8, 1, 0) == 1024                    # rounded up to 1 KiB
     assert L.gq_hessian_workspace_bytes(8192, 4096, 4, 2) == 0                 # unknown flag
     assert L.gq_hessian_workspace_bytes(8192, 4100, 4, 0) == 0                 # d_in % 8 != 0
-    # objective: two bf16 copies of delta + 8 fp64 partial sums per (upper-triangular 256 x 256 tile, group)
+    # objective: two bf16 copies of delta + room for 16 fp64 partial sums per (upper-triangular 256 x 256 tile, group)
     nj = 4096 // 256
-    assert L.gq_objective_workspace_bytes(4096, 4096, 4) == 2 * 4096 * 4096 * 2 + (nj * (nj + 1) // 2) * 4 * 8 * 8
+    assert L.gq_objective_workspace_bytes(4096, 4096, 4) == 2 * 4096 * 4096 * 2 + (nj * (nj + 1) // 2) * 4 * 16 * 8
     assert L.gq_objective_workspace_bytes(4096, 4096, 3) == 0          # d_out % g != 0
     assert L.gq_objective_workspace_bytes(4096, 24, 6) == 0            # (d_out / g) % 8 != 0
     assert L.gq_layer_host_arena_bytes(0, 4096, 4096, 4) == 0
