@@ -967,14 +967,8 @@ int32_t gq_selftest_wait_timeout(int32_t budget_ms, void *stream)
 
 int32_t gq_kernel_timing_enable(int32_t enable)
 {
-    std::lock_guard<std::mutex> lock(g_timing_mutex);
-    for (auto &v : g_timing_events) {
-        for (auto &pr : v) {
-            cudaEventDestroy(pr.first);
-            cudaEventDestroy(pr.second);
-        }
-        v.clear();
-    }
+    // Only the switch: what has been recorded so far stays until gq_kernel_timing_read collects it, so that a
+    // caller can time a sample of its launches (switch on, run, switch off, run untimed, ...).
     g_timing_on.store(enable ? 1 : 0);
     return GQ_OK;
 }
