@@ -237,6 +237,8 @@ int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, i
  * decision, is fp32.  Decisions can therefore differ from exact arithmetic only where the rounding
  * target lies within about 1e-5 (relative to the values involved) of the midpoint between two codebook
  * values; from such a coordinate on that channel follows its own, equally valid, descent path.
+ * The pieces of a block's tensor-core product are combined with atomic adds in no fixed order, so two runs
+ * on the same inputs agree bit for bit only as long as no decision falls within that rounding of a tie.
  */
 int32_t gq_cd_cycles(const float *W, float *W_hat, uint8_t *Q, const float *codebook, int32_t m,
                      int64_t d_in, int64_t d_out, const float *H, int32_t g, int32_t cycles,
