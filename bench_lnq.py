@@ -2,14 +2,13 @@
 """Times gq_cd_cycles (cyclic coordinate descent with fixed codebooks, Algorithm 4) and, optionally, the LNQ loop
 (Algorithm 2: gq_codebook_update + gq_cd_cycles) on a synthetic layer.
 
-    python -m paper_2505_07004_b200.bench_cd [--d-in 4096] [--d-out 4096] [--g 4] [--levels 16] [--cycles 2]
-                                             [--tokens 8192] [--oracle-channels 0] [--lnq-rounds 0]
+    python bench_lnq.py [--d-in 4096] [--d-out 4096] [--g 4] [--levels 16] [--cycles 2]
+                        [--tokens 8192] [--lnq-rounds 0]
 
 The layer's guided Hessians come from the library's own path (gq_saliency, gq_hessian_accumulate,
 gq_hessian_finalize on seeded synthetic activations and gradients), the codebooks are per-channel grids
 between the smallest and largest weight, and the starting point is nearest-level rounding.  Prints one JSON
-line: milliseconds per cycle, per-kernel device time, the objective before and after (gq_objective), and,
-with --oracle-channels C > 0, the time the CPU fp64 oracle needs for one cycle on C channels per group.
+line: milliseconds per cycle, per-kernel device time, and the objective before and after (gq_objective).
 """
 from __future__ import annotations
 
@@ -17,11 +16,10 @@ import argparse
 import json
 import os
 import sys
-import time
 
 import torch
 
-ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
@@ -36,12 +34,11 @@ def main():
     ap.add_argument("--levels", type=int, default=16)
     ap.add_argument("--cycles", type=int, default=2)
     ap.add_argument("--tokens", type=int, default=8192)
-    ap.add_argument("--oracle-channels", type=int, default=0)
     ap.add_argument("--lnq-rounds", type=int, default=0,
                     help="also time Algorithm 2: this many rounds of (codebook step, --cycles CD cycles) + a final codebook step")
     args = ap.parse_args()
     if not torch.cuda.is_available():
-        raise RuntimeError("bench_cd needs a CUDA device: libgq has no CPU path")
+        raise RuntimeError("bench_lnq.py needs a CUDA device: libgq has no CPU path")
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
     cfg = synth.LayerConfig("cd", args.tokens, min(args.tokens, 8192), args.d_in, args.d_out, (args.g,), "lognormal",
@@ -107,18 +104,6 @@ def main():
         out["lnq"] = {"rounds": args.lnq_rounds, "cd_cycles_per_round": args.cycles, "ms_total": e0.elapsed_time(e1),
                       "kernels_ms": {k: {"ms": round(v[0], 4), "launches": v[1]} for k, v in kern.items() if v[1]},
                       "objective_start": traj[0], "objective_end": traj[1]}
-    if args.oracle_channels > 0:
-        from oracle import cd_oracle as cdo
-        mk = cfg.d_out // g
-        cpg = min(args.oracle_channels, mk)
-        rows = torch.cat([torch.arange(k * mk, k * mk + cpg) for k in range(g)])
-        Wn, W0n, cbn = (t[rows].contiguous().cpu().numpy() for t in (W, W0, cb))
-        Hn = H.cpu().numpy()
-        t0 = time.perf_counter()
-        cdo.cd(Wn, W0n, cbn, Hn, 1, 128)
-        dt = time.perf_counter() - t0
-        out["oracle"] = {"seconds_one_cycle": dt, "channels_per_group": cpg,
-                         "seconds_one_cycle_all_channels_scaled": dt * mk / cpg}
     print(json.dumps(out), flush=True)
 
 

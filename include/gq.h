@@ -4,9 +4,9 @@
  * For one linear layer with input activations X (n tokens x d_in), end-loss gradients of the
  * layer output dl/dZ (n x d_out) and weights W, the library computes
  *
- *   J_k   = { m k, ..., m (k+1) - 1 },  m = d_out / g          (Algorithm 1, line 1)
- *   s_k   = 1/|J_k| * sum_{j in J_k} (dl/dz_j)^2                (Algorithm 1, line 2)
- *   H_k   = X^T Diag(s_k) X                                     (Algorithm 1, line 4; Section 3.2)
+ *   J_k   = { m k, ..., m (k+1) - 1 },  m = d_out / g          (Algorithm 1, grouping step)
+ *   s_k   = 1/|J_k| * sum_{j in J_k} (dl/dz_j)^2                (Algorithm 1, saliency step)
+ *   H_k   = X^T Diag(s_k) X                                     (Algorithm 1, Hessian step; Section 3.2)
  *   loss  = sum_k sum_{j in J_k} (w_j - what_j)^T H_k (w_j - what_j)          (Eq. 7)
  *
  * Conventions shared by every call
@@ -18,6 +18,9 @@
  *     ordered after the call on `stream`.
  *   - Return value: GQ_OK or a negative gq_status.  Invalid arguments are detected on the host
  *     before anything is launched; nothing is written in that case.
+ *   - Buffers a call writes (outputs, in/out arguments, workspaces) must not share memory with a buffer
+ *     the same call reads, nor with each other: overlapping ranges return GQ_ERR_INVALID_ARG.  Two
+ *     read-only arguments may be the same buffer.
  *   - Problems that can only be seen on the device (a pipeline wait that ran out of its time
  *     budget) are recorded in a per-device status word that gq_check() reads.
  *   - Tokens are rows: X is [n, ld_x] and dl/dZ is [n, ld_grad], both bf16, row-major.
@@ -35,7 +38,7 @@ extern "C" {
 
 typedef enum gq_status {
     GQ_OK = 0,
-    GQ_ERR_INVALID_ARG = -1,       /* null pointer, negative size, g < 1, d_out % g != 0, bad flags  */
+    GQ_ERR_INVALID_ARG = -1,       /* null pointer, negative size, g < 1, d_out % g != 0, bad flags, aliasing */
     GQ_ERR_ALIGNMENT = -2,         /* pointer or leading dimension not aligned as documented          */
     GQ_ERR_UNSUPPORTED_SHAPE = -3, /* size outside what the kernels index (see each call)             */
     GQ_ERR_WORKSPACE = -4,         /* workspace missing or smaller than the *_workspace_bytes() value */
@@ -54,7 +57,7 @@ const char *gq_status_string(int32_t status);
 int32_t gq_last_cuda_error(void);
 
 /*
- * Saliency: Algorithm 1, line 2, with the gradient scaling of Section 3.2 applied to the gradient
+ * Saliency: Algorithm 1, saliency step, with the gradient scaling of Section 3.2 applied to the gradient
  * before it is squared:
  *     s[k * ld_s + i] = (grad_scale^2 / m) * sum_{j = m k}^{m (k+1) - 1} grad[i * ld_grad + j]^2
  *
@@ -69,7 +72,7 @@ int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad,
                     float grad_scale, float *s, int64_t ld_s, void *stream);
 
 /*
- * Guided Hessian, one token chunk: Algorithm 1, line 4, streamed,
+ * Guided Hessian, one token chunk: Algorithm 1, Hessian step, streamed,
  *     H[k][a][b] += sum_{i < n} s[k * ld_s + i] * X[i * ld_x + a] * X[i * ld_x + b]
  * for every group k and every a <= b (the upper triangle including the diagonal).  No 1/n factor.
  *
@@ -112,7 +115,7 @@ size_t gq_hessian_workspace_bytes(int64_t n_max, int64_t d_in, int32_t g, uint32
 int32_t gq_hessian_finalize(float *H, int64_t d_in, int32_t g, void *stream);
 
 /*
- * Token-sharded accumulation over several GPUs: H_k is a sum over tokens (Algorithm 1, line 4), so every GPU
+ * Token-sharded accumulation over several GPUs: H_k is a sum over tokens (Algorithm 1, Hessian step), so every GPU
  * may run gq_hessian_accumulate on its own share of the tokens and the partial matrices are then added.
  * These two calls do that exchange with plain loads from the other GPUs' memory (peer access enabled by the
  * caller, e.g. through CUDA IPC or symmetric memory); no kernel waits for another GPU, the CALLER provides
@@ -163,7 +166,7 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
 size_t gq_objective_workspace_bytes(int64_t d_in, int64_t d_out, int32_t g);
 
 /*
- * The whole path for one layer with HOST inputs and outputs (Algorithm 1 lines 1, 2, 4 and Eq. 7):
+ * The whole path for one layer with HOST inputs and outputs (Algorithm 1's grouping, saliency and Hessian steps, and Eq. 7):
  * streams X and dl/dZ from host memory in chunks of `chunk` tokens, builds s and H on the device,
  * finalizes H, evaluates the objective and copies the results back.
  *
@@ -207,8 +210,12 @@ size_t gq_layer_host_arena_bytes(int64_t chunk, int64_t d_in, int64_t d_out, int
  *     order them on one stream or with events.  The array keeps what the last call wrote; every
  *     byte a call reads it has written itself first, so stale contents never leak into a result.
  *
- * Arguments, arithmetic and results are exactly those of gq_objective (W, W_hat, H, loss_out are the
- * caller's device buffers); for shapes within the limit both entry points return identical values.
+ * Arguments and arithmetic (delta as two bf16 terms, three tensor-core products, fp64 reduction in a
+ * fixed order) are those described for gq_objective; W, W_hat, H, loss_out are the caller's device
+ * buffers.  The kernel behind this entry point works on one 256 x 256 tile of H at a time, the one behind
+ * gq_objective on other units and, since version 0.2, with other operand types, so the two entry
+ * points agree to rounding (well inside the 1e-3 relative tolerance of the objective), not bit for bit.
+ * Repeated calls of this entry point on the same inputs do return identical bits.
  */
 int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, int64_t d_out,
                              const float *H, int32_t g, double *loss_out, void *stream);
@@ -256,7 +263,7 @@ size_t gq_cd_workspace_bytes(int64_t d_in, int64_t d_out, int32_t g);
 int32_t gq_check(void *stream, uint32_t *detail /* HOST, may be NULL */);
 
 /*
- * Codebook step of the layer-wise quantiser (Section 4.2, Eq. 8; Algorithm 2 lines 4 and 14): with the
+ * Codebook step of the layer-wise quantiser (Section 4.2, Eq. 8; the codebook steps of Algorithm 2): with the
  * assignment matrix P^(j) in {0,1}^{d_in x m} given by the codes of channel j (P_iq = 1 iff Q[j][i] == q),
  *     codebook[j] = (P^T H_k P + lambda I)^-1 P^T H_k w_j          for every channel j of every group k,
  * the minimiser of channel j's objective over its m codebook values for fixed codes (lambda is the small
@@ -320,8 +327,8 @@ uint64_t gq_launch_count(void);
  * Measurement aid (no counterpart in the paper).  The library's kernels, in launch order of a layer:
  */
 enum gq_kernel_id {
-    GQ_KERNEL_SALIENCY = 0,    /* Algorithm 1 line 2                                    */
-    GQ_KERNEL_HESSIAN = 1,     /* tensor-core H += X^T Diag(s_k) X, scaling fused (Algorithm 1 l. 4) */
+    GQ_KERNEL_SALIENCY = 0,    /* Algorithm 1, saliency step                                    */
+    GQ_KERNEL_HESSIAN = 1,     /* tensor-core H += X^T Diag(s_k) X, scaling fused (Algorithm 1, Hessian step) */
     GQ_KERNEL_MIRROR = 2,      /* gq_hessian_finalize                                    */
     GQ_KERNEL_SPLIT_DELTA = 3, /* W - W_hat -> bf16 hi/lo                                */
     GQ_KERNEL_GRAM_DOT = 4,    /* tensor-core Delta_k^T Delta_k contracted with H_k (Eq. 7) */

@@ -18,6 +18,19 @@
  * channel's codebook).  Inputs are fp32 bit patterns widened exactly; all
  * arithmetic is fp64.
  *
+ * How the sums of Eq. 10 are carried (derived from Eq. 10, not taken from the printed pseudo-code).
+ * Write Ht = diag(H)^-1 H and E = What - W.  Coordinate i needs  t_i = sum_{c != i} Ht_ic E_c  with the
+ * E_c of the moment at which i is visited: E_c already updated in this cycle for c < i, still the
+ * previous cycle's for c > i.  Split the sum at i:
+ *     t_i = sum_{c > i} Ht_ic E_c(old)  +  sum_{c < i} Ht_ic E_c(new).
+ * The first part is known before the cycle starts; it is formed for all i at once as
+ * B = StrictUpper(Ht) E.  The second part grows as the cycle proceeds: once coordinate c has been
+ * decided, Ht_ic E_c(new) is owed to every later coordinate i > c.  Paying that debt immediately, row
+ * by row, is the plain form (block size >= d_in).  With a block size b the debt of a coordinate is paid
+ * at once only to the later coordinates of its own block, and the whole block's debt to everything
+ * after the block is paid in one matrix product when the block is finished.  Each B_i has received
+ * exactly the same terms by the time coordinate i is visited, so the decisions do not depend on b.
+ *
  * Readings where the paper is silent or at odds with itself:
  *  - Round_j ties: the smaller codebook index wins.
  *  - Algorithms 3/4 write the in-loop correction as U_{(i+1):,i} with U the STRICT UPPER
@@ -45,8 +58,8 @@ static int32_t round_idx(double x, const float *cb, int32_t m)
 }
 
 /*
- * Algorithm 4 (CD with precomputation and lazy batch-updates), `cycles` cycles, block size b.
- * b >= d_in reproduces Algorithm 3 (no deferred corrections).
+ * Cyclic CD with the sums carried as described above (the scheme of Algorithm 4; with b >= d_in that of
+ * Algorithm 3), `cycles` cycles, block size b.
  * W_hat is read as the feasible starting point and overwritten; Q receives the codes.
  * Returns 0, or -1 on bad sizes / allocation failure.
  */
@@ -71,7 +84,7 @@ int gq_oracle_cd(const float *W, float *W_hat, int32_t *Q, const float *codebook
             for (int64_t i = 0; i < d_in; ++i)
                 for (int64_t j = 0; j < mk; ++j)
                     E[i * mk + j] = (double)W_hat[(k * mk + j) * d_in + i] - (double)W[(k * mk + j) * d_in + i];
-            /* line 3: B = StrictUpper(Htilde) (What - W) */
+            /* the part of every t_i that is known before the cycle: B = StrictUpper(Ht) E */
 #pragma omp parallel for schedule(static)
             for (int64_t r = 0; r < d_in; ++r)
                 for (int64_t j = 0; j < mk; ++j) {
@@ -82,7 +95,7 @@ int gq_oracle_cd(const float *W, float *W_hat, int32_t *Q, const float *codebook
             for (int64_t s = 0; s < d_in; s += b) {
                 const int64_t e = s + b < d_in ? s + b : d_in;
                 for (int64_t i = s; i < e; ++i) {
-                    /* line 6: round coordinate i of every channel */
+                    /* Eq. 10 for coordinate i of every channel: Round_j(W_ij - t_i) */
                     for (int64_t j = 0; j < mk; ++j) {
                         const int64_t ch = k * mk + j;
                         const double target = (double)W[ch * d_in + i] - B[i * mk + j];
@@ -91,11 +104,11 @@ int gq_oracle_cd(const float *W, float *W_hat, int32_t *Q, const float *codebook
                         W_hat[ch * d_in + i] = codebook[ch * m + q];
                         E[i * mk + j] = (double)codebook[ch * m + q] - (double)W[ch * d_in + i];
                     }
-                    /* line 7: correct the not-yet-visited coordinates of this block */
+                    /* coordinate i's debt to the later coordinates of its own block */
                     for (int64_t r = i + 1; r < e; ++r)
                         for (int64_t j = 0; j < mk; ++j) B[r * mk + j] += Ht[r * d_in + i] * E[i * mk + j];
                 }
-                /* line 9: deferred correction of all later coordinates by the whole block */
+                /* the finished block's debt to every coordinate after it, in one product */
 #pragma omp parallel for schedule(static)
                 for (int64_t r = e; r < d_in; ++r)
                     for (int64_t j = 0; j < mk; ++j) {

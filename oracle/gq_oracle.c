@@ -13,7 +13,7 @@
  *
  * Notation (paper, Section 2 "Preliminaries" and Section 3.2):
  *   n tokens, X in R^{n x d_in}, dl/dZ in R^{n x d_out}, g groups,
- *   J_k = {m k, ..., m (k+1) - 1} with m = d_out / g (0-based; Algorithm 1 line 1).
+ *   J_k = {m k, ..., m (k+1) - 1} with m = d_out / g (0-based; Algorithm 1, grouping step).
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -28,7 +28,7 @@ static double bf16_to_f64(uint16_t b)
 }
 
 /*
- * Algorithm 1 line 2 (and the averaged-squared-gradient form under Eq. 7):
+ * Algorithm 1, saliency step (and the averaged-squared-gradient form under Eq. 7):
  *   s_k[i] = 1/|J_k| * sum_{j in J_k} (grad_scale * dl/dZ[i][j])^2
  * grad_scale is the constant the paper multiplies gradients by (10^3 in its
  * experiments, Section 3.2); it is applied to the gradient before squaring.
@@ -54,7 +54,7 @@ int gq_oracle_saliency(const uint16_t *grad, int64_t n, int64_t d_out, int64_t l
 }
 
 /*
- * Algorithm 1 line 4:  H_k = X^T Diag(s_k) X, i.e.
+ * Algorithm 1, Hessian step:  H_k = X^T Diag(s_k) X, i.e.
  *   H_k[a][b] (+)= sum_{i=1..n} s_k[i] * X[i][a] * X[i][b]      for all a, b.
  * No 1/n factor (Section 3.2 writes the unguided case as H = X^T X).
  * The whole d_in x d_in matrix is computed entry by entry (no use of symmetry).
@@ -145,6 +145,73 @@ int gq_oracle_objective(const float *W, const float *What, int64_t d_in, int64_t
         total += lk;
     }
     loss[g] = total;
+    return 0;
+}
+
+/*
+ * Two consequences of the definition H_k = X^T Diag(s_k) X (Algorithm 1, Hessian step) that need only
+ * O(n d_in) work per group and can therefore be evaluated at full size, where the d_in x d_in matrix
+ * cannot: its diagonal and its action on a vector.  Both are ADDED to, token chunk after token chunk.
+ *
+ *   diag[k][a]   (+)= sum_i s_k[i] * X[i][a]^2                                (= H_k[a][a])
+ */
+int gq_oracle_hessian_diag(const uint16_t *X, int64_t n, int64_t d_in, int64_t ld_x,
+                           const double *s, int64_t ld_s, int32_t g, double *diag)
+{
+    if (g < 1 || d_in < 1 || ld_x < d_in || ld_s < n || n < 0) return -1;
+    for (int32_t k = 0; k < g; ++k) {
+        const double *sk = s + (int64_t)k * ld_s;
+        double *dk = diag + (int64_t)k * d_in;
+        /* the entries a are independent: threads take runs of 64 of them and walk the tokens in order */
+#pragma omp parallel for schedule(static)
+        for (int64_t a0 = 0; a0 < d_in; a0 += 64) {
+            const int64_t a1 = a0 + 64 < d_in ? a0 + 64 : d_in;
+            for (int64_t i = 0; i < n; ++i)
+                for (int64_t a = a0; a < a1; ++a) {
+                    const double x = bf16_to_f64(X[i * ld_x + a]);
+                    dk[a] += sk[i] * x * x;
+                }
+        }
+    }
+    return 0;
+}
+
+/*
+ *   out[k][v][a] (+)= sum_i s_k[i] * (sum_b X[i][b] V[v][b]) * X[i][a]        (= (H_k V[v])[a])
+ * V: [nv][d_in] fp64 probe vectors, out: [g][nv][d_in] fp64.  Returns 0, -1 on bad sizes, -2 if out of memory.
+ */
+int gq_oracle_hessian_apply(const uint16_t *X, int64_t n, int64_t d_in, int64_t ld_x,
+                            const double *s, int64_t ld_s, int32_t g, const double *V, int32_t nv,
+                            double *out)
+{
+    if (g < 1 || d_in < 1 || ld_x < d_in || ld_s < n || n < 0 || nv < 1) return -1;
+    if (n == 0) return 0;
+    double *y = (double *)malloc(sizeof(double) * (size_t)n * (size_t)nv);      /* y[v][i] = x_i . V[v] */
+    if (!y) return -2;
+    for (int32_t v = 0; v < nv; ++v) {
+#pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < n; ++i) {
+            double acc = 0.0;
+            for (int64_t b = 0; b < d_in; ++b) acc += bf16_to_f64(X[i * ld_x + b]) * V[(int64_t)v * d_in + b];
+            y[(int64_t)v * n + i] = acc;
+        }
+    }
+    for (int32_t k = 0; k < g; ++k) {
+        const double *sk = s + (int64_t)k * ld_s;
+        for (int32_t v = 0; v < nv; ++v) {
+            const double *yv = y + (int64_t)v * n;
+            double *ov = out + ((int64_t)k * nv + v) * d_in;
+#pragma omp parallel for schedule(static)
+            for (int64_t a0 = 0; a0 < d_in; a0 += 64) {
+                const int64_t a1 = a0 + 64 < d_in ? a0 + 64 : d_in;
+                for (int64_t i = 0; i < n; ++i) {
+                    const double wi = sk[i] * yv[i];
+                    for (int64_t a = a0; a < a1; ++a) ov[a] += wi * bf16_to_f64(X[i * ld_x + a]);
+                }
+            }
+        }
+    }
+    free(y);
     return 0;
 }
 

@@ -49,8 +49,10 @@ def _c():
         lib.gq_oracle_saliency.argtypes = [vp, i64, i64, i64, i32, dbl, vp, i64]
         lib.gq_oracle_hessian_accumulate.argtypes = [vp, i64, i64, i64, vp, i64, i32, vp]
         lib.gq_oracle_objective.argtypes = [vp, vp, i64, i64, vp, i32, vp]
+        lib.gq_oracle_hessian_diag.argtypes = [vp, i64, i64, i64, vp, i64, i32, vp]
+        lib.gq_oracle_hessian_apply.argtypes = [vp, i64, i64, i64, vp, i64, i32, vp, i32, vp]
         for f in (lib.gq_oracle_saliency, lib.gq_oracle_hessian_accumulate, lib.gq_oracle_objective,
-                  lib.gq_oracle_threads):
+                  lib.gq_oracle_hessian_diag, lib.gq_oracle_hessian_apply, lib.gq_oracle_threads):
             f.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -78,7 +80,7 @@ def _ptr(a: np.ndarray):
 
 
 def saliency(grad_bits: np.ndarray, g: int, grad_scale: float = 1.0, impl: str = "c") -> np.ndarray:
-    """Algorithm 1 line 2: ``s[k, i] = mean_{j in J_k} (grad_scale * grad[i, j])**2``."""
+    """Algorithm 1, saliency step: ``s[k, i] = mean_{j in J_k} (grad_scale * grad[i, j])**2``."""
     grad_bits = np.ascontiguousarray(grad_bits, dtype=np.uint16)
     n, d_out = grad_bits.shape
     if g < 1 or d_out % g:
@@ -94,7 +96,7 @@ def saliency(grad_bits: np.ndarray, g: int, grad_scale: float = 1.0, impl: str =
 
 
 def hessian(x_bits: np.ndarray, s: np.ndarray, H: np.ndarray | None = None, impl: str = "c") -> np.ndarray:
-    """Algorithm 1 line 4: ``H[k] (+)= X^T Diag(s[k]) X`` (full matrices, no 1/n).
+    """Algorithm 1, Hessian step: ``H[k] (+)= X^T Diag(s[k]) X`` (full matrices, no 1/n).
 
     Passing ``H`` accumulates into it (streaming over token chunks)."""
     x_bits = np.ascontiguousarray(x_bits, dtype=np.uint16)
@@ -115,6 +117,69 @@ def hessian(x_bits: np.ndarray, s: np.ndarray, H: np.ndarray | None = None, impl
     if rc:
         raise RuntimeError("gq_oracle_hessian_accumulate rc=%d" % rc)
     return H
+
+
+def _is_widened(x) -> bool:
+    """True for activations already widened to fp64 (``bf16_bits_to_f64`` of the bit patterns): the numpy
+    statements of the two O(n d_in) forms accept either, so a caller streaming large chunks widens once."""
+    return isinstance(x, np.ndarray) and x.dtype == np.float64
+
+
+def hessian_diag(x_bits: np.ndarray, s: np.ndarray, diag: np.ndarray | None = None, impl: str = "c") -> np.ndarray:
+    """The diagonal of Algorithm 1's guided Hessians straight from their definition,
+    ``diag[k, a] (+)= sum_i s[k, i] * X[i, a]**2`` -- O(n d_in) per group, so it can be formed for all
+    tokens of the large layers.  Passing ``diag`` accumulates into it (streaming over token chunks).
+    ``x_bits``: bf16 bit patterns, or (numpy statement only) the same values already widened to fp64."""
+    wide = _is_widened(x_bits)
+    x_bits = x_bits if wide else np.ascontiguousarray(x_bits, dtype=np.uint16)
+    s = np.ascontiguousarray(s, dtype=np.float64)
+    n, d_in = x_bits.shape
+    g = s.shape[0]
+    if s.shape[1] != n:
+        raise ValueError("s must be [g, n]")
+    if diag is None:
+        diag = np.zeros((g, d_in), dtype=np.float64)
+    assert diag.shape == (g, d_in) and diag.dtype == np.float64 and diag.flags.c_contiguous
+    if impl == "numpy":
+        x = x_bits if wide else bf16_bits_to_f64(x_bits)
+        diag += s @ (x * x)
+        return diag
+    if wide:
+        raise ValueError("the C loops take bf16 bit patterns")
+    rc = _c().gq_oracle_hessian_diag(_ptr(x_bits), n, d_in, d_in, _ptr(s), n, g, _ptr(diag))
+    if rc:
+        raise RuntimeError("gq_oracle_hessian_diag rc=%d" % rc)
+    return diag
+
+
+def hessian_apply(x_bits: np.ndarray, s: np.ndarray, V: np.ndarray, out: np.ndarray | None = None,
+                  impl: str = "c") -> np.ndarray:
+    """The guided Hessians applied to probe vectors without forming them,
+    ``out[k, v] (+)= X^T (s[k] * (X V[v]))`` ( = H_k V[v] by the definition of H_k) -- O(n d_in) per group
+    and probe.  ``V`` is ``[nv, d_in]``; passing ``out`` (``[g, nv, d_in]``) accumulates over token chunks."""
+    wide = _is_widened(x_bits)
+    x_bits = x_bits if wide else np.ascontiguousarray(x_bits, dtype=np.uint16)
+    s = np.ascontiguousarray(s, dtype=np.float64)
+    V = np.ascontiguousarray(V, dtype=np.float64)
+    n, d_in = x_bits.shape
+    g, nv = s.shape[0], V.shape[0]
+    if s.shape[1] != n or V.shape[1] != d_in:
+        raise ValueError("shape mismatch")
+    if out is None:
+        out = np.zeros((g, nv, d_in), dtype=np.float64)
+    assert out.shape == (g, nv, d_in) and out.dtype == np.float64 and out.flags.c_contiguous
+    if impl == "numpy":
+        x = x_bits if wide else bf16_bits_to_f64(x_bits)
+        y = x @ V.T                                                     # [n, nv]: x_i . V[v]
+        z = (s[:, :, None] * y[None, :, :]).transpose(1, 0, 2).reshape(n, g * nv)      # s[k, i] * y[i, v]
+        out += (x.T @ z).T.reshape(g, nv, d_in)
+        return out
+    if wide:
+        raise ValueError("the C loops take bf16 bit patterns")
+    rc = _c().gq_oracle_hessian_apply(_ptr(x_bits), n, d_in, d_in, _ptr(s), n, g, _ptr(V), nv, _ptr(out))
+    if rc:
+        raise RuntimeError("gq_oracle_hessian_apply rc=%d" % rc)
+    return out
 
 
 def objective(W: np.ndarray, W_hat: np.ndarray, H: np.ndarray, impl: str = "c") -> np.ndarray:

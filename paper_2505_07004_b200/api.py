@@ -102,9 +102,47 @@ def lib() -> ctypes.CDLL:
     return _lib
 
 
-def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
-    st = stream if stream is not None else torch.cuda.current_stream()
+def _stream_ptr(stream: Optional[torch.cuda.Stream], device=None) -> int:
+    st = stream if stream is not None else torch.cuda.current_stream(device)
     return int(st.cuda_stream)
+
+
+def _same_device(*named):
+    """The one CUDA device all given (name, tensor) pairs live on; ValueError if they differ.  The library
+    launches on the CURRENT device, so every wrapper makes this device current around its call: pointers of one
+    GPU must never reach kernels of another."""
+    dev = None
+    for name, t in named:
+        if t is None:
+            continue
+        d = t.device
+        if d.type != "cuda":
+            raise ValueError("%s must be a CUDA tensor" % name)
+        if dev is None:
+            dev, first = d, name
+        elif d != dev:
+            raise ValueError("%s is on %s but %s is on %s: all arguments of a call must live on one device"
+                             % (name, d, first, dev))
+    if dev is None:
+        raise ValueError("no device tensor given")
+    return dev
+
+
+class _on:
+    """Context: make `device` current for a library call and resolve the stream on that device."""
+
+    def __init__(self, device, stream):
+        if stream is not None and getattr(stream, "device", device) != device:
+            raise ValueError("stream belongs to %s, the tensors to %s" % (stream.device, device))
+        self.guard = torch.cuda.device(device)
+        self.device, self.stream = device, stream
+
+    def __enter__(self) -> int:
+        self.guard.__enter__()
+        return _stream_ptr(self.stream, self.device)
+
+    def __exit__(self, *exc):
+        return self.guard.__exit__(*exc)
 
 
 def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
@@ -139,7 +177,7 @@ def gq_launch_count() -> int:
 
 def gq_saliency(grad: torch.Tensor, g: int, grad_scale: float = 1.0, s: Optional[torch.Tensor] = None,
                 stream=None) -> torch.Tensor:
-    """``s[k, i] = grad_scale**2 / m * sum_{j in J_k} grad[i, j]**2`` (Algorithm 1, line 2)."""
+    """``s[k, i] = grad_scale**2 / m * sum_{j in J_k} grad[i, j]**2`` (Algorithm 1, saliency step)."""
     _dev(grad, torch.bfloat16, "grad")
     n, d_out, ld = _rows(grad, "grad")
     if s is None:
@@ -148,8 +186,8 @@ def gq_saliency(grad: torch.Tensor, g: int, grad_scale: float = 1.0, s: Optional
     _, s_n, ld_s = _rows(s, "s")
     if s.shape[0] != g or s_n < n:
         raise ValueError("s must be [g, >= n]")
-    rc = lib().gq_saliency(grad.data_ptr(), n, d_out, ld, g, float(grad_scale), s.data_ptr(), ld_s,
-                           _stream_ptr(stream))
+    with _on(_same_device(("grad", grad), ("s", s)), stream) as st:
+        rc = lib().gq_saliency(grad.data_ptr(), n, d_out, ld, g, float(grad_scale), s.data_ptr(), ld_s, st)
     if rc:
         raise GQError("gq_saliency", rc)
     return s
@@ -161,7 +199,7 @@ def gq_hessian_workspace_bytes(n_max: int, d_in: int, g: int, flags: int = 0) ->
 
 def gq_hessian_accumulate(X: torch.Tensor, s: torch.Tensor, H: torch.Tensor, workspace: torch.Tensor,
                           flags: int = 0, stream=None) -> torch.Tensor:
-    """``H[k] += X^T Diag(s[k]) X`` on the upper triangle (Algorithm 1, line 4), one token chunk."""
+    """``H[k] += X^T Diag(s[k]) X`` on the upper triangle (Algorithm 1, Hessian step), one token chunk."""
     _dev(X, torch.bfloat16, "X")
     _dev(s, torch.float32, "s")
     _dev(H, torch.float32, "H")
@@ -172,9 +210,9 @@ def gq_hessian_accumulate(X: torch.Tensor, s: torch.Tensor, H: torch.Tensor, wor
     s_n = n
     if tuple(H.shape) != (g, d_in, d_in) or not H.is_contiguous():
         raise ValueError("H must be a contiguous [g, d_in, d_in] tensor")
-    rc = lib().gq_hessian_accumulate(X.data_ptr(), n, d_in, ld_x, s.data_ptr(), ld_s, g, H.data_ptr(), flags,
-                                     workspace.data_ptr(), workspace.numel() * workspace.element_size(),
-                                     _stream_ptr(stream))
+    with _on(_same_device(("X", X), ("s", s), ("H", H), ("workspace", workspace)), stream) as st:
+        rc = lib().gq_hessian_accumulate(X.data_ptr(), n, d_in, ld_x, s.data_ptr(), ld_s, g, H.data_ptr(), flags,
+                                         workspace.data_ptr(), workspace.numel() * workspace.element_size(), st)
     if rc:
         raise GQError("gq_hessian_accumulate", rc)
     return H
@@ -185,7 +223,8 @@ def gq_hessian_finalize(H: torch.Tensor, stream=None) -> torch.Tensor:
     _dev(H, torch.float32, "H")
     if H.dim() != 3 or H.shape[1] != H.shape[2] or not H.is_contiguous():
         raise ValueError("H must be a contiguous [g, d_in, d_in] tensor")
-    rc = lib().gq_hessian_finalize(H.data_ptr(), H.shape[1], H.shape[0], _stream_ptr(stream))
+    with _on(_same_device(("H", H)), stream) as st:
+        rc = lib().gq_hessian_finalize(H.data_ptr(), H.shape[1], H.shape[0], st)
     if rc:
         raise GQError("gq_hessian_finalize", rc)
     return H
@@ -204,11 +243,20 @@ def _rank_pointers(H_ranks, d_in: int, g: int):
     return (ctypes.c_void_p * len(ptrs))(*ptrs)
 
 
+def _own_device(H_ranks, rank: int):
+    """Device of the calling rank's own matrix (peers may be given as raw pointers)."""
+    own = H_ranks[rank]
+    if not isinstance(own, torch.Tensor):
+        raise ValueError("H_ranks[rank] must be this process's own tensor")
+    return _same_device(("H_ranks[rank]", own))
+
+
 def gq_hessian_reduce_share(H_ranks, rank: int, d_in: int, g: int, stream=None) -> None:
     """Token-sharded accumulation, step 1: add rank ``rank``'s blocks of the upper triangle over all ranks'
     matrices (tensors of this process, or peers' device pointers as integers) into ``H_ranks[rank]``."""
     arr = _rank_pointers(H_ranks, d_in, g)
-    rc = lib().gq_hessian_reduce_share(arr, len(arr), rank, d_in, g, _stream_ptr(stream))
+    with _on(_own_device(H_ranks, rank), stream) as st:
+        rc = lib().gq_hessian_reduce_share(arr, len(arr), rank, d_in, g, st)
     if rc:
         raise GQError("gq_hessian_reduce_share", rc)
 
@@ -216,7 +264,8 @@ def gq_hessian_reduce_share(H_ranks, rank: int, d_in: int, g: int, stream=None) 
 def gq_hessian_gather_shares(H_ranks, rank: int, d_in: int, g: int, stream=None) -> None:
     """Token-sharded accumulation, step 2: copy the other ranks' reduced blocks into ``H_ranks[rank]``."""
     arr = _rank_pointers(H_ranks, d_in, g)
-    rc = lib().gq_hessian_gather_shares(arr, len(arr), rank, d_in, g, _stream_ptr(stream))
+    with _on(_own_device(H_ranks, rank), stream) as st:
+        rc = lib().gq_hessian_gather_shares(arr, len(arr), rank, d_in, g, st)
     if rc:
         raise GQError("gq_hessian_gather_shares", rc)
 
@@ -240,8 +289,10 @@ def gq_objective(W: torch.Tensor, W_hat: torch.Tensor, H: torch.Tensor, workspac
     if loss is None:
         loss = torch.empty(g + 1, dtype=torch.float64, device=W.device)
     _dev(loss, torch.float64, "loss")
-    rc = lib().gq_objective(W.data_ptr(), W_hat.data_ptr(), d_in, d_out, H.data_ptr(), g, loss.data_ptr(),
-                            workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    dev = _same_device(("W", W), ("W_hat", W_hat), ("H", H), ("loss", loss), ("workspace", workspace))
+    with _on(dev, stream) as st:
+        rc = lib().gq_objective(W.data_ptr(), W_hat.data_ptr(), d_in, d_out, H.data_ptr(), g, loss.data_ptr(),
+                                workspace.data_ptr(), workspace.numel() * workspace.element_size(), st)
     if rc:
         raise GQError("gq_objective", rc)
     return loss
@@ -271,19 +322,24 @@ def gq_layer_objective_host(X_host: torch.Tensor, grad_host: torch.Tensor, chunk
         raise ValueError("H_host must be a contiguous host fp32 [g, d_in, d_in] tensor")
     if not arena.is_cuda:
         raise ValueError("arena must be device memory")
-    rc = lib().gq_layer_objective_host(X_host.data_ptr(), grad_host.data_ptr(), n, chunk, d_in, d_out, g,
-                                       float(grad_scale), W_host.data_ptr(), W_hat_host.data_ptr(),
-                                       loss_host.data_ptr(), H_host.data_ptr() if H_host is not None else None,
-                                       arena.data_ptr(), arena.numel() * arena.element_size(), _stream_ptr(stream))
+    with _on(_same_device(("arena", arena)), stream) as st:
+        rc = lib().gq_layer_objective_host(X_host.data_ptr(), grad_host.data_ptr(), n, chunk, d_in, d_out, g,
+                                           float(grad_scale), W_host.data_ptr(), W_hat_host.data_ptr(),
+                                           loss_host.data_ptr(), H_host.data_ptr() if H_host is not None else None,
+                                           arena.data_ptr(), arena.numel() * arena.element_size(), st)
     if rc:
         raise GQError("gq_layer_objective_host", rc)
     return loss_host
 
 
-def gq_check(stream=None):
-    """Synchronises the stream and raises :class:`GQError` if a kernel recorded a device-side error."""
+def gq_check(stream=None, device=None):
+    """Synchronises the stream and raises :class:`GQError` if a kernel recorded a device-side error on `device`
+    (default: the stream's device, else the current one)."""
     detail = (ctypes.c_uint32 * 4)()
-    rc = lib().gq_check(_stream_ptr(stream), detail)
+    if device is None:
+        device = stream.device if stream is not None else torch.device("cuda", torch.cuda.current_device())
+    with _on(torch.device(device), stream) as st:
+        rc = lib().gq_check(st, detail)
     if rc:
         err = GQError("gq_check", rc)
         err.detail = tuple(int(v) for v in detail)
@@ -323,8 +379,8 @@ def gq_objective_noalloc(W: torch.Tensor, W_hat: torch.Tensor, H: torch.Tensor, 
     g = H.shape[0]
     if tuple(H.shape) != (g, d_in, d_in) or not H.is_contiguous() or loss.numel() != g + 1:
         raise ValueError("H must be contiguous [g, d_in, d_in] and loss must have g + 1 entries")
-    rc = lib().gq_objective_noalloc(W.data_ptr(), W_hat.data_ptr(), d_in, d_out, H.data_ptr(), g, loss.data_ptr(),
-                                    _stream_ptr(stream))
+    with _on(_same_device(("W", W), ("W_hat", W_hat), ("H", H), ("loss", loss)), stream) as st:
+        rc = lib().gq_objective_noalloc(W.data_ptr(), W_hat.data_ptr(), d_in, d_out, H.data_ptr(), g, loss.data_ptr(), st)
     if rc:
         raise GQError("gq_objective_noalloc", rc)
     return loss
@@ -353,9 +409,11 @@ def gq_cd_cycles(W: torch.Tensor, W_hat: torch.Tensor, codebook: torch.Tensor, H
     if Q is None:
         Q = torch.empty((d_out, d_in), dtype=torch.uint8, device=W.device)
     _dev(Q, torch.uint8, "Q")
-    rc = lib().gq_cd_cycles(W.data_ptr(), W_hat.data_ptr(), Q.data_ptr(), codebook.data_ptr(), codebook.shape[1], d_in,
-                            d_out, H.data_ptr(), g, int(cycles), workspace.data_ptr(),
-                            workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    dev = _same_device(("W", W), ("W_hat", W_hat), ("Q", Q), ("codebook", codebook), ("H", H), ("workspace", workspace))
+    with _on(dev, stream) as st:
+        rc = lib().gq_cd_cycles(W.data_ptr(), W_hat.data_ptr(), Q.data_ptr(), codebook.data_ptr(), codebook.shape[1],
+                                d_in, d_out, H.data_ptr(), g, int(cycles), workspace.data_ptr(),
+                                workspace.numel() * workspace.element_size(), st)
     if rc:
         raise GQError("gq_cd_cycles", rc)
     return W_hat, Q
@@ -364,7 +422,9 @@ def gq_cd_cycles(W: torch.Tensor, W_hat: torch.Tensor, codebook: torch.Tensor, H
 def gq_selftest_wait_timeout(budget_ms: int = 20, stream=None) -> None:
     """Launches the kernel whose wait runs out after ``budget_ms``; the next :func:`gq_check` raises
     ``GQ_ERR_TIMEOUT`` (site 99)."""
-    rc = lib().gq_selftest_wait_timeout(int(budget_ms), _stream_ptr(stream))
+    device = stream.device if stream is not None else torch.device("cuda", torch.cuda.current_device())
+    with _on(device, stream) as st:
+        rc = lib().gq_selftest_wait_timeout(int(budget_ms), st)
     if rc:
         raise GQError("gq_selftest_wait_timeout", rc)
 
@@ -392,9 +452,10 @@ def gq_lnq(W: torch.Tensor, Q: torch.Tensor, m: int, H: torch.Tensor, T: int, K:
         raise ValueError("H must be a contiguous [g, d_in, d_in] tensor")
     codebook = torch.empty((d_out, max(int(m), 1)), dtype=torch.float32, device=W.device)
     W_hat = torch.empty_like(W)
-    rc = lib().gq_lnq(W.data_ptr(), Q.data_ptr(), int(m), d_in, d_out, H.data_ptr(), g, int(T), int(K), float(lam),
-                  codebook.data_ptr(), W_hat.data_ptr(), workspace.data_ptr(),
-                  workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    with _on(_same_device(("W", W), ("Q", Q), ("H", H), ("workspace", workspace)), stream) as st:
+        rc = lib().gq_lnq(W.data_ptr(), Q.data_ptr(), int(m), d_in, d_out, H.data_ptr(), g, int(T), int(K), float(lam),
+                          codebook.data_ptr(), W_hat.data_ptr(), workspace.data_ptr(),
+                          workspace.numel() * workspace.element_size(), st)
     if rc:
         raise GQError("gq_lnq", rc)
     return W_hat, Q, codebook
@@ -421,9 +482,11 @@ def gq_codebook_update(W: torch.Tensor, Q: torch.Tensor, m: int, H: torch.Tensor
         _dev(W_hat, torch.float32, "W_hat")
         if W_hat.shape != W.shape or not W_hat.is_contiguous():
             raise ValueError("W_hat must be contiguous [d_out, d_in]")
-    rc = lib().gq_codebook_update(W.data_ptr(), Q.data_ptr(), int(m), d_in, d_out, H.data_ptr(), g, float(lam),
-                                  codebook.data_ptr(), W_hat.data_ptr() if W_hat is not None else None,
-                                  workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    dev = _same_device(("W", W), ("Q", Q), ("H", H), ("codebook", codebook), ("W_hat", W_hat), ("workspace", workspace))
+    with _on(dev, stream) as st:
+        rc = lib().gq_codebook_update(W.data_ptr(), Q.data_ptr(), int(m), d_in, d_out, H.data_ptr(), g, float(lam),
+                                      codebook.data_ptr(), W_hat.data_ptr() if W_hat is not None else None,
+                                      workspace.data_ptr(), workspace.numel() * workspace.element_size(), st)
     if rc:
         raise GQError("gq_codebook_update", rc)
     return codebook, W_hat

@@ -1,4 +1,4 @@
-"""Hooks that run Algorithm 1 (lines 2-4) on a PyTorch model: plumbing around the library calls.
+"""Hooks that run Algorithm 1 (saliency and Hessian steps) on a PyTorch model: plumbing around the library calls.
 
 The method needs, per linear layer, the end-loss gradients of the layer's outputs (only their group-wise
 mean squares s_k are kept: O(n g) per layer, Section 3.2) and the layer's inputs.  As in the paper this takes

@@ -1,4 +1,4 @@
-// Codebook step of the layer-wise quantiser (Section 4.2, Eq. 8; Algorithm 2 lines 4 and 14): for every
+// Codebook step of the layer-wise quantiser (Section 4.2, Eq. 8; the codebook steps of Algorithm 2): for every
 // output channel j of group k, with the assignment matrix P in {0,1}^{d_in x m} given by the codes Q,
 //
 //     c^(j) = (P^T H_k P + lambda I)^-1  P^T H_k w_j .

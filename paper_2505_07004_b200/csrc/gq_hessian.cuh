@@ -1,4 +1,4 @@
-// Guided Hessian of Algorithm 1 line 4 with the row scaling fused into the operand path:
+// Guided Hessian of Algorithm 1, Hessian step with the row scaling fused into the operand path:
 //
 //     H_k[a][b] += sum_i  (s_k[i] * X[i][a]) * X[i][b]          for a <= b, all groups k
 //

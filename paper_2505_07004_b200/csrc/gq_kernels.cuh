@@ -29,7 +29,7 @@ __device__ __forceinline__ uint4 float_to_bf16x8(const float (&f)[8])
 }
 
 // ------------------------------------------------------------------------------------------------
-// Algorithm 1 line 2.  One warp per (token, group) segment of m = d_out / g gradients:
+// Algorithm 1, saliency step.  One warp per (token, group) segment of m = d_out / g gradients:
 //   s[k][i] = (grad_scale^2 / m) * sum_j grad[i][m k + j]^2.
 // A lane reads 16 bytes (8 bf16) per load and issues eight (long segments) or four loads (the last ones
 // predicated off at the end of the segment) before it touches the first result.

@@ -87,6 +87,20 @@ PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
 inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// True if the byte ranges [a, a + na) and [b, b + nb) share a byte (empty ranges never do).
+inline bool overlaps(const void *a, size_t na, const void *b, size_t nb)
+{
+    if (!a || !b || na == 0 || nb == 0) return false;
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return a0 < b0 + nb && b0 < a0 + na;
+}
+// Bytes spanned by `rows` rows of `width` elements with leading dimension `ld` (elements of `elem` bytes).
+inline size_t span_bytes(int64_t rows, int64_t width, int64_t ld, size_t elem)
+{
+    if (rows <= 0 || width <= 0) return 0;
+    return (static_cast<size_t>(rows - 1) * static_cast<size_t>(ld) + static_cast<size_t>(width)) * elem;
+}
+
 int32_t device_info(DeviceInfo **out)
 {
     int dev = 0;
@@ -252,6 +266,40 @@ int32_t check_layer_shape(int64_t d_in, int64_t d_out, int32_t g, bool need_out)
     return GQ_OK;
 }
 
+struct ByteRange {
+    const void *p;
+    size_t bytes;
+};
+// No written range may share a byte with a read-only range or with another written range.
+template <int NW, int NR>
+int32_t check_disjoint(const ByteRange (&written)[NW], const ByteRange (&read_only)[NR])
+{
+    for (int a = 0; a < NW; ++a) {
+        for (int b = 0; b < NR; ++b)
+            if (overlaps(written[a].p, written[a].bytes, read_only[b].p, read_only[b].bytes)) return GQ_ERR_INVALID_ARG;
+        for (int b = a + 1; b < NW; ++b)
+            if (overlaps(written[a].p, written[a].bytes, written[b].p, written[b].bytes)) return GQ_ERR_INVALID_ARG;
+    }
+    return GQ_OK;
+}
+
+// gq_objective / gq_objective_noalloc: the outputs (loss, scratch) must not share memory with W, W_hat, H or each
+// other (W and W_hat may be the same buffer: both are only read).
+int32_t check_objective_aliasing(const float *W, const float *W_hat, int64_t d_in, int64_t d_out, const float *H, int32_t g,
+                                 const double *loss_out, const void *workspace, size_t ws_bytes)
+{
+    const size_t w_bytes = static_cast<size_t>(d_out) * d_in * 4, h_bytes = static_cast<size_t>(g) * d_in * d_in * 4;
+    const size_t l_bytes = static_cast<size_t>(g + 1) * 8;
+    const void *outs[2] = {loss_out, workspace};
+    const size_t out_bytes[2] = {l_bytes, ws_bytes};
+    for (int o = 0; o < 2; ++o)
+        if (overlaps(outs[o], out_bytes[o], W, w_bytes) || overlaps(outs[o], out_bytes[o], W_hat, w_bytes) ||
+            overlaps(outs[o], out_bytes[o], H, h_bytes))
+            return GQ_ERR_INVALID_ARG;
+    if (overlaps(loss_out, l_bytes, workspace, ws_bytes)) return GQ_ERR_INVALID_ARG;
+    return GQ_OK;
+}
+
 // Scratch of gq_hessian_accumulate: the split saliency words, 8 bytes per (pair of groups, token).
 size_t hessian_ws_bytes(int64_t n_max, int64_t, int32_t g)
 {
@@ -359,6 +407,7 @@ int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad,
     if (n == 0) return GQ_OK;              // nothing to read or write: pointers are not looked at
     if (!grad || !s) return GQ_ERR_INVALID_ARG;
     if (!aligned(grad, 16) || !aligned(s, 4)) return GQ_ERR_ALIGNMENT;
+    if (overlaps(grad, span_bytes(n, d_out, ld_grad, 2), s, span_bytes(g, n, ld_s, 4))) return GQ_ERR_INVALID_ARG;
     DeviceInfo *di;
     if (int32_t rc = device_info(&di)) return rc;
     const int m = static_cast<int>(d_out / g);
@@ -395,6 +444,14 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
     if (!aligned(X, 16) || !aligned(H, 16) || !aligned(s, 4)) return GQ_ERR_ALIGNMENT;
     if (!workspace || workspace_bytes < hessian_ws_bytes(n, d_in, g)) return GQ_ERR_WORKSPACE;
     if (!aligned(workspace, 1024)) return GQ_ERR_ALIGNMENT;
+    {
+        // the output and the scratch must not share memory with an input or with each other
+        const size_t h_bytes = static_cast<size_t>(g) * d_in * d_in * 4, ws_bytes = hessian_ws_bytes(n, d_in, g);
+        const size_t x_bytes = span_bytes(n, d_in, ld_x, 2), s_bytes = span_bytes(g, n, ld_s, 4);
+        if (overlaps(H, h_bytes, X, x_bytes) || overlaps(H, h_bytes, s, s_bytes) || overlaps(H, h_bytes, workspace, ws_bytes) ||
+            overlaps(workspace, ws_bytes, X, x_bytes) || overlaps(workspace, ws_bytes, s, s_bytes))
+            return GQ_ERR_INVALID_ARG;
+    }
     DeviceInfo *di;
     if (int32_t rc = device_info(&di)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -514,6 +571,7 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     const ObjectiveLayout L = objective_layout(d_in, d_out, g);
     if (!workspace || workspace_bytes < L.total) return GQ_ERR_WORKSPACE;
     if (!aligned(workspace, 1024)) return GQ_ERR_ALIGNMENT;
+    if (int32_t rc = check_objective_aliasing(W, W_hat, d_in, d_out, H, g, loss_out, workspace, L.total)) return rc;
     DeviceInfo *di;
     if (int32_t rc = device_info(&di)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -601,6 +659,7 @@ int32_t gq_objective_noalloc(const float *W, const float *W_hat, int64_t d_in, i
     const int tiles = tiles_for(d_in);
     if (d_in * d_out > GQ_NOALLOC_MAX_WEIGHTS || static_cast<int64_t>(tiles) * g > GQ_NOALLOC_MAX_UNITS)
         return GQ_ERR_UNSUPPORTED_SHAPE;       // larger layers must use gq_objective with a caller workspace
+    if (int32_t rc = check_objective_aliasing(W, W_hat, d_in, d_out, H, g, loss_out, nullptr, 0)) return rc;
     DeviceInfo *di;
     if (int32_t rc = device_info(&di)) return rc;
 
@@ -687,6 +746,13 @@ int32_t gq_cd_cycles(const float *W, float *W_hat, uint8_t *Q, const float *code
     const CdLayout L = cd_layout(d_in, d_out, g);
     if (!workspace || workspace_bytes < L.total) return GQ_ERR_WORKSPACE;
     if (!aligned(workspace, 1024)) return GQ_ERR_ALIGNMENT;
+    {
+        const size_t w4 = static_cast<size_t>(d_out) * d_in * 4;
+        const ByteRange wr[3] = {{W_hat, w4}, {Q, static_cast<size_t>(d_out) * d_in}, {workspace, L.total}};
+        const ByteRange ro[3] = {{W, w4}, {codebook, static_cast<size_t>(d_out) * m * 4},
+                                 {H, static_cast<size_t>(g) * d_in * d_in * 4}};
+        if (int32_t rc = check_disjoint(wr, ro)) return rc;
+    }
     DeviceInfo *di;
     if (int32_t rc = device_info(&di)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -802,6 +868,12 @@ int32_t gq_codebook_update(const float *W, const uint8_t *Q, int32_t m, int64_t 
     const CodebookLayout L = codebook_layout(d_in, d_out, g, m);
     if (!workspace || workspace_bytes < L.total) return GQ_ERR_WORKSPACE;
     if (!aligned(workspace, 1024)) return GQ_ERR_ALIGNMENT;
+    {
+        const size_t w4 = static_cast<size_t>(d_out) * d_in * 4;
+        const ByteRange wr[3] = {{codebook, static_cast<size_t>(d_out) * m * 4}, {W_hat, W_hat ? w4 : 0}, {workspace, L.total}};
+        const ByteRange ro[3] = {{W, w4}, {Q, static_cast<size_t>(d_out) * d_in}, {H, static_cast<size_t>(g) * d_in * d_in * 4}};
+        if (int32_t rc = check_disjoint(wr, ro)) return rc;
+    }
     DeviceInfo *di;
     if (int32_t rc = device_info(&di)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -942,6 +1014,13 @@ int32_t gq_lnq(const float *W, uint8_t *Q, int32_t m, int64_t d_in, int64_t d_ou
         return (m < 1) ? GQ_ERR_INVALID_ARG : GQ_ERR_UNSUPPORTED_SHAPE;
     }
     if (!workspace || workspace_bytes < need) return GQ_ERR_WORKSPACE;
+    {
+        const size_t w4 = static_cast<size_t>(d_out) * d_in * 4;
+        const ByteRange wr[4] = {{Q, static_cast<size_t>(d_out) * d_in}, {codebook, static_cast<size_t>(d_out) * m * 4},
+                                 {W_hat, w4}, {workspace, need}};
+        const ByteRange ro[2] = {{W, w4}, {H, static_cast<size_t>(g) * d_in * d_in * 4}};
+        if (int32_t rc = check_disjoint(wr, ro)) return rc;
+    }
     for (int32_t t = 0; t < T; ++t) {
         if (int32_t rc = gq_codebook_update(W, Q, m, d_in, d_out, H, g, lambda, codebook, W_hat, workspace,
                                             workspace_bytes, stream))
@@ -1025,7 +1104,7 @@ size_t gq_layer_host_arena_bytes(int64_t chunk, int64_t d_in, int64_t d_out, int
     total += round_up(static_cast<size_t>(g) * chunk * 4, 1024);             // s
     total += round_up(static_cast<size_t>(g) * d_in * d_in * 4, 1024);       // H
     total += 2 * round_up(static_cast<size_t>(d_out) * d_in * 4, 1024);      // W, W_hat
-    total += 1024;                                                           // loss
+    total += round_up(static_cast<size_t>(g + 1) * sizeof(double), 1024);    // loss: g + 1 fp64 values
     total += hessian_ws_bytes(chunk, d_in, g);
     total += objective_layout(d_in, d_out, g).total;
     return total;
@@ -1057,7 +1136,7 @@ int32_t gq_layer_objective_host(const void *X_host, const void *grad_host, int64
     const size_t w_bytes = static_cast<size_t>(d_out) * d_in * 4;
     float *W = reinterpret_cast<float *>(take(w_bytes));
     float *What = reinterpret_cast<float *>(take(w_bytes));
-    double *loss = reinterpret_cast<double *>(take(1024));
+    double *loss = reinterpret_cast<double *>(take(static_cast<size_t>(g + 1) * sizeof(double)));
     const size_t hws_bytes = hessian_ws_bytes(chunk, d_in, g);
     void *hws = take(hws_bytes);
     const size_t ows_bytes = objective_layout(d_in, d_out, g).total;

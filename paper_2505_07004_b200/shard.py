@@ -4,7 +4,7 @@ Default: the path shards over independent layers, one per rank, with no data-pat
 computes Hessians of different layers / groups on different GPUs, Section 3.2 and Appendix C); the only
 communication is the reduction of timings and of per-rank scalar results.
 
-Token sharding of ONE layer (H_k is a sum over tokens, Algorithm 1 line 4): every rank accumulates the chunks
+Token sharding of ONE layer (H_k is a sum over tokens, Algorithm 1, Hessian step): every rank accumulates the chunks
 `chunks_for_rank` gives it into its own H, then `exchange_hessian` adds the partial matrices with the library's
 reduce / gather kernels over peer memory, the ranks meeting at host barriers in between."""
 from __future__ import annotations

@@ -55,6 +55,15 @@ def test_workspace_sizes(L):
     assert L.gq_objective_workspace_bytes(4096, 24, 6) == 0            # (d_out / g) % 8 != 0
     assert L.gq_layer_host_arena_bytes(0, 4096, 4096, 4) == 0
     assert L.gq_layer_host_arena_bytes(8192, 4096, 4096, 4) > 4 * 4096 * 4096 * 4
+    # the loss slot holds g + 1 fp64 values rounded up to 1 KiB: 1 KiB for g = 64, 2 KiB for g = 128
+    r1k = lambda b: (b + 1023) // 1024 * 1024
+
+    def loss_slot(g, chunk=64, d_in=64, d_out=1024):
+        rest = (2 * r1k(chunk * d_in * 2) + 2 * r1k(chunk * d_out * 2) + r1k(g * chunk * 4) + r1k(g * d_in * d_in * 4)
+                + 2 * r1k(d_out * d_in * 4) + L.gq_hessian_workspace_bytes(chunk, d_in, g, 0)
+                + L.gq_objective_workspace_bytes(d_in, d_out, g))
+        return L.gq_layer_host_arena_bytes(chunk, d_in, d_out, g) - rest
+    assert loss_slot(64) == 1024 and loss_slot(128) == 2048
 
 
 def test_host_side_validation_needs_no_gpu(L):
@@ -84,6 +93,52 @@ def test_host_side_validation_needs_no_gpu(L):
     assert L.gq_objective(p16, p16, 64, 64, p16, 2, p16, p16, 16, None) == WS
     assert L.gq_objective(None, p16, 64, 64, p16, 2, p16, p16, 1 << 20, None) == INVALID
     assert L.gq_kernel_timing_read(None, None) == INVALID
+
+
+def test_aliasing_between_outputs_and_inputs_is_rejected(L):
+    """A buffer a call writes may not overlap one it reads (or another one it writes): GQ_ERR_INVALID_ARG on the
+    host, before any launch.  Two read-only arguments may alias."""
+    buf = (ctypes.c_uint8 * (1 << 20))()
+    base = (ctypes.addressof(buf) + 1023) // 1024 * 1024
+    INVALID, WS = -1, -4
+    # saliency: grad [4, 64] bf16 = 512 bytes, s [2, 4] fp32 = 32 bytes
+    assert L.gq_saliency(base, 4, 64, 64, 2, 1.0, base + 496, 4, None) == INVALID       # s inside grad's last row
+    assert L.gq_saliency(base + 16, 4, 64, 64, 2, 1.0, base, 4, None) == INVALID        # grad starts inside s
+    # hessian: X [4, 64] = 512 B, s [2, 4] = 32 B, H [2, 64, 64] = 32 KiB, workspace 1 KiB
+    X, s_, H, ws = base, base + 1024, base + 2048, base + 65536
+    assert L.gq_hessian_accumulate(X, 4, 64, 64, s_, 4, 2, X, 0, ws, 1024, None) == INVALID          # H over X
+    assert L.gq_hessian_accumulate(X, 4, 64, 64, H + 64, 4, 2, H, 0, ws, 1024, None) == INVALID      # s inside H
+    assert L.gq_hessian_accumulate(X, 4, 64, 64, s_, 4, 2, H, 0, H + 1024, 1024, None) == INVALID    # workspace inside H
+    assert L.gq_hessian_accumulate(X, 4, 64, 64, s_, 4, 2, H, 0, X, 1024, None) == INVALID           # workspace over X
+    # objective: W, W_hat [64, 64] fp32 = 16 KiB each, H [2, 64, 64] = 32 KiB, loss 24 B
+    need = L.gq_objective_workspace_bytes(64, 64, 2)
+    W, Wh, Hh, loss, ows = base, base + 16384, base + 32768, base + 65536, base + 131072
+    assert need > 0 and need < (1 << 20) - 131072 - 1024
+    assert L.gq_objective(W, Wh, 64, 64, Hh, 2, W + 8, ows, need, None) == INVALID                   # loss inside W
+    assert L.gq_objective(W, Wh, 64, 64, Hh, 2, loss, Hh, need, None) == INVALID                     # workspace over H
+    assert L.gq_objective(W, Wh, 64, 64, Hh, 2, ows + 16, ows, need, None) == INVALID                # loss inside workspace
+    assert L.gq_objective(W, Wh, 64, 64, Hh, 2, loss, ows, need - 1, None) == WS                     # size check first
+    assert L.gq_objective_noalloc(W, Wh, 64, 64, Hh, 2, Hh + 8, None) == INVALID                     # loss inside H
+
+
+def test_binding_refuses_tensors_on_different_devices():
+    """The library launches on the current device; the binding makes the tensors' device current and refuses
+    arguments that live on different GPUs before anything is launched."""
+    import types
+    import torch
+    t0 = types.SimpleNamespace(device=torch.device("cuda", 0))
+    t1 = types.SimpleNamespace(device=torch.device("cuda", 1))
+    host = types.SimpleNamespace(device=torch.device("cpu"))
+    assert libgq._same_device(("X", t0), ("H", t0), ("W_hat", None)) == torch.device("cuda", 0)
+    with pytest.raises(ValueError, match="one device"):
+        libgq._same_device(("X", t0), ("H", t1))
+    with pytest.raises(ValueError, match="CUDA tensor"):
+        libgq._same_device(("X", host))
+    with pytest.raises(ValueError):
+        libgq._same_device(("W_hat", None))
+    stream1 = types.SimpleNamespace(device=torch.device("cuda", 1), cuda_stream=0)
+    with pytest.raises(ValueError, match="stream belongs"):
+        libgq._on(torch.device("cuda", 0), stream1)
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

@@ -28,11 +28,54 @@ def test_hand_example():
         if line.startswith("#") or not line.strip():
             continue
         name, rest = line.split(None, 1)
-        w, start, after, _targets = [np.array(p.split(), dtype=np.float64) for p in rest.split("|")]
+        w, start, after, targets = [np.array(p.split(), dtype=np.float64) for p in rest.split("|")]
         for fn in (lambda *a: cdo.cd(*a, 1, 128), lambda *a: cdo.cd_rowwise(*a, 1), lambda *a: cdo.cd_naive(*a, 1)):
             What, Q = fn(w[None].astype(np.float32), start[None].astype(np.float32), cb, H)
             assert np.array_equal(What[0], after.astype(np.float32)), name
             assert np.array_equal(Q[0], after.astype(np.int32)), name
+        # the arguments of Round_j written out by hand in the file: coordinate 1 sees the starting point,
+        # coordinate 2 sees coordinate 1 already updated
+        cur = start.copy()
+        for i in range(2):
+            t, mag = cdo.coordinate_target(w, cur, H[0], i)
+            assert abs(t - targets[i]) <= 1e-12, (name, i, t)
+            assert abs(mag - (abs(w[i]) + 0.5 * abs(cur[1 - i] - w[1 - i]))) <= 1e-12, (name, i, mag)
+            cur[i] = after[i]
+
+
+def test_coordinate_target_is_the_minimiser_of_the_one_coordinate_quadratic():
+    """Eq. 10 before rounding: with every other coordinate of the channel held fixed, the channel objective as a
+    function of the value t of coordinate i is a parabola; its vertex, found here from three evaluations of the
+    objective alone (no algebra on H), is what coordinate_target must return.  The second return value is the
+    sum of the magnitudes of the terms, re-added here one by one."""
+    rng = np.random.default_rng(11)
+    for trial in range(20):
+        d = int(rng.integers(2, 9))
+        A = rng.standard_normal((d + 3, d))
+        Hk = A.T @ A
+        w = rng.standard_normal(d)
+        what = rng.standard_normal(d)
+        i = int(rng.integers(0, d))
+
+        def f(t):
+            trial_w = what.copy()
+            trial_w[i] = t
+            return cdo.channel_objective(trial_w - w, Hk)
+
+        fm, f0, fp = f(-1.0), f(0.0), f(1.0)
+        vertex = 0.5 * (fm - fp) / (fm - 2.0 * f0 + fp)
+        t, mag = cdo.coordinate_target(w, what, Hk, i)
+        assert abs(t - vertex) <= 1e-9 * max(1.0, abs(vertex)), (trial, t, vertex)
+        assert f(t) <= min(f(t + 1e-3), f(t - 1e-3))
+        expect_mag = abs(w[i])
+        for c in range(d):
+            if c != i:
+                expect_mag += abs(Hk[i, c] / Hk[i, i] * (what[c] - w[c]))
+        assert abs(mag - expect_mag) <= 1e-12 * expect_mag
+    # a feature that never fired: the target is the weight itself
+    Hk = np.diag([1.0, 0.0, 2.0])
+    t, mag = cdo.coordinate_target(np.array([0.3, -0.7, 0.1]), np.array([1.0, 1.0, 1.0]), Hk, 1)
+    assert t == -0.7 and mag == 0.7
 
 
 @pytest.mark.parametrize("seed,d_in,d_out,g,m,b", [(0, 24, 8, 2, 4, 8), (1, 37, 6, 3, 8, 16), (2, 16, 4, 1, 2, 5),
@@ -152,3 +195,47 @@ def test_lnq_descends():
         assert np.all(f_prev <= f_c * (1 + 1e-12))           # CD
     What, Qf, cf = cdo.lnq(W, Q0, H, 4, T=3, K=2, b=16)
     assert np.all(per_channel(What) <= f_prev * (1 + 1e-5))
+
+
+def test_lnq_is_algorithm_2_in_order():
+    """Algorithm 2: T times (codebook step, then K CD cycles), then one more codebook step.  lnq() must equal that
+    sequence composed here by hand from codebook_update and cd, bit for bit, and every deviation from the order
+    (no final codebook step, CD before the codebook step, one round fewer) must give another result on this
+    problem."""
+    W, W0, cb, H = make_problem(12, 40, 8, 2, 4, n=160)
+    _, Q0 = cdo.round_to_codebook(W, cb)
+    m, T, K, b = 4, 2, 2, 16
+
+    def cstep(Q):
+        c = cdo.codebook_update(W, Q, H, m).astype(np.float32)
+        return c, np.take_along_axis(c, Q, axis=1)
+
+    Q = Q0.copy()
+    for _ in range(T):
+        c, What = cstep(Q)
+        What, Q = cdo.cd(W, What, c, H, K, b)
+    Q_before_final, What_before_final, c_before_final = Q, What, c
+    c, What = cstep(Q)
+    got = cdo.lnq(W, Q0, H, m, T=T, K=K, b=b)
+    assert np.array_equal(got[1], Q) and np.array_equal(got[0], What) and np.array_equal(got[2], c)
+    # without the final codebook step the codebook (and W_hat) would be the previous round's
+    assert not np.array_equal(got[2], c_before_final)
+    assert not np.array_equal(got[0], What_before_final)
+    # the final step can only lower every channel's objective, and lowers some
+    mk = W.shape[0] // H.shape[0]
+    f = lambda Wh: np.array([cdo.channel_objective(Wh[j].astype(np.float64) - W[j], H[j // mk].astype(np.float64))
+                             for j in range(W.shape[0])])
+    assert np.all(f(got[0]) <= f(What_before_final) * (1 + 1e-5)) and np.any(f(got[0]) < f(What_before_final))
+    # CD first, codebook step second (the wrong order) ends elsewhere
+    Qw, cw = Q0.copy(), cb.copy()
+    Whw = np.take_along_axis(cw, Qw, axis=1)
+    for _ in range(T):
+        Whw, Qw = cdo.cd(W, Whw, cw, H, K, b)
+        cw, Whw = cstep(Qw)
+    assert not (np.array_equal(Qw, got[1]) and np.array_equal(cw, got[2]))
+    # T - 1 rounds end elsewhere, T = 0 is the codebook step alone
+    fewer = cdo.lnq(W, Q0, H, m, T=T - 1, K=K, b=b)
+    assert not np.array_equal(fewer[2], got[2])
+    only = cdo.lnq(W, Q0, H, m, T=0, K=K, b=b)
+    c0, What0 = cstep(Q0)
+    assert np.array_equal(only[1], Q0) and np.array_equal(only[2], c0) and np.array_equal(only[0], What0)

@@ -1,9 +1,15 @@
 """GPU parity: libgq (through the C-ABI binding) against the CPU fp64 oracle, same seeded inputs.
 
-Tolerances (stated by the benchmark spec for this path):
+Tolerances of this path:
   saliency   |s - s_o| <= 1e-4 * |s_o| per element (plus a floor of 1e-4 * max|s_o| * 1e-6 for zeros)
   Hessian    ||H_k - H_k_o||_F <= 5e-3 ||H_k_o||_F   and   max|H_k - H_k_o| <= 1e-2 max|H_k_o|
+             and, entry by entry, |H_k - H_k_o|[a][b] <= 3e-3 sqrt(H_k_o[a][a] H_k_o[b][b])
   objective  |loss - loss_o| <= 1e-3 |loss_o|
+The entry-wise bound does not depend on the scale of a feature (the first two are set by the few outlier
+features): the only rounding of the Hessian kernel that is not of fp32 size is the one bf16 rounding of each
+product s_k[i] X[i][a], a relative error of at most 2^-9, so
+|error of H[a][b]| <= 2^-9 sum_i s_i |X[i][a]| |X[i][b]| <= 2^-9 sqrt(H[a][a] H[b][b]) (Cauchy-Schwarz) = 1.95e-3 of
+that geometric mean; 3e-3 leaves room for the two-term saliency (2^-17) and fp32 accumulation.
 """
 import numpy as np
 import pytest
@@ -15,7 +21,7 @@ from paper_2505_07004_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
-S_RTOL, H_FRO, H_MAX, L_RTOL = 1e-4, 5e-3, 1e-2, 1e-3
+S_RTOL, H_FRO, H_MAX, H_ENTRY, L_RTOL = 1e-4, 5e-3, 1e-2, 3e-3, 1e-3
 
 
 @pytest.fixture(scope="module")
@@ -41,6 +47,12 @@ def check_H(H_gpu, H_ref, upper_only=False):
         fro = np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300)
         mx = np.abs(a - b).max() / max(np.abs(b).max(), 1e-300)
         assert fro <= H_FRO and mx <= H_MAX, "group %d: rel Frobenius %.3e, max-elem %.3e" % (k, fro, mx)
+        # scale-free companion: every entry against the geometric mean of its two diagonal entries
+        dg = np.sqrt(np.maximum(np.diag(H_ref[k]), 0.0))
+        scale = np.outer(dg, dg)
+        excess = np.abs(a - b) - H_ENTRY * scale
+        assert np.all(excess <= 1e-30), "group %d: entry %s off by %.3e of sqrt(H_aa H_bb)" % (
+            k, np.unravel_index(np.argmax(excess), excess.shape), (np.abs(a - b) / np.maximum(scale, 1e-300)).max())
 
 
 def check_loss(loss_gpu, loss_ref):
@@ -286,19 +298,19 @@ def test_large_shapes_token_prefix(dev, name, prefix):
         torch.cuda.empty_cache()
 
 
-@pytest.mark.parametrize("name,g,n_tokens,s_chunks", [
+@pytest.mark.parametrize("name,g,n_tokens,_unused", [
     ("c1_7b_attn", 4, None, None),      # the workload bench.py times, in full: 131072 tokens, 16 chunks
-    ("c2_7b_down", 4, None, 2),         # in full: 131072 tokens, d_in 11008 (H 1.9 GB); saliency checked on 2 chunks
+    ("c2_7b_down", 4, None, None),      # in full: 131072 tokens, d_in 11008 (H 1.9 GB)
     ("c3_70b_mlp", 2, 8192, None),      # full d_in 28672 (H 6.6 GB resident), two 4096-token chunks
     ("c4_sweep", 16, 32768, None),      # sixteen groups, two 16384-token chunks
-    ("c4_sweep", 1, 32768, 1),          # one group (units of two column tiles)
+    ("c4_sweep", 1, 32768, None),       # one group (units of two column tiles)
 ])
-def test_full_shapes_sampled(dev, name, g, n_tokens, s_chunks):
+def test_full_shapes_sampled(dev, name, g, n_tokens, _unused):
     """The large configurations at full layer size, launched exactly as bench.py launches them.
 
     The oracle cannot form g x d_in^2 x n products in seconds, so it is run exactly on a sampled
     sub-problem: for ~48 sampled input features F it computes H_k[F][:, F] from the columns X[:, F] alone,
-    which are the same entries of the full H_k; s is checked against the oracle on whole chunks; the objective
+    which are the same entries of the full H_k; s is checked against the oracle on every chunk; the objective
     is checked with the weight error restricted to the sampled features (W_hat = W elsewhere), which needs
     only those entries of H."""
     base = synth.CONFIGS[name]
@@ -310,14 +322,10 @@ def test_full_shapes_sampled(dev, name, g, n_tokens, s_chunks):
     F = np.unique(np.concatenate([rng.choice(cfg.d_in, 40, replace=False), syn.outlier_features[:8].cpu().numpy()]))
     Ft = torch.from_numpy(F).to(dev)
     xb = np.concatenate([synth.bf16_bits(x[:, Ft].contiguous()) for x in xs])          # [n, |F|]
-    # saliency: the oracle on whole chunks of the gradient
-    n_s = len(gs) if s_chunks is None else s_chunks
-    s_ref_part = np.concatenate([orc.saliency(synth.bf16_bits(gc), g) for gc in gs[:n_s]], axis=1)
-    check_s(torch.cat(ss[:n_s], dim=1), s_ref_part)
-    # H on the sampled features, from the GPU's saliency where the oracle's was not computed (it was checked
-    # above on the chunks where both exist, to 1e-4)
-    s_all = torch.cat(ss, dim=1).cpu().numpy().astype(np.float64)
-    s_all[:, :s_ref_part.shape[1]] = s_ref_part
+    # saliency: the oracle on every chunk of the gradient; the oracle's Hessian is built from the oracle's own
+    # saliency throughout
+    s_all = np.concatenate([orc.saliency(synth.bf16_bits(gc), g) for gc in gs], axis=1)
+    check_s(torch.cat(ss, dim=1), s_all)
     H_ref = orc.hessian(xb, s_all)                                                     # [g, |F|, |F|]
     H_sub = H[:, Ft][:, :, Ft]
     check_H(H_sub, H_ref)
@@ -367,8 +375,9 @@ def test_hessian_padded_rows_and_saliency_stride(dev):
 
 
 # ------------------------------------------------------------------------------------------ host path
-def test_host_pipeline_matches_device_calls(dev):
-    cfg = synth.LayerConfig("host", 700, 256, 384, 256, (2,), "lognormal", 0.01, 20.0)
+@pytest.mark.parametrize("d_out,g", [(256, 2), (1024, 128)])       # 129 fp64 results need more than 1 KiB
+def test_host_pipeline_matches_device_calls(dev, d_out, g):
+    cfg = synth.LayerConfig("host", 700, 256, 384, d_out, (g,), "lognormal", 0.01, 20.0)
     xs, gs, ss, H, W, What, loss = run_layer(cfg, dev)
     X_host = torch.cat(xs).cpu().pin_memory()
     grad_host = torch.cat(gs).cpu().pin_memory()

@@ -37,7 +37,7 @@ def read_fixture(path):
 # --------------------------------------------------------------------------- P0
 @pytest.mark.parametrize("impl", IMPLS)
 def test_hand_example(impl):
-    """Algorithm 1 lines 1/2/4 and Eq. 7 on the worked example in golden/hand_example.txt."""
+    """Algorithm 1 (groups, saliency, guided Hessian) and Eq. 7 on the worked example in golden/hand_example.txt."""
     fx = read_fixture(os.path.join(GOLDEN, "hand_example.txt"))
     xb = orc.f64_to_bf16_bits(fx["X"])
     gb = orc.f64_to_bf16_bits(fx["grad"])
@@ -217,6 +217,42 @@ def test_scalings_permutations_and_chunking(impl):
     np.testing.assert_allclose(orc.saliency(gb[:, perm], g, impl=impl), s, rtol=1e-14)
     swapped = np.concatenate([np.arange(m, 2 * m), np.arange(m)])
     np.testing.assert_allclose(orc.saliency(gb[:, swapped], g, impl=impl), s[::-1], rtol=1e-14)
+
+
+# --------------------------------------------------------------------------- P8 / P9
+@pytest.mark.parametrize("impl", IMPLS)
+def test_diagonal_and_probe_forms_equal_the_full_hessian(impl):
+    """hessian_diag and hessian_apply (the O(n d_in) checks used where the d_in x d_in oracle cannot go) against
+    the full oracle matrix on small inputs, streamed in ragged chunks; and against what a planted mistake would
+    give (unsquared x, s of the wrong group, a transposed probe product)."""
+    rng = np.random.default_rng(21)
+    n, d_in, g, nv = 131, 40, 3, 4
+    xb, x = bf16_exact(rng, (n, d_in))
+    s = rng.random((g, n)) * np.exp(rng.standard_normal(n))
+    V = rng.standard_normal((nv, d_in))
+    H = orc.hessian(xb, s, impl="c")
+    diag, out = None, None
+    for lo, hi in [(0, 50), (50, 51), (51, 51), (51, n)]:
+        diag = orc.hessian_diag(xb[lo:hi], s[:, lo:hi], diag, impl=impl)
+        out = orc.hessian_apply(xb[lo:hi], s[:, lo:hi], V, out, impl=impl)
+    for k in range(g):
+        np.testing.assert_allclose(diag[k], np.diag(H[k]), rtol=1e-12)
+        np.testing.assert_allclose(out[k], (H[k] @ V.T).T, rtol=1e-11, atol=1e-11 * np.abs(out[k]).max())
+    # planted mistakes are far outside those tolerances
+    assert not np.allclose(diag[0], np.diag(H[1]), rtol=1e-3)
+    assert not np.allclose(diag[0], (s[0][:, None] * np.abs(x)).sum(0), rtol=1e-3)
+    assert not np.allclose(out[0, 0], H[0].T @ V[1], rtol=1e-3)
+    # closed forms: one-hot rows give diag = per-feature sums of s and H v = diag * v
+    hot = rng.integers(0, d_in, n)
+    xh = np.zeros((n, d_in))
+    xh[np.arange(n), hot] = 1.0
+    xhb = orc.f64_to_bf16_bits(xh)
+    d1 = orc.hessian_diag(xhb, s, impl=impl)
+    o1 = orc.hessian_apply(xhb, s, V, impl=impl)
+    for k in range(g):
+        expect = np.bincount(hot, weights=s[k], minlength=d_in)
+        np.testing.assert_allclose(d1[k], expect, rtol=1e-13)
+        np.testing.assert_allclose(o1[k], expect[None, :] * V, rtol=1e-12, atol=1e-13)
 
 
 # --------------------------------------------------------------------------- P10

@@ -2,15 +2,17 @@
 
 Some callers of libgq cannot call cudaMalloc (a region being captured into a CUDA graph, an allocator-free
 callback, a process whose memory was all given to another pool), so this entry point keeps its scratch in a
-fixed 4 MiB + 128 KiB array inside the library.  The test drives it through the C-ABI and compares it with
-gq_objective (caller workspace) on two consecutive calls with different inputs: the second call runs over
-whatever the first one left in the shared scratch and must not be affected by it.  This file is named so
-that pytest collects it after every other test file.
+fixed 4 MiB + 256 KiB array inside the library.  The test drives it through the C-ABI and compares it with
+gq_objective (caller workspace) AND with the CPU fp64 oracle's objective on two consecutive calls with different
+inputs: the second call runs over whatever the first one left in the shared scratch and must not be affected by
+it.  (The oracle comparison matters: the kernel behind this entry point is not the one behind gq_objective.)
+This file is named so that pytest collects it after every other test file.
 """
 import numpy as np
 import pytest
 import torch
 
+from oracle import gq_oracle as orc
 from paper_2505_07004_b200 import api as libgq
 from paper_2505_07004_b200 import synth
 
@@ -47,6 +49,8 @@ def test_noalloc_objective_matches_workspace_objective_twice():
         ref_h, got_h = ref.cpu().numpy(), loss.cpu().numpy()
         assert np.all(np.isfinite(got_h)) and np.all(ref_h > 0)
         assert np.all(np.abs(got_h - ref_h) <= L_RTOL * np.abs(ref_h)), (got_h, ref_h)
+        oracle = orc.objective(W.cpu().numpy(), What.cpu().numpy(), H.cpu().numpy().astype(np.float64))
+        assert np.all(np.abs(got_h - oracle) <= L_RTOL * np.abs(oracle)), (got_h, oracle)
     # the same inputs again straight after: identical values (nothing stale is read)
     loss2 = torch.empty_like(loss)
     libgq.gq_objective_noalloc(W, What, H, loss2)
