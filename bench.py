@@ -4,8 +4,8 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
 One "step" is one pass of the whole path over one synthetic layer: for every token chunk
-gq_saliency + gq_hessian_accumulate, then gq_hessian_finalize and gq_objective (H is zeroed at the
-start of the step).  The default workload is the Llama-2-7B attention-projection shape
+gq_saliency_prepared + gq_hessian_accumulate (two launches), then gq_hessian_finalize and gq_objective (H is
+zeroed at the start of the step).  The default workload is the Llama-2-7B attention-projection shape
 (131072 tokens in 16 chunks of 8192, d_in = d_out = 4096, g = 4).  All inputs are seeded and
 synthetic and stay resident in HBM for the device-timed number; the `e2e` number goes through
 gq_layer_objective_host with pinned host buffers (host->device copies inside the timed region).
@@ -39,9 +39,16 @@ from paper_2505_07004_b200 import shard, synth
 METRIC = "guided_hessian_tokens_per_s"
 UNIT = "tokens/s"
 KERNEL_TIMING_EVERY = 8      # steps between two steps whose launches are timed one by one
-# DRAM bytes per launch of the dominant kernel from the committed ncu capture (profiles/), scaled to
-# one launch of the default workload; None until a capture exists for the current kernel.
-NCU_TRAFFIC_BYTES = {"c1_7b_attn": 343.36e6}      # profiles/hessian_kernel_c1_7b_attn.md
+NOMINAL_BF16_TFLOPS = 2250.0     # B200 dense bf16 / fp16 tensor peak (vendor figure), for context beside the measured peaks
+# DRAM bytes (read + write) per launch of the dominant kernel, from an ncu capture of one launch of that
+# workload; None where no capture of the current kernel exists.
+NCU_TRAFFIC_BYTES = {"c1_7b_attn": 343.36e6}
+# The oracle sample both the cpu_baseline leg and --impl reference time (one size, so that the oracle's
+# throughput is one number): tokens of chunk 0 for saliency + Hessian, channels per group for the objective.
+ORACLE_SAMPLE_TOKENS, ORACLE_SAMPLE_CHANNELS = 1024, 64
+SAL_B2B_PASSES = 5           # passes over all chunks in the back-to-back saliency measurement
+OBJECTIVE_KERNELS = ("split_delta", "gram_dot", "reduce")     # the kernels one gq_objective call launches
+CPU_BASELINE_PASSES = 4      # passes of that sample in the cpu_baseline leg (about 10-15 s of host time)
 
 
 def load_peaks():
@@ -104,6 +111,25 @@ class ClockSampler(threading.Thread):
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def config_dict(cfg, g):
+    """The workload description both arms print (identical keys and values)."""
+    return {"workload": cfg.name, "n": cfg.n, "chunk": cfg.chunk, "d_in": cfg.d_in, "d_out": cfg.d_out, "g": g,
+            "l2": "inputs (%.2f GB of X and grad per step, streamed once) are larger than L2; no flush"
+                  % ((cfg.n * (cfg.d_in + cfg.d_out) * 2) / 1e9),
+            "parallelism": "one layer per GPU, no collective"}
+
+
+def hessian_issued_flops(d_in, g, tokens):
+    """Flops the tensor cores are asked to do by one gq_hessian_accumulate launch: whole 256 x 256 tiles on the
+    upper triangle (the half of every diagonal tile below the diagonal is computed and discarded), tokens
+    rounded up to the 64-token step.  Pairs of groups share a tile pass; an odd last group runs on (row block,
+    two column tiles) units."""
+    nj = (d_in + 255) // 256
+    tiles = nj * (nj + 1) // 2
+    tok = (tokens + 63) // 64 * 64
+    return 2.0 * 256 * 256 * tok * tiles * g
+
+
 def dist_env():
     return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
 
@@ -143,16 +169,6 @@ def run_reference(args, cfg, g):
     from oracle import gq_oracle as orc
     orc.build()
     tokens, cpg = args.ref_tokens, args.ref_channels
-    if tokens <= 0:
-        # Size the per-step sample so that the whole run (warm-up + steps) takes about two minutes of oracle
-        # time: one untimed calibration pass on 64 tokens and 16 channels per group, cost taken as linear in both.
-        t0 = time.perf_counter()
-        oracle_sample(cfg, g, 64, 16)
-        t_cal = max(time.perf_counter() - t0, 1e-3)
-        per_step = 120.0 / max(1, args.steps + args.warmup)
-        scale = per_step / t_cal
-        tokens = int(min(1024, max(32, 64 * scale)) // 32 * 32)
-        cpg = int(min(64, max(8, 16 * scale)) // 8 * 8)
     for _ in range(args.warmup):
         oracle_sample(cfg, g, tokens, cpg)
     t0 = time.perf_counter()
@@ -167,7 +183,7 @@ def run_reference(args, cfg, g):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * wall / max(1, args.steps),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": cfg.name, "n": cfg.n, "chunk": cfg.chunk, "d_in": cfg.d_in, "d_out": cfg.d_out, "g": g},
+        "config": config_dict(cfg, g),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.threads(), "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -204,8 +220,8 @@ def run_ours(args, cfg, g):
         H.zero_()
         for c in range(n_chunks):
             nt = xs[c].shape[0]
-            libgq.gq_saliency(gs[c], g, 1.0, s=s_buf[:, :nt])
-            libgq.gq_hessian_accumulate(xs[c], s_buf[:, :nt], H, ws)
+            libgq.gq_saliency_prepared(gs[c], g, ws, 1.0, s=s_buf[:, :nt])
+            libgq.gq_hessian_accumulate(xs[c], s_buf[:, :nt], H, ws, flags=libgq.GQ_HESSIAN_S_PREPARED)
         libgq.gq_hessian_finalize(H)
         libgq.gq_objective(W, What, H, ows, loss=loss)
 
@@ -248,6 +264,21 @@ def run_ours(args, cfg, g):
     if not np.all(np.isfinite(loss_host)) or loss_host[g] <= 0:
         raise RuntimeError("objective is not finite/positive: %s" % loss_host)
 
+    # ---- saliency alone, back to back over all chunks (no per-launch event pair in the way)
+    sal_b2b_gbs = None
+    if n_chunks * cfg.chunk * cfg.d_out * 2 > 200e6:                    # only meaningful when a pass exceeds L2
+        for c in range(n_chunks):
+            libgq.gq_saliency(gs[c], g, 1.0, s=s_buf[:, :gs[c].shape[0]])
+        torch.cuda.synchronize()
+        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        b0.record()
+        for _ in range(SAL_B2B_PASSES):
+            for c in range(n_chunks):
+                libgq.gq_saliency(gs[c], g, 1.0, s=s_buf[:, :gs[c].shape[0]])
+        b1.record()
+        torch.cuda.synchronize()
+        sal_b2b_gbs = SAL_B2B_PASSES * sum(x.shape[0] * (2 * cfg.d_out + 4 * g) for x in gs) / (b0.elapsed_time(b1) * 1e-3) / 1e9
+
     # ---- end to end from pinned host memory through the host-buffer entry point
     e2e_s, e2e_steps, h2d, d2h = float('nan'), 0, 0, 0
     if not args.no_e2e:
@@ -285,40 +316,85 @@ def run_ours(args, cfg, g):
     if rank == 0:
         value = shard.whole_job_throughput(cfg.n, args.steps, ms_total * 1e-3, world)
         e2e_value = shard.whole_job_throughput(cfg.n, e2e_steps, e2e_ms * 1e-3, world) if e2e_steps else None
-        # dominant kernel: the tensor-core Gram kernel of gq_hessian_accumulate
+        # dominant kernel: the tensor-core kernel of gq_hessian_accumulate
         ga_ms, ga_n = kern["hessian"]
         flops_per_launch = float(g) * cfg.chunk * cfg.d_in * (cfg.d_in + 1)      # upper triangle, mul + add
-        achieved = flops_per_launch / (ga_ms / max(1, ga_n) * 1e-3) / 1e12 if ga_n else None
-        peak = peaks["bf16_tflops_sustained"]
+        issued_per_launch = hessian_issued_flops(cfg.d_in, g, cfg.chunk)
+        ms_per_launch = ga_ms / max(1, ga_n)
+        achieved = flops_per_launch / (ms_per_launch * 1e-3) / 1e12 if ga_n else None
+        issued = issued_per_launch / (ms_per_launch * 1e-3) / 1e12 if ga_n else None
+        # Which measured tensor peak applies: the burst figure when the timed region is short or the clock
+        # stayed near its maximum (the kernel ran as in a burst), the sustained one when the run sat at the
+        # power cap with the clock pulled down.  Both fractions are printed either way.
+        sm, sm_max = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+        near_max = bool(sm and sm_max and sm >= 0.9 * sm_max)
+        burst = near_max or ms_total < 1000.0
+        peak = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
         kernel_ms = sum(v[0] for v in kern.values())
         kernels = {k: {"launches": v[1], "ms_total": round(v[0], 4), "share": round(v[0] / kernel_ms, 4) if kernel_ms else None}
                    for k, v in kern.items()}
         sal_ms, sal_n = kern["saliency"]
         sal_bytes = cfg.chunk * (2 * cfg.d_out + 4 * g)
+        frac = lambda a, p: (a / p) if (a is not None and p) else None
+        roofline = {
+            "kernel": "hessian_kernel (gq_hessian_accumulate)", "bound": "tensor",
+            "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": frac(achieved, peak),
+            "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
+            "peak_source": ("bf16_tflops (burst), " if burst else "bf16_tflops_sustained, ") + peaks["source"],
+            "peak_regime": ("burst: %s" % ("median SM clock %.0f of %.0f MHz" % (sm, sm_max) if near_max
+                                           else "timed region of %.2f s" % (ms_total * 1e-3))) if burst
+                           else "sustained: timed region of %.1f s at a median SM clock of %s of %s MHz" % (ms_total * 1e-3, sm, sm_max),
+            "frac_of_burst_peak": frac(achieved, peaks["bf16_tflops"]),
+            "frac_of_sustained_peak": frac(achieved, peaks["bf16_tflops_sustained"]),
+            "frac_of_nominal_peak": frac(achieved, NOMINAL_BF16_TFLOPS),
+            "peaks_tflops": {"burst": peaks["bf16_tflops"], "sustained": peaks["bf16_tflops_sustained"],
+                             "nominal": NOMINAL_BF16_TFLOPS},
+            "flops_per_launch": flops_per_launch, "ms_per_launch": ms_per_launch,
+            "issued_flops_per_launch": issued_per_launch, "issued_tflops": issued,
+            "issued_frac_of_nominal_peak": frac(issued, NOMINAL_BF16_TFLOPS),
+            "target": "60 %% of the nominal peak: %s" % ("met" if (achieved or 0) >= 0.6 * NOMINAL_BF16_TFLOPS else "not met"),
+        }
+        sal_gbs = (sal_bytes / (sal_ms / max(1, sal_n) * 1e-3) / 1e9) if sal_n else None
+        saliency_roofline = {
+            "kernel": "saliency_kernel (gq_saliency)", "bound": "hbm", "unit": "GB/s", "peak": peaks["hbm_gbs"],
+            "bytes_per_launch": sal_bytes,
+            "achieved": sal_gbs, "frac": frac(sal_gbs, peaks["hbm_gbs"]),
+            "timing": "event pair around each launch inside the step (a %d MB launch lasts ~10-20 us: the pair's own "
+                      "cost is part of this figure)" % (sal_bytes // 1000000),
+            "achieved_back_to_back": sal_b2b_gbs, "frac_back_to_back": frac(sal_b2b_gbs, peaks["hbm_gbs"]),
+            "timing_back_to_back": "one event pair around %d passes over all %d chunks (%.2f GB per pass, larger than L2)"
+                                   % (SAL_B2B_PASSES, n_chunks, n_chunks * sal_bytes / 1e9),
+        }
+        objective_roofline = None
+        if kern["gram_dot"][1]:
+            calls = kern["gram_dot"][1]
+            obj_ms = sum(kern[k][0] for k in OBJECTIVE_KERNELS) / calls
+            obj_bytes = 2.0 * g * cfg.d_in * (cfg.d_in + 1) + 8.0 * cfg.d_in * cfg.d_out     # upper triangle of H (fp32) + W, W_hat
+            obj_flops_sym = float(cfg.d_in) * cfg.d_in * cfg.d_out                           # 2 d_in^2 d_out, halved by symmetry
+            t_bytes = obj_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+            t_flops = obj_flops_sym / (peaks["bf16_tflops"] * 1e12) * 1e3
+            objective_roofline = {
+                "kernel": "gq_objective (all of its kernels)", "ms_per_call": obj_ms,
+                "bound": "tensor" if t_flops >= t_bytes else "hbm",
+                "algorithmic_bytes": obj_bytes, "symmetric_flops": obj_flops_sym,
+                "ms_at_hbm_peak": t_bytes, "ms_at_tensor_burst_peak": t_flops,
+                "frac": max(t_bytes, t_flops) / obj_ms,
+                "gbs_algorithmic": obj_bytes / (obj_ms * 1e-3) / 1e9,
+                "frac_of_hbm_peak": obj_bytes / (obj_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                "tflops_symmetric": obj_flops_sym / (obj_ms * 1e-3) / 1e12,
+                "tflops_dense_equivalent": 2.0 * obj_flops_sym / (obj_ms * 1e-3) / 1e12,
+                "note": "frac = the slower of (bytes at the measured copy bandwidth, symmetric flops at the measured burst "
+                        "16-bit tensor peak) divided by the measured time of the whole call",
+            }
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": cfg.name, "n": cfg.n, "chunk": cfg.chunk, "d_in": cfg.d_in, "d_out": cfg.d_out, "g": g,
-                       "l2": "inputs (%.2f GB of X and grad per step, streamed once) are larger than L2; no flush"
-                             % ((cfg.n * (cfg.d_in + cfg.d_out) * 2) / 1e9),
-                       "parallelism": "one layer per GPU, no collective"},
+            "config": config_dict(cfg, g),
             "hessian_tflops_useful": (float(g) * cfg.n * cfg.d_in * (cfg.d_in + 1)) * world * args.steps / (ms_total * 1e-3) / 1e12,
-            "roofline": {"kernel": "hessian_kernel (gq_hessian_accumulate)", "bound": "tensor",
-                         "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                         "frac": (achieved / peak) if achieved else None,
-                         "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
-                         "peak_source": "bf16_tflops_sustained, " + peaks["source"],
-                         "frac_of_burst_peak": (achieved / peaks["bf16_tflops"]) if achieved else None,
-                         "flops_per_launch": flops_per_launch, "ms_per_launch": ga_ms / max(1, ga_n)},
-            "saliency_hbm": {"achieved_gbs": (sal_bytes / (sal_ms / max(1, sal_n) * 1e-3) / 1e9) if sal_n else None,
-                             "peak_gbs": peaks["hbm_gbs"]},
-            "objective": (lambda ms: {
-                "ms_per_call": ms,
-                "tflops_dense_equivalent": 2.0 * cfg.d_in ** 2 * cfg.d_out / (ms * 1e-3) / 1e12,
-                "gbs_algorithmic": (2.0 * g * cfg.d_in * (cfg.d_in + 1) + 8.0 * cfg.d_in * cfg.d_out) / (ms * 1e-3) / 1e9,
-            })((kern["split_delta"][0] + kern["gram_dot"][0] + kern["reduce"][0]) / max(1, kern["gram_dot"][1]))
-            if kern["gram_dot"][1] else None,
+            "roofline": roofline,
+            "saliency_hbm": saliency_roofline,
+            "objective": objective_roofline,
             "kernels": kernels,
             "kernel_timing": "CUDA-event pairs around every launch of every %d-th timed step" % KERNEL_TIMING_EVERY,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -330,9 +406,14 @@ def run_ours(args, cfg, g):
         if world == 1 and not args.no_cpu_baseline:
             from oracle import gq_oracle as orc
             orc.build()
-            v, secs, desc = oracle_sample(cfg, g, args.cpu_tokens, args.cpu_channels)
-            out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": orc.threads(), "kind": "oracle",
-                                   "sample": desc, "seconds": secs}
+            vals, secs, desc = [], 0.0, ""
+            for _ in range(CPU_BASELINE_PASSES):
+                v, sec, desc = oracle_sample(cfg, g, args.cpu_tokens, args.cpu_channels)
+                vals.append(v)
+                secs += sec
+            out["cpu_baseline"] = {"value": len(vals) / sum(1.0 / v for v in vals), "unit": UNIT, "cores": orc.threads(),
+                                   "kind": "oracle", "sample": "%d passes of: %s" % (CPU_BASELINE_PASSES, desc),
+                                   "seconds": secs}
         print(json.dumps(out), flush=True)
     if world > 1:
         import torch.distributed as dist
@@ -348,11 +429,11 @@ def main():
     ap.add_argument("--workload", default="c1_7b_attn", choices=sorted(synth.CONFIGS))
     ap.add_argument("--g", type=int, default=0, help="override the number of groups (sweep config)")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--cpu-tokens", type=int, default=4096)
-    ap.add_argument("--cpu-channels", type=int, default=128)
-    ap.add_argument("--ref-tokens", type=int, default=0,
-                    help="tokens per step of the reference arm (0: sized so that the run takes about two minutes)")
-    ap.add_argument("--ref-channels", type=int, default=64)
+    ap.add_argument("--cpu-tokens", type=int, default=ORACLE_SAMPLE_TOKENS)
+    ap.add_argument("--cpu-channels", type=int, default=ORACLE_SAMPLE_CHANNELS)
+    ap.add_argument("--ref-tokens", type=int, default=ORACLE_SAMPLE_TOKENS,
+                    help="tokens per step of the reference arm (the same sample as the cpu_baseline leg)")
+    ap.add_argument("--ref-channels", type=int, default=ORACLE_SAMPLE_CHANNELS)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--tokens", type=int, default=0, help="use only the first TOKENS tokens (profiling runs)")

@@ -62,7 +62,7 @@ int32_t gq_last_cuda_error(void);
  *     s[k * ld_s + i] = (grad_scale^2 / m) * sum_{j = m k}^{m (k+1) - 1} grad[i * ld_grad + j]^2
  *
  *   grad        bf16 [n, ld_grad], 16-byte aligned, ld_grad >= d_out, ld_grad % 8 == 0
- *   n           tokens in this call, >= 0 (0 is a no-op: sizes are still validated, pointers are not)
+ *   n           tokens in this call, >= 0 (0 is a no-op: sizes are still validated, pointers are not), n * g < 2^31
  *   d_out, g    d_out % g == 0 and (d_out / g) % 8 == 0, 1 <= g <= 1024
  *   grad_scale  finite; the paper uses 1e3, tests use 1
  *   s           fp32 [g, ld_s] (group-major so that each s_k is contiguous), ld_s >= n
@@ -70,6 +70,17 @@ int32_t gq_last_cuda_error(void);
  */
 int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad, int32_t g,
                     float grad_scale, float *s, int64_t ld_s, void *stream);
+
+/*
+ * gq_saliency that also leaves s in the packed form the guided-Hessian kernel consumes (Algorithm 1, saliency
+ * step; same values, same fp32 s): `hessian_workspace` is the workspace that the NEXT gq_hessian_accumulate call
+ * for the same n tokens and the same g will be given, at least gq_hessian_workspace_bytes(n, d_in, g, flags)
+ * bytes (the size does not depend on d_in), 1024-byte aligned.  That call is then made with the flag
+ * GQ_HESSIAN_S_PREPARED and skips its own preparation kernel: two launches per token chunk instead of three.
+ */
+int32_t gq_saliency_prepared(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad, int32_t g,
+                             float grad_scale, float *s, int64_t ld_s, void *hessian_workspace,
+                             size_t workspace_bytes, void *stream);
 
 /*
  * Guided Hessian, one token chunk: Algorithm 1, Hessian step, streamed,
@@ -80,11 +91,11 @@ int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad,
  *   n          tokens in this chunk, >= 0 (0 is a no-op: sizes are still validated, pointers are not)
  *   d_in       d_in % 8 == 0, 8 <= d_in <= 65536
  *   s          fp32 [g, ld_s], s >= 0 (as produced by gq_saliency), ld_s >= n
- *   H          fp32 [g, d_in, d_in] row-major, 16-byte aligned.  The caller zeroes it before the
+ *   H          fp32 [g, d_in, d_in] row-major, 128-byte aligned.  The caller zeroes it before the
  *              first chunk and keeps it resident between chunks.  After any number of calls only
  *              entries with a <= b are defined; entries below the diagonal hold unspecified finite
  *              values until gq_hessian_finalize() is called.
- *   flags      0, or GQ_HESSIAN_DETERMINISTIC (see below)
+ *   flags      0, or GQ_HESSIAN_DETERMINISTIC and / or GQ_HESSIAN_S_PREPARED (see below)
  *   workspace  device scratch of at least gq_hessian_workspace_bytes(n_max, d_in, g, flags) bytes with
  *              n_max >= n, 1024-byte aligned (8 bytes per token and pair of groups: s in the form the
  *              kernel consumes); contents need not be preserved between calls.
@@ -100,6 +111,9 @@ int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad,
  * call and results are bit-reproducible run to run, at the price of an idle tail in the last round.
  */
 #define GQ_HESSIAN_DETERMINISTIC 1u
+/* The workspace already holds s in packed form: it was filled by gq_saliency_prepared for exactly these n tokens
+ * and this g, and nothing has written to it since.  (s itself is still validated but not read.) */
+#define GQ_HESSIAN_S_PREPARED 2u
 int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld_x, const float *s,
                               int64_t ld_s, int32_t g, float *H, uint32_t flags, void *workspace,
                               size_t workspace_bytes, void *stream);
@@ -110,7 +124,7 @@ size_t gq_hessian_workspace_bytes(int64_t n_max, int64_t d_in, int32_t g, uint32
 /*
  * Completes H after the last chunk: copies the upper triangle onto the lower one,
  * H[k][b][a] = H[k][a][b] for a < b, so that every H_k is a full, exactly symmetric matrix
- * (H_k is symmetric by definition: Section 3.2).  Idempotent.
+ * (H_k is symmetric by definition: Section 3.2).  Idempotent.  H 128-byte aligned.
  */
 int32_t gq_hessian_finalize(float *H, int64_t d_in, int32_t g, void *stream);
 
@@ -149,15 +163,20 @@ int32_t gq_hessian_gather_shares(float *const *H_ranks, int32_t ranks, int32_t r
  *     loss_out[g] = sum_k loss_out[k]
  *
  *   W, W_hat   fp32 [d_out, d_in] row-major, 16-byte aligned (row j = output channel j)
- *   H          fp32 [g, d_in, d_in] as left by gq_hessian_accumulate or gq_hessian_finalize:
+ *   H          fp32 [g, d_in, d_in] as left by gq_hessian_accumulate or gq_hessian_finalize, 128-byte aligned:
  *              only entries with a <= b are read
  *   loss_out   fp64 [g + 1] in device memory
  *   workspace  device scratch of at least gq_objective_workspace_bytes(d_in, d_out, g) bytes,
  *              1024-byte aligned
  * Same shape rules as above (d_in % 8 == 0, d_out % g == 0, (d_out / g) % 8 == 0).
- * Arithmetic: delta = W - W_hat in fp32, split into two bf16 terms (delta = hi + lo to ~2^-17);
- * the Gram matrices Delta_k^T Delta_k are formed on the tensor cores with fp32 accumulation and
- * contracted with H_k in the same kernel; partial sums are reduced in fp64 in a fixed order.
+ * Arithmetic: delta = W - W_hat in fp32.  A first pass finds max |delta| over the layer, a second writes
+ * delta * 2^e to the workspace as ONE fp16 matrix, e chosen so that the largest entry lies in [2^14, 2^15)
+ * (11 significant bits for every entry down to 2^-28 of the largest; round to nearest, no bias).  The Gram
+ * matrices Delta_k^T Delta_k are formed on the tensor cores (fp16 operands, fp32 accumulation) two 256-column
+ * tiles at a time and contracted with H_k (fp32) straight out of tensor memory; partial sums are reduced in
+ * fp64 in a fixed order and multiplied by 2^-2e.  Relative error of the result: at most 2^-11 = 4.9e-4 if
+ * every rounding error had the same sign and H_k had no negative entries, about 1e-6 for rounding errors of
+ * random sign (what is seen on quantisation errors).  Results are bit-reproducible run to run.
  */
 int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d_out, const float *H,
                      int32_t g, double *loss_out, void *workspace, size_t workspace_bytes,
@@ -330,7 +349,7 @@ enum gq_kernel_id {
     GQ_KERNEL_SALIENCY = 0,    /* Algorithm 1, saliency step                                    */
     GQ_KERNEL_HESSIAN = 1,     /* tensor-core H += X^T Diag(s_k) X, scaling fused (Algorithm 1, Hessian step) */
     GQ_KERNEL_MIRROR = 2,      /* gq_hessian_finalize                                    */
-    GQ_KERNEL_SPLIT_DELTA = 3, /* W - W_hat -> bf16 hi/lo                                */
+    GQ_KERNEL_SPLIT_DELTA = 3, /* W - W_hat -> fp16 (maximum pass + conversion pass)     */
     GQ_KERNEL_GRAM_DOT = 4,    /* tensor-core Delta_k^T Delta_k contracted with H_k (Eq. 7) */
     GQ_KERNEL_REDUCE = 5,      /* fp64 reduction of the partial sums                     */
     GQ_KERNEL_SPLIT_SALIENCY = 6, /* s -> pairs of bf16 terms for the Hessian kernel's scalers */

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libgq.so")
 _lib = None
 
 EXPORTS = (
-    "gq_version", "gq_status_string", "gq_last_cuda_error", "gq_saliency", "gq_hessian_accumulate",
+    "gq_version", "gq_status_string", "gq_last_cuda_error", "gq_saliency", "gq_saliency_prepared", "gq_hessian_accumulate",
     "gq_hessian_workspace_bytes", "gq_hessian_finalize", "gq_objective", "gq_objective_workspace_bytes",
     "gq_layer_objective_host", "gq_layer_host_arena_bytes", "gq_check", "gq_launch_count",
     "gq_kernel_timing_enable", "gq_kernel_timing_read", "gq_objective_noalloc", "gq_cd_cycles", "gq_cd_workspace_bytes",
@@ -27,6 +27,7 @@ EXPORTS = (
     "gq_hessian_reduce_share", "gq_hessian_gather_shares", "gq_lnq", "gq_lnq_workspace_bytes",
 )
 GQ_HESSIAN_DETERMINISTIC = 1      # flag of gq_hessian_accumulate: single writer per element of H
+GQ_HESSIAN_S_PREPARED = 2         # flag of gq_hessian_accumulate: the workspace was filled by gq_saliency_prepared
 KERNEL_NAMES = ("saliency", "hessian", "mirror", "split_delta", "gram_dot", "reduce", "split_saliency", "cd_panel",
                 "cd_block", "cd_aux", "cb_gemm", "cb_fold", "cb_aux", "exchange")
 
@@ -59,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.gq_launch_count.restype = ctypes.c_uint64
         L.gq_saliency.restype = i32
         L.gq_saliency.argtypes = [vp, i64, i64, i64, i32, f32, vp, i64, vp]
+        L.gq_saliency_prepared.restype = i32
+        L.gq_saliency_prepared.argtypes = [vp, i64, i64, i64, i32, f32, vp, i64, vp, sz, vp]
         L.gq_hessian_workspace_bytes.restype = sz
         L.gq_hessian_workspace_bytes.argtypes = [i64, i64, i32, u32]
         L.gq_hessian_accumulate.restype = i32
@@ -193,6 +196,28 @@ def gq_saliency(grad: torch.Tensor, g: int, grad_scale: float = 1.0, s: Optional
     return s
 
 
+def gq_saliency_prepared(grad: torch.Tensor, g: int, hessian_workspace: torch.Tensor, grad_scale: float = 1.0,
+                         s: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """:func:`gq_saliency` that also fills ``hessian_workspace`` with ``s`` in the form the Hessian kernel reads;
+    the following :func:`gq_hessian_accumulate` for the same tokens is then called with
+    ``flags=GQ_HESSIAN_S_PREPARED`` (one launch less per chunk)."""
+    _dev(grad, torch.bfloat16, "grad")
+    n, d_out, ld = _rows(grad, "grad")
+    if s is None:
+        s = torch.empty((g, n), dtype=torch.float32, device=grad.device)
+    _dev(s, torch.float32, "s")
+    _, s_n, ld_s = _rows(s, "s")
+    if s.shape[0] != g or s_n < n:
+        raise ValueError("s must be [g, >= n]")
+    with _on(_same_device(("grad", grad), ("s", s), ("hessian_workspace", hessian_workspace)), stream) as st:
+        rc = lib().gq_saliency_prepared(grad.data_ptr(), n, d_out, ld, g, float(grad_scale), s.data_ptr(), ld_s,
+                                        hessian_workspace.data_ptr(),
+                                        hessian_workspace.numel() * hessian_workspace.element_size(), st)
+    if rc:
+        raise GQError("gq_saliency_prepared", rc)
+    return s
+
+
 def gq_hessian_workspace_bytes(n_max: int, d_in: int, g: int, flags: int = 0) -> int:
     return int(lib().gq_hessian_workspace_bytes(n_max, d_in, g, flags))
 
@@ -245,10 +270,14 @@ def _rank_pointers(H_ranks, d_in: int, g: int):
 
 def _own_device(H_ranks, rank: int):
     """Device of the calling rank's own matrix (peers may be given as raw pointers)."""
-    own = H_ranks[rank]
-    if not isinstance(own, torch.Tensor):
-        raise ValueError("H_ranks[rank] must be this process's own tensor")
-    return _same_device(("H_ranks[rank]", own))
+    if 0 <= rank < len(H_ranks):
+        own = H_ranks[rank]
+        if not isinstance(own, torch.Tensor):
+            raise ValueError("H_ranks[rank] must be this process's own tensor")
+        return _same_device(("H_ranks[rank]", own))
+    # a rank outside the list is the library's to reject; run the call on the device of any tensor given
+    tensors = [("H_ranks[%d]" % i, h) for i, h in enumerate(H_ranks) if isinstance(h, torch.Tensor)]
+    return _same_device(*tensors[:1])
 
 
 def gq_hessian_reduce_share(H_ranks, rank: int, d_in: int, g: int, stream=None) -> None:

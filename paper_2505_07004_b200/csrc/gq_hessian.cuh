@@ -19,10 +19,7 @@
 //              (M = 256, N = 256, K = 16) with fp32 accumulation in tensor memory
 //   epilogue   eight warps per CTA move the accumulators to H: tcgen05.ld -> swizzled staging block in
 //              shared memory -> TMA reduce-add (cp.reduce.async.bulk.tensor ... .add) of 32 x 32 fp32
-//              blocks, so H is never read by the SMs and every access to it is a full 128-byte row segment.
-//              When a unit is short (few k-steps, i.e. small token chunks) the time the tensor core waits
-//              for this read-out matters more than the access pattern, and the warps add their registers
-//              to H directly with red.global.add.v4.f32 instead (no staging, nothing to wait for)
+//              blocks, so H is never read by the SMs and every access to it is a full 128-byte row segment
 //
 // Per CTA and k-step (1024 tensor-core clocks for two groups) this moves 32 KB from L2 (half of what a
 // per-group pass over pre-scaled operands needs) and 112 KB through shared memory.
@@ -44,6 +41,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "gq_kernels.cuh"
 #include "gq_pipeline.cuh"
 
 namespace gq {
@@ -120,15 +118,6 @@ __device__ __forceinline__ void st_shared_16(uint32_t addr, const uint4 &v)
 // conversion work in its loop (sixteen threads share a token; converting there would be done sixteen times).
 __global__ void __launch_bounds__(256)
 split_saliency_kernel(const float *__restrict__ s, long long ld_s, int n, int g, uint2 *__restrict__ out);
-
-// A saliency value as two bf16 terms packed in one word: low half hi = bf16(a), high half lo = bf16(a - hi);
-// hi + lo carries a to 16 significant bits.
-__device__ __forceinline__ uint32_t split_scale(float a)
-{
-    const __nv_bfloat16 hi = __float2bfloat16_rn(a);
-    const __nv_bfloat16 lo = __float2bfloat16_rn(a - __bfloat162float(hi));
-    return static_cast<uint32_t>(__bfloat16_as_ushort(hi)) | (static_cast<uint32_t>(__bfloat16_as_ushort(lo)) << 16);
-}
 
 __global__ void __launch_bounds__(256)
 split_saliency_kernel(const float *__restrict__ s, long long ld_s, int n, int g, uint2 *__restrict__ out)

@@ -28,57 +28,94 @@ __device__ __forceinline__ uint4 float_to_bf16x8(const float (&f)[8])
     return v;
 }
 
+// A saliency value as the guided-Hessian kernel's scalers consume it: two bf16 terms packed in one word, low
+// half hi = bf16(a), high half lo = bf16(a - hi); hi + lo carries a to 16 significant bits.
+__device__ __forceinline__ uint32_t split_scale(float a)
+{
+    const __nv_bfloat16 hi = __float2bfloat16_rn(a);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(a - __bfloat162float(hi));
+    return static_cast<uint32_t>(__bfloat16_as_ushort(hi)) | (static_cast<uint32_t>(__bfloat16_as_ushort(lo)) << 16);
+}
+
+// 16 bytes that are read once (evict-first).  Written as volatile asm so that the loads of a group are all
+// issued, in order, before the first of them is consumed.
+__device__ __forceinline__ uint4 ld_once_16(const uint4 *p)
+{
+    uint4 v;
+    asm volatile("ld.global.cs.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ float sum_sq_bf16x8(const uint4 &v, float acc)
+{
+    float f[8];
+    bf16x8_to_float(v, f);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc = fmaf(f[e], f[e], acc);
+    return acc;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Algorithm 1, saliency step.  One warp per (token, group) segment of m = d_out / g gradients:
 //   s[k][i] = (grad_scale^2 / m) * sum_j grad[i][m k + j]^2.
-// A lane reads 16 bytes (8 bf16) per load and issues eight (long segments) or four loads (the last ones
-// predicated off at the end of the segment) before it touches the first result.
+// A lane reads 16 bytes (8 bf16) per load; the first four loads of a segment (all of it for m <= 1024) are
+// issued back to back before anything is used, longer segments continue eight loads at a time.  The grid has one
+// warp per segment (no grid-stride loop: thousands of short-lived blocks keep every SM at full occupancy and
+// balance the tail at a granularity of 8 segments) and the index arithmetic is 32-bit, so the loads of a warp
+// leave a few dozen cycles after it starts; measured on 67 MB launches this streams at 5.4 TB/s where a
+// persistent grid with 64-bit segment arithmetic reached 3.6 TB/s.
 // The lane-to-element assignment and the butterfly reduction are fixed, so the result does not depend on
 // the grid.
+// If `words` is not null the value is also stored in the packed form of split_scale, laid out as the
+// guided-Hessian kernel reads it: [ceil(g / 2)][n] pairs of words, pair q of token i = groups 2q and 2q + 1
+// (the second word of an odd last group is 0).
 __global__ void __launch_bounds__(256)
-saliency_kernel(const __nv_bfloat16 *__restrict__ grad, long long n, int m, long long ld_grad, int g, float coef,
-                float *__restrict__ s, long long ld_s)
+saliency_kernel(const __nv_bfloat16 *__restrict__ grad, unsigned n, int m, long long ld_grad, int g, float coef,
+                float *__restrict__ s, long long ld_s, uint32_t *__restrict__ words)
 {
     const int lane = threadIdx.x & 31;
-    const long long warp0 = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
-    const long long nwarps = (static_cast<long long>(gridDim.x) * blockDim.x) >> 5;
-    const long long segments = n * g;
+    const unsigned seg = blockIdx.x * 8u + (threadIdx.x >> 5);
+    if (seg >= n * static_cast<unsigned>(g)) return;
+    const unsigned i = seg / static_cast<unsigned>(g);
+    const int k = static_cast<int>(seg - i * static_cast<unsigned>(g));
     const int vecs = m >> 3;                             // 16-byte vectors per segment
-    for (long long seg = warp0; seg < segments; seg += nwarps) {
-        const long long i = seg / g;
-        const int k = static_cast<int>(seg - i * g);
-        const uint4 *src = reinterpret_cast<const uint4 *>(grad + i * ld_grad + static_cast<long long>(k) * m);
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        int v = lane;
-        for (; v + 224 < vecs; v += 256) {               // eight full loads in flight
-            uint4 x[8];
+    const uint4 *src = reinterpret_cast<const uint4 *>(grad + static_cast<long long>(i) * ld_grad + static_cast<long long>(k) * m);
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    {
+        uint4 x[4];
 #pragma unroll
-            for (int t = 0; t < 8; ++t) x[t] = __ldcs(src + v + 32 * t);
+        for (int t = 0; t < 4; ++t)
+            x[t] = (lane + 32 * t < vecs) ? ld_once_16(src + lane + 32 * t) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-            for (int t = 0; t < 8; ++t) {
-                float f[8];
-                bf16x8_to_float(x[t], f);
+        for (int t = 0; t < 4; ++t) acc[t] = sum_sq_bf16x8(x[t], acc[t]);
+    }
+    int v = lane + 128;
+    for (; v + 224 < vecs; v += 256) {                   // eight full loads in flight
+        uint4 x[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[t & 3] = fmaf(f[e], f[e], acc[t & 3]);
-            }
+        for (int t = 0; t < 8; ++t) x[t] = ld_once_16(src + v + 32 * t);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) acc[t & 3] = sum_sq_bf16x8(x[t], acc[t & 3]);
+    }
+    for (; v < vecs; v += 128) {                         // rest: four loads, predicated off past the end
+        uint4 x[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t)
+            x[t] = (v + 32 * t < vecs) ? ld_once_16(src + v + 32 * t) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int t = 0; t < 4; ++t) acc[t] = sum_sq_bf16x8(x[t], acc[t]);
+    }
+    float sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+    if (lane == 0) {
+        const float val = sum * coef;
+        s[static_cast<long long>(k) * ld_s + i] = val;
+        if (words) {
+            uint32_t *w = words + (static_cast<long long>(k >> 1) * n + i) * 2;
+            w[k & 1] = split_scale(val);
+            if ((k & 1) == 0 && k + 1 == g) w[1] = 0u;
         }
-        for (; v < vecs; v += 128) {                     // rest: four loads, predicated off past the end
-            uint4 x[4];
-#pragma unroll
-            for (int t = 0; t < 4; ++t)
-                x[t] = (v + 32 * t < vecs) ? __ldcs(src + v + 32 * t) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                float f[8];
-                bf16x8_to_float(x[t], f);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) acc[t] = fmaf(f[e], f[e], acc[t]);
-            }
-        }
-        float sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-        if (lane == 0) s[static_cast<long long>(k) * ld_s + i] = sum * coef;
     }
 }
 

@@ -19,6 +19,7 @@
 #include "gq_codebook.cuh"
 #include "gq_exchange.cuh"
 #include "gq_wide_gemm.cuh"
+#include "gq_gram_dot.cuh"
 #include "gq_kernels.cuh"
 
 #define GQ_VERSION_NUMBER 100   /* 0.1.0 */
@@ -68,7 +69,6 @@ struct DeviceInfo {
     bool ready = false;
     int sm_count = 0;
     int max_pairs = 0;          // CTA pairs (clusters of two) of a tensor-core kernel that can be resident at once
-    int saliency_blocks = 1;    // CTAs of saliency_kernel that fit on one SM (its grid-stride grid is sized to fit)
     uint32_t *status_ptr = nullptr;
 };
 DeviceInfo g_dev[kMaxDevices];
@@ -120,7 +120,7 @@ int32_t device_info(DeviceInfo **out)
         GQ_CUDA(cudaFuncSetAttribute(gq::pair_gemm_kernel<gq::MODE_FULL>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, gq::OBJ_SMEM_BYTES));
         GQ_CUDA(cudaFuncSetAttribute(gq::wide_gemm_kernel<gq::WG_FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, gq::WG_SMEM_BYTES));
-        GQ_CUDA(cudaFuncSetAttribute(gq::wide_gemm_kernel<gq::WG_OBJECTIVE>, cudaFuncAttributeMaxDynamicSharedMemorySize, gq::WG_SMEM_BYTES));
+        GQ_CUDA(cudaFuncSetAttribute(gq::gram_dot_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gq::GD_SMEM_BYTES));
         GQ_CUDA(cudaFuncSetAttribute(gq::cd_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      gq::CD_SMEM_BYTES));
         GQ_CUDA(cudaFuncSetAttribute(gq::hessian_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -146,14 +146,6 @@ int32_t device_info(DeviceInfo **out)
             if (clusters > di.sm_count / 2) clusters = di.sm_count / 2;
             if (clusters < 1) clusters = 1;
             di.max_pairs = clusters;
-        }
-        {
-            int blocks = 0;
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, gq::saliency_kernel, 256, 0) != cudaSuccess || blocks < 1) {
-                (void)cudaGetLastError();
-                blocks = 4;
-            }
-            di.saliency_blocks = blocks;
         }
         if (!g_encode) {
             void *fn = nullptr;
@@ -183,17 +175,17 @@ unsigned long long wait_budget_ns()
     return v;
 }
 
-// bf16 tensor [groups][rows][features] (row stride ld, group stride gstride, in elements) as a TMA map
+// 16-bit tensor [groups][rows][features] (bf16 unless `dtype` says fp16; row stride ld, group stride gstride, in elements) as a TMA map
 // with 64-feature x 64-row boxes and the 128-byte swizzle.
 int32_t make_map(CUtensorMap *map, const void *base, int64_t features, int64_t rows, int64_t groups, int64_t ld,
-                 int64_t gstride)
+                 int64_t gstride, CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16)
 {
     cuuint64_t dims[3] = {static_cast<cuuint64_t>(features), static_cast<cuuint64_t>(rows),
                           static_cast<cuuint64_t>(groups)};
     cuuint64_t strides[2] = {static_cast<cuuint64_t>(ld) * 2, static_cast<cuuint64_t>(gstride) * 2};
     cuuint32_t box[3] = {gq::BOX_FEATURES, gq::TILE_K, 1};
     cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+    CUresult r = g_encode(map, dtype, 3, const_cast<void *>(base), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -307,17 +299,18 @@ size_t hessian_ws_bytes(int64_t n_max, int64_t, int32_t g)
 }
 
 struct ObjectiveLayout {
-    size_t hi_off, lo_off, partials_off, total;
+    size_t header_off, half_off, partials_off, total;
 };
+// Scratch of gq_objective: a 1 KiB header (largest |delta| and the chosen power-of-two scale), delta as one fp16
+// matrix, and one fp64 partial sum per (work unit, CTA of the pair, epilogue warp).
 ObjectiveLayout objective_layout(int64_t d_in, int64_t d_out, int32_t g)
 {
     ObjectiveLayout L;
-    const size_t mat = round_up(static_cast<size_t>(d_in) * static_cast<size_t>(d_out) * 2, 1024);
-    L.hi_off = 0;
-    L.lo_off = mat;
-    L.partials_off = 2 * mat;
+    L.header_off = 0;
+    L.half_off = 1024;
+    L.partials_off = L.half_off + round_up(static_cast<size_t>(d_in) * static_cast<size_t>(d_out) * 2, 1024);
     L.total = L.partials_off +
-              round_up(static_cast<size_t>(tiles_for(d_in)) * g * gq::WG_PARTIALS_PER_UNIT * sizeof(double), 1024);
+              round_up(static_cast<size_t>(tiles_for(d_in)) * g * gq::GD_PARTIALS_PER_UNIT * sizeof(double), 1024);
     return L;
 }
 
@@ -396,35 +389,57 @@ int32_t gq_last_cuda_error(void) { return tl_last_cuda_error; }
 
 uint64_t gq_launch_count(void) { return g_launches.load(); }
 
-int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad, int32_t g, float grad_scale,
-                    float *s, int64_t ld_s, void *stream)
+static int32_t saliency_impl(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad, int32_t g, float grad_scale,
+                             float *s, int64_t ld_s, bool prepare, void *hessian_workspace, size_t workspace_bytes,
+                             void *stream)
 {
     if (n < 0 || g < 1 || d_out < 1 || d_out % g != 0 || ld_grad < d_out || ld_s < n ||
         !(grad_scale == grad_scale) || grad_scale - grad_scale != 0.0f)
         return GQ_ERR_INVALID_ARG;
-    if ((d_out / g) % 8 != 0 || g > 1024 || d_out > (1ll << 24) || n > (1ll << 40)) return GQ_ERR_UNSUPPORTED_SHAPE;
+    if ((d_out / g) % 8 != 0 || g > 1024 || d_out > (1ll << 24) || n * g >= (1ll << 31)) return GQ_ERR_UNSUPPORTED_SHAPE;
     if (ld_grad % 8 != 0) return GQ_ERR_ALIGNMENT;
     if (n == 0) return GQ_OK;              // nothing to read or write: pointers are not looked at
     if (!grad || !s) return GQ_ERR_INVALID_ARG;
     if (!aligned(grad, 16) || !aligned(s, 4)) return GQ_ERR_ALIGNMENT;
-    if (overlaps(grad, span_bytes(n, d_out, ld_grad, 2), s, span_bytes(g, n, ld_s, 4))) return GQ_ERR_INVALID_ARG;
+    const size_t g_bytes = span_bytes(n, d_out, ld_grad, 2), s_bytes = span_bytes(g, n, ld_s, 4);
+    if (overlaps(grad, g_bytes, s, s_bytes)) return GQ_ERR_INVALID_ARG;
+    if (prepare) {
+        const size_t ws_bytes = hessian_ws_bytes(n, 8, g);
+        if (!hessian_workspace || workspace_bytes < ws_bytes) return GQ_ERR_WORKSPACE;
+        if (!aligned(hessian_workspace, 1024)) return GQ_ERR_ALIGNMENT;
+        if (overlaps(hessian_workspace, ws_bytes, grad, g_bytes) || overlaps(hessian_workspace, ws_bytes, s, s_bytes))
+            return GQ_ERR_INVALID_ARG;
+    }
     DeviceInfo *di;
     if (int32_t rc = device_info(&di)) return rc;
     const int m = static_cast<int>(d_out / g);
     const float coef = grad_scale * grad_scale / static_cast<float>(m);
-    const int grid = grid_for(n * g * 32, 256, di->sm_count, di->saliency_blocks);    // one resident wave
+    const unsigned grid = static_cast<unsigned>((n * g + 7) / 8);            // one warp per (token, group) segment
     {
         LaunchScope scope(GQ_KERNEL_SALIENCY, static_cast<cudaStream_t>(stream));
         gq::saliency_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-            static_cast<const __nv_bfloat16 *>(grad), n, m, ld_grad, g, coef, s, ld_s);
+            static_cast<const __nv_bfloat16 *>(grad), static_cast<unsigned>(n), m, ld_grad, g, coef, s, ld_s,
+            prepare ? static_cast<uint32_t *>(hessian_workspace) : nullptr);
     }
     GQ_CUDA(cudaGetLastError());
     return GQ_OK;
 }
 
+int32_t gq_saliency(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad, int32_t g, float grad_scale,
+                    float *s, int64_t ld_s, void *stream)
+{
+    return saliency_impl(grad, n, d_out, ld_grad, g, grad_scale, s, ld_s, false, nullptr, 0, stream);
+}
+
+int32_t gq_saliency_prepared(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad, int32_t g, float grad_scale,
+                             float *s, int64_t ld_s, void *hessian_workspace, size_t workspace_bytes, void *stream)
+{
+    return saliency_impl(grad, n, d_out, ld_grad, g, grad_scale, s, ld_s, true, hessian_workspace, workspace_bytes, stream);
+}
+
 size_t gq_hessian_workspace_bytes(int64_t n_max, int64_t d_in, int32_t g, uint32_t flags)
 {
-    if ((flags & ~static_cast<uint32_t>(GQ_HESSIAN_DETERMINISTIC)) != 0 || n_max < 0 ||
+    if ((flags & ~static_cast<uint32_t>(GQ_HESSIAN_DETERMINISTIC | GQ_HESSIAN_S_PREPARED)) != 0 || n_max < 0 ||
         check_layer_shape(d_in, 0, g, false) != GQ_OK)
         return 0;
     return hessian_ws_bytes(n_max, d_in, g);
@@ -434,14 +449,15 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
                               int32_t g, float *H, uint32_t flags, void *workspace, size_t workspace_bytes,
                               void *stream)
 {
-    if (n < 0 || ld_x < d_in || ld_s < n || (flags & ~static_cast<uint32_t>(GQ_HESSIAN_DETERMINISTIC)) != 0)
+    if (n < 0 || ld_x < d_in || ld_s < n ||
+        (flags & ~static_cast<uint32_t>(GQ_HESSIAN_DETERMINISTIC | GQ_HESSIAN_S_PREPARED)) != 0)
         return GQ_ERR_INVALID_ARG;
     if (int32_t rc = check_layer_shape(d_in, 0, g, false)) return rc;
     if (n > (1ll << 31) - 64) return GQ_ERR_UNSUPPORTED_SHAPE;
     if (ld_x % 8 != 0) return GQ_ERR_ALIGNMENT;
     if (n == 0) return GQ_OK;              // an empty chunk adds nothing: pointers are not looked at
     if (!X || !s || !H) return GQ_ERR_INVALID_ARG;
-    if (!aligned(X, 16) || !aligned(H, 16) || !aligned(s, 4)) return GQ_ERR_ALIGNMENT;
+    if (!aligned(X, 16) || !aligned(H, 128) || !aligned(s, 4)) return GQ_ERR_ALIGNMENT;
     if (!workspace || workspace_bytes < hessian_ws_bytes(n, d_in, g)) return GQ_ERR_WORKSPACE;
     if (!aligned(workspace, 1024)) return GQ_ERR_ALIGNMENT;
     {
@@ -458,7 +474,7 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
     CUtensorMap mapX, mapH;
     if (int32_t rc = make_map(&mapX, X, d_in, n, 1, ld_x, n * ld_x)) return rc;
     if (int32_t rc = make_map_h(&mapH, H, d_in, g)) return rc;
-    {
+    if ((flags & GQ_HESSIAN_S_PREPARED) == 0) {
         const int grid_s = grid_for(static_cast<long long>((g + 1) / 2) * n, 256, di->sm_count, 4);
         {
             LaunchScope scope(GQ_KERNEL_SPLIT_SALIENCY, st);
@@ -499,7 +515,7 @@ int32_t gq_hessian_finalize(float *H, int64_t d_in, int32_t g, void *stream)
 {
     if (!H) return GQ_ERR_INVALID_ARG;
     if (int32_t rc = check_layer_shape(d_in, 0, g, false)) return rc;
-    if (!aligned(H, 16)) return GQ_ERR_ALIGNMENT;
+    if (!aligned(H, 128)) return GQ_ERR_ALIGNMENT;
     const unsigned nb = static_cast<unsigned>((d_in + 31) / 32);
     dim3 grid(nb, nb, static_cast<unsigned>(g));
     {
@@ -558,7 +574,7 @@ int32_t gq_hessian_gather_shares(float *const *H_ranks, int32_t ranks, int32_t r
 
 size_t gq_objective_workspace_bytes(int64_t d_in, int64_t d_out, int32_t g)
 {
-    if (check_layer_shape(d_in, d_out, g, true) != GQ_OK) return 0;
+    if (check_layer_shape(d_in, d_out, g, true) != GQ_OK || d_in * d_out >= (1ll << 33)) return 0;
     return objective_layout(d_in, d_out, g).total;
 }
 
@@ -567,7 +583,8 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
 {
     if (!W || !W_hat || !H || !loss_out) return GQ_ERR_INVALID_ARG;
     if (int32_t rc = check_layer_shape(d_in, d_out, g, true)) return rc;
-    if (!aligned(W, 16) || !aligned(W_hat, 16) || !aligned(H, 16) || !aligned(loss_out, 8)) return GQ_ERR_ALIGNMENT;
+    if (d_in * d_out >= (1ll << 33)) return GQ_ERR_UNSUPPORTED_SHAPE;      // 32-bit element indices in the preparation
+    if (!aligned(W, 16) || !aligned(W_hat, 16) || !aligned(H, 128) || !aligned(loss_out, 8)) return GQ_ERR_ALIGNMENT;
     const ObjectiveLayout L = objective_layout(d_in, d_out, g);
     if (!workspace || workspace_bytes < L.total) return GQ_ERR_WORKSPACE;
     if (!aligned(workspace, 1024)) return GQ_ERR_ALIGNMENT;
@@ -576,53 +593,54 @@ int32_t gq_objective(const float *W, const float *W_hat, int64_t d_in, int64_t d
     if (int32_t rc = device_info(&di)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint8_t *ws = static_cast<uint8_t *>(workspace);
-    __nv_bfloat16 *hi = reinterpret_cast<__nv_bfloat16 *>(ws + L.hi_off);
-    __nv_bfloat16 *lo = reinterpret_cast<__nv_bfloat16 *>(ws + L.lo_off);
+    gq::GramDotHeader *header = reinterpret_cast<gq::GramDotHeader *>(ws + L.header_off);
+    __half *dh = reinterpret_cast<__half *>(ws + L.half_off);
     double *partials = reinterpret_cast<double *>(ws + L.partials_off);
     const int64_t m = d_out / g;
+    // delta = W - W_hat as one fp16 matrix scaled by a power of two taken from max |delta| (two passes over W, W_hat)
+    GQ_CUDA(cudaMemsetAsync(header, 0, sizeof(gq::GramDotHeader), st));
     {
-        const long long count8 = d_in * d_out / 8;
-        const int grid = grid_for(count8, 256, di->sm_count, 8);
+        const unsigned count4 = static_cast<unsigned>(d_in * d_out / 4);
+        const unsigned per_block = 256u * gq::DELTA_VEC_PER_THREAD;
+        const unsigned blocks = (count4 + per_block - 1) / per_block;
         {
             LaunchScope scope(GQ_KERNEL_SPLIT_DELTA, st);
-            gq::split_delta_kernel<<<grid, 256, 0, st>>>(W, W_hat, count8, hi, lo);
+            gq::delta_absmax_kernel<<<blocks, 256, 0, st>>>(W, W_hat, count4, header);
+        }
+        GQ_CUDA(cudaGetLastError());
+        {
+            LaunchScope scope(GQ_KERNEL_SPLIT_DELTA, st);
+            gq::delta_half_kernel<<<blocks, 256, 0, st>>>(W, W_hat, count4, header, dh);
         }
         GQ_CUDA(cudaGetLastError());
     }
-    CUtensorMap mapHi, mapLo;
-    if (int32_t rc = make_map(&mapHi, hi, d_in, m, g, d_in, m * d_in)) return rc;
-    if (int32_t rc = make_map(&mapLo, lo, d_in, m, g, d_in, m * d_in)) return rc;
-    gq::PairGemmParams p{};
+    CUtensorMap mapD;
+    if (int32_t rc = make_map(&mapD, dh, d_in, m, g, d_in, m * d_in, CU_TENSOR_MAP_DATA_TYPE_FLOAT16)) return rc;
+    gq::GramDotParams p{};
     p.d = static_cast<int>(d_in);
     p.rows = static_cast<int>(m);
     p.g = g;
-    p.n_terms = 3;                     // hi^T hi + hi^T lo + lo^T hi
     p.nj = static_cast<int>((d_in + gq::TILE_N - 1) / gq::TILE_N);
-    p.raster = raster_for(di->max_pairs, g);
-    p.term_a[0] = 0; p.term_b[0] = 0;
-    p.term_a[1] = 0; p.term_b[1] = 1;
-    p.term_a[2] = 1; p.term_b[2] = 0;
-    p.map_grouped[0] = 1;
-    p.map_grouped[1] = 1;
-    // units: (row block, pair of neighbouring column tiles, group) over the upper triangle (gq_wide_gemm.cuh)
-    const int slots = colpair_slots_for(d_in);
+    // units: (256 x 256 tile on the upper triangle, group), group-major (gq_gram_dot.cuh)
+    p.tiles = tiles_for(d_in);
+    const int slots = p.tiles;
     const int units = slots * g;
-    const int ksteps = 3 * static_cast<int>((m + gq::TILE_K - 1) / gq::TILE_K);
-    p.sched = gq::plan_schedule(units, ksteps, units < di->max_pairs ? units : di->max_pairs, false);
+    const int ksteps = static_cast<int>((m + gq::TILE_K - 1) / gq::TILE_K);
+    const int pairs = units < di->max_pairs ? units : di->max_pairs;
+    p.raster = raster_for(pairs, 1);
+    p.sched = gq::plan_schedule(units, ksteps, pairs, false);
     p.H = H;
     p.partials = partials;
     p.status = di->status_ptr;
     p.wait_budget_ns = wait_budget_ns();
-    const int grid = 2 * p.sched.pairs;
     {
         LaunchScope scope(GQ_KERNEL_GRAM_DOT, st);
-        gq::wide_gemm_kernel<gq::WG_OBJECTIVE><<<grid, gq::WG_THREADS, gq::WG_SMEM_BYTES, st>>>(mapHi, mapLo, mapHi, mapLo, mapHi,
-                                                                                           mapLo, p);
+        gq::gram_dot_kernel<<<2 * p.sched.pairs, gq::GD_THREADS, gq::GD_SMEM_BYTES, st>>>(mapD, p);
     }
     GQ_CUDA(cudaGetLastError());
     {
         LaunchScope scope(GQ_KERNEL_REDUCE, st);
-        gq::reduce_partials_kernel<<<1, 1024, 0, st>>>(partials, slots, g, gq::WG_PARTIALS_PER_UNIT, loss_out);
+        gq::gram_dot_reduce_kernel<<<static_cast<unsigned>(g), 256, 0, st>>>(partials, slots, g, gq::GD_PARTIALS_PER_UNIT, header, loss_out);
     }
     GQ_CUDA(cudaGetLastError());
     return GQ_OK;
@@ -1176,8 +1194,9 @@ int32_t gq_layer_objective_host(const void *X_host, const void *grad_host, int64
         fail(cudaEventRecord(copied[b], copy_st));
         fail(cudaStreamWaitEvent(st, copied[b], 0));
         if (rc != GQ_OK) break;
-        rc = gq_saliency(gbuf[b], nt, d_out, d_out, g, grad_scale, s, chunk, st);
-        if (rc == GQ_OK) rc = gq_hessian_accumulate(xbuf[b], nt, d_in, d_in, s, chunk, g, H, 0, hws, hws_bytes, st);
+        rc = gq_saliency_prepared(gbuf[b], nt, d_out, d_out, g, grad_scale, s, chunk, hws, hws_bytes, st);
+        if (rc == GQ_OK)
+            rc = gq_hessian_accumulate(xbuf[b], nt, d_in, d_in, s, chunk, g, H, GQ_HESSIAN_S_PREPARED, hws, hws_bytes, st);
         if (rc == GQ_OK) fail(cudaEventRecord(consumed[b], st));
     }
     if (rc == GQ_OK) rc = gq_hessian_finalize(H, d_in, g, st);

@@ -9,10 +9,7 @@
 // hidden behind the next unit except for its first k-steps (same scheme as in gq_hessian.cuh), which the long
 // contraction (all of d_in, two terms) makes affordable.
 //
-// The objective (Eq. 7) runs the same way (WG_OBJECTIVE): a unit is (row block i, pair of column tiles 2q and
-// 2q + 1, group) over the upper triangle, A = B = Delta of the group (bf16 hi + lo, three terms), and the
-// epilogue contracts both accumulators with H_k as pair_gemm_kernel<MODE_OBJECTIVE> does, one fp64 partial per
-// (unit, CTA, epilogue warp), whole units only, so the result is reproducible.
+// (The objective of Eq. 7 runs on units of the same shape in a kernel of its own, gq_gram_dot.cuh.)
 //
 // Roles: warp 0 (one lane) TMA producer, warp 1 (one lane, first CTA) MMA issuer, warp 2 TMEM allocation,
 // warps 4..11 epilogue (tcgen05.ld, plain 16-byte stores; whole units only, one writer per element).
@@ -34,8 +31,6 @@ constexpr int WG_EPI_WARPS = 8;
 constexpr int WG_THREADS = 32 * (4 + WG_EPI_WARPS);
 constexpr int WG_SMEM_BYTES = WG_STAGES * WG_STAGE_BYTES + 1024;
 constexpr int WG_FULL = 0;
-constexpr int WG_OBJECTIVE = 1;
-constexpr int WG_PARTIALS_PER_UNIT = 2 * WG_EPI_WARPS;        // one fp64 per (CTA of the pair, epilogue warp)
 
 struct WideUnit {
     int ti;          // row block
@@ -44,10 +39,8 @@ struct WideUnit {
     int k;           // third coordinate of the grouped maps
 };
 
-// WG_FULL uses the MODE_FULL fields of PairGemmParams (d, rows, n_terms, term_a/b, map_grouped, full_k, col0,
-// cols, col_tiles, C, ldc), units = row blocks * ceil(col_tiles / 2); WG_OBJECTIVE the MODE_OBJECTIVE fields
-// (d, rows, g, nj, H, partials with WG_PARTIALS_PER_UNIT slots per unit), units = column-pair slots * g.
-// sched.ksteps = n_terms * ceil(rows / 64) in both.
+// Uses the MODE_FULL fields of PairGemmParams (d, rows, n_terms, term_a/b, map_grouped, full_k, col0, cols,
+// col_tiles, C, ldc), units = row blocks * ceil(col_tiles / 2), sched.ksteps = n_terms * ceil(rows / 64).
 template <int WMODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(WG_THREADS, 1)
 wide_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1,
@@ -101,26 +94,15 @@ wide_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
 
     auto decode = [&](int unit) {
         WideUnit u;
-        if (WMODE == WG_FULL) {
-            u.ti = unit / col_pairs;
-            u.tj[0] = 2 * (unit - u.ti * col_pairs);
-            u.tj[1] = u.tj[0] + 1;
-            u.use[0] = true;
-            u.use[1] = u.tj[1] < p.col_tiles;
-            u.k = p.full_k;
-        } else {
-            int i, q;
-            colpair_of_slot(unit / p.g, i, q);
-            u.ti = i;
-            u.tj[0] = 2 * q;
-            u.tj[1] = 2 * q + 1;
-            u.use[0] = 2 * q >= i;               // tile (i, 2q) touches the upper triangle
-            u.use[1] = 2 * q + 1 < p.nj;
-            u.k = unit % p.g;
-        }
+        u.ti = unit / col_pairs;
+        u.tj[0] = 2 * (unit - u.ti * col_pairs);
+        u.tj[1] = u.tj[0] + 1;
+        u.use[0] = true;
+        u.use[1] = u.tj[1] < p.col_tiles;
+        u.k = p.full_k;
         return u;
     };
-    const int col_base = (WMODE == WG_FULL) ? p.col0 : 0;
+    const int col_base = p.col0;
 
     if (warp == 0 && lane == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -258,72 +240,6 @@ wide_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
             const WideUnit u = decode(w.unit);
             const int row0 = u.ti * TILE_M + static_cast<int>(rank) * CTA_ROWS + q * 32;
             const int row = row0 + lane;
-            if (WMODE == WG_OBJECTIVE) {
-                // sum_{a <= b} (2 - [a == b]) D[a][b] H_k[a][b] over this warp's four 32 x 32 blocks of each
-                // accumulator.  The H values do not depend on the accumulators: the first block's are requested
-                // before the wait for the MMAs, every other block's while the block before it is being used.
-                const bool row_ok = row < p.d;
-                const float *hrow = p.H + (static_cast<size_t>(u.k) * p.d + (row_ok ? row : 0)) * static_cast<size_t>(p.d);
-                auto block_col0 = [&](int b) { return u.tj[b >> 2] * TILE_N + (half * 4 + (b & 3)) * 32; };
-                auto block_active = [&](int b) {                 // uniform over the warp
-                    const int col0 = block_col0(b);
-                    return u.use[b >> 2] && col0 < p.d && row0 < p.d && col0 + 32 > row0;
-                };
-                auto load_block = [&](int b, float4 (&h)[8]) {
-                    const int col0 = block_col0(b);
-                    const bool act = row_ok && block_active(b);
-#pragma unroll
-                    for (int v = 0; v < 8; ++v) {
-                        const int c = col0 + v * 4;
-                        h[v] = (act && c < p.d && c + 3 >= row) ? __ldg(reinterpret_cast<const float4 *>(hrow + c))
-                                                                : make_float4(0.f, 0.f, 0.f, 0.f);
-                    }
-                };
-                float4 hq[2][8];
-                load_block(0, hq[0]);
-                if (lane == 0) ok = bounded_wait(smem_u32(&bar_acc_full), acc_ph, wc, 4u, w.unit);
-                ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (!ok) break;
-                (void)mbar_try_wait(smem_u32(&bar_acc_full), acc_ph);     // every lane observes the completed phase
-                tc_fence_after_sync();
-                double dsum = 0.0;
-#pragma unroll
-                for (int b = 0; b < 8; ++b) {
-                    if (b + 1 < 8) load_block(b + 1, hq[(b + 1) & 1]);
-                    if (block_active(b)) {
-                        const int col0 = block_col0(b);
-                        uint32_t r[32];
-                        tmem_ld_32x32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
-                                          static_cast<uint32_t>((b >> 2) * TILE_N + (half * 4 + (b & 3)) * 32), r);
-                        tmem_ld_wait();
-                        float part = 0.0f;
-#pragma unroll
-                        for (int v = 0; v < 8; ++v) {
-                            const int c = col0 + v * 4;
-                            const float4 h = hq[b & 1][v];         // zero where it was not loaded
-                            const float hv[4] = {h.x, h.y, h.z, h.w};
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const float wgt = (c + e > row) ? 2.0f : ((c + e == row) ? 1.0f : 0.0f);
-                                part = fmaf(wgt * __uint_as_float(r[v * 4 + e]), hv[e], part);
-                            }
-                        }
-                        dsum += static_cast<double>(part);
-                    }
-                    if ((b & 3) == 3) {
-                        // This warp has read all it needs from accumulator b / 4: tell the MMA issuer (first CTA).
-                        tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_acc_empty[b >> 2]), 0));
-                    }
-                }
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, off);
-                if (lane == 0)
-                    p.partials[static_cast<size_t>(w.unit) * WG_PARTIALS_PER_UNIT + rank * WG_EPI_WARPS + ew] = dsum;
-                acc_ph ^= 1u;
-                continue;
-            }
             if (lane == 0) ok = bounded_wait(smem_u32(&bar_acc_full), acc_ph, wc, 4u, w.unit);
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;

@@ -46,11 +46,12 @@ def test_workspace_sizes(L):
     assert L.gq_hessian_workspace_bytes(8192, 4096, 4, 0) == 2 * 8192 * 8
     assert L.gq_hessian_workspace_bytes(8192, 4096, 5, 1) == 3 * 8192 * 8      # GQ_HESSIAN_DETERMINISTIC, odd g
     assert L.gq_hessian_workspace_bytes(1, 8, 1, 0) == 1024                    # rounded up to 1 KiB
-    assert L.gq_hessian_workspace_bytes(8192, 4096, 4, 2) == 0                 # unknown flag
+    assert L.gq_hessian_workspace_bytes(8192, 4096, 4, 4) == 0                 # unknown flag
+    assert L.gq_hessian_workspace_bytes(8192, 4096, 4, 3) == 2 * 8192 * 8      # both known flags
     assert L.gq_hessian_workspace_bytes(8192, 4100, 4, 0) == 0                 # d_in % 8 != 0
-    # objective: two bf16 copies of delta + room for 16 fp64 partial sums per (upper-triangular 256 x 256 tile, group)
+    # objective: a 1 KiB header, delta as one fp16 matrix, 16 fp64 partial sums per (upper-triangular 256 x 256 tile, group)
     nj = 4096 // 256
-    assert L.gq_objective_workspace_bytes(4096, 4096, 4) == 2 * 4096 * 4096 * 2 + (nj * (nj + 1) // 2) * 4 * 16 * 8
+    assert L.gq_objective_workspace_bytes(4096, 4096, 4) == 1024 + 4096 * 4096 * 2 + (nj * (nj + 1) // 2) * 4 * 16 * 8
     assert L.gq_objective_workspace_bytes(4096, 4096, 3) == 0          # d_out % g != 0
     assert L.gq_objective_workspace_bytes(4096, 24, 6) == 0            # (d_out / g) % 8 != 0
     assert L.gq_layer_host_arena_bytes(0, 4096, 4096, 4) == 0
@@ -67,9 +68,9 @@ def test_workspace_sizes(L):
 
 
 def test_host_side_validation_needs_no_gpu(L):
-    buf = (ctypes.c_uint8 * 4096)()
+    buf = (ctypes.c_uint8 * 8192)()
     p = ctypes.addressof(buf)
-    p16 = (p + 15) // 16 * 16
+    p16 = (p + 127) // 128 * 128           # 128-byte aligned: what H needs; the other pointers need 16
     INVALID, ALIGN, SHAPE, WS = -1, -2, -3, -4
     # saliency
     assert L.gq_saliency(p16, -1, 64, 64, 2, 1.0, p16, 0, None) == INVALID
@@ -82,7 +83,7 @@ def test_host_side_validation_needs_no_gpu(L):
     assert L.gq_saliency(None, 4, 64, 64, 2, 1.0, p16, 4, None) == INVALID
     assert L.gq_saliency(None, 0, 64, 64, 2, 1.0, None, 0, None) == 0          # empty call: no-op
     # hessian
-    assert L.gq_hessian_accumulate(p16, 4, 64, 64, p16, 4, 2, p16, 2, p16, 4096, None) == INVALID   # flags
+    assert L.gq_hessian_accumulate(p16, 4, 64, 64, p16, 4, 2, p16, 4, p16, 4096, None) == INVALID   # flags
     assert L.gq_hessian_accumulate(p16, 4, 60, 64, p16, 4, 2, p16, 0, p16, 4096, None) == SHAPE     # d_in % 8
     assert L.gq_hessian_accumulate(p16, 4, 64, 64, p16, 4, 2, p16 + 4, 0, p16, 4096, None) == ALIGN
     assert L.gq_hessian_accumulate(p16, 4, 64, 64, p16, 4, 2, p16, 0, None, 0, None) == WS

@@ -3,13 +3,14 @@
 Tolerances of this path:
   saliency   |s - s_o| <= 1e-4 * |s_o| per element (plus a floor of 1e-4 * max|s_o| * 1e-6 for zeros)
   Hessian    ||H_k - H_k_o||_F <= 5e-3 ||H_k_o||_F   and   max|H_k - H_k_o| <= 1e-2 max|H_k_o|
-             and, entry by entry, |H_k - H_k_o|[a][b] <= 3e-3 sqrt(H_k_o[a][a] H_k_o[b][b])
+             and, entry by entry, |H_k - H_k_o|[a][b] <= 4.5e-3 sqrt(H_k_o[a][a] H_k_o[b][b])
   objective  |loss - loss_o| <= 1e-3 |loss_o|
 The entry-wise bound does not depend on the scale of a feature (the first two are set by the few outlier
 features): the only rounding of the Hessian kernel that is not of fp32 size is the one bf16 rounding of each
-product s_k[i] X[i][a], a relative error of at most 2^-9, so
-|error of H[a][b]| <= 2^-9 sum_i s_i |X[i][a]| |X[i][b]| <= 2^-9 sqrt(H[a][a] H[b][b]) (Cauchy-Schwarz) = 1.95e-3 of
-that geometric mean; 3e-3 leaves room for the two-term saliency (2^-17) and fp32 accumulation.
+product s_k[i] X[i][a] (8 significant bits), a relative error of at most 2^-8, so
+|error of H[a][b]| <= 2^-8 sum_i s_i |X[i][a]| |X[i][b]| <= 2^-8 sqrt(H[a][a] H[b][b]) (Cauchy-Schwarz) = 3.9e-3 of
+that geometric mean, reached only by a single token whose product rounds by half a unit; 4.5e-3 leaves room for
+the two-term saliency (2^-17) and fp32 accumulation.
 """
 import numpy as np
 import pytest
@@ -21,7 +22,7 @@ from paper_2505_07004_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
-S_RTOL, H_FRO, H_MAX, H_ENTRY, L_RTOL = 1e-4, 5e-3, 1e-2, 3e-3, 1e-3
+S_RTOL, H_FRO, H_MAX, H_ENTRY, L_RTOL = 1e-4, 5e-3, 1e-2, 4.5e-3, 1e-3
 
 
 @pytest.fixture(scope="module")
@@ -162,6 +163,32 @@ def test_hessian_unit_saliency_is_gram_and_deterministic(dev):
     assert rel.item() < 1e-5            # unit weights are exact in bf16: only fp32 accumulation error remains
 
 
+@pytest.mark.parametrize("n,d_in,d_out,g", [(700, 520, 512, 4), (333, 264, 120, 3), (64, 256, 8, 1)])
+def test_prepared_saliency_gives_the_same_hessian(dev, n, d_in, d_out, g):
+    """gq_saliency_prepared + GQ_HESSIAN_S_PREPARED (two launches) against gq_saliency + gq_hessian_accumulate
+    (three): same fp32 s, and with the single-writer schedule the same H bit for bit."""
+    gen = torch.Generator(device=dev).manual_seed(n + d_in + g)
+    X = torch.randn(n, d_in, generator=gen, device=dev).to(torch.bfloat16)
+    grad = (torch.randn(n, d_out, generator=gen, device=dev) * torch.exp(torch.randn(n, 1, generator=gen, device=dev)))
+    grad = grad.to(torch.bfloat16)
+    flags = libgq.GQ_HESSIAN_DETERMINISTIC
+    ws = libgq.alloc_workspace(libgq.gq_hessian_workspace_bytes(n, d_in, g, flags), dev)
+    s1 = libgq.gq_saliency(grad, g)
+    H1 = torch.zeros((g, d_in, d_in), dtype=torch.float32, device=dev)
+    libgq.gq_hessian_accumulate(X, s1, H1, ws, flags=flags)
+    ws.fill_(0xFF)                                       # nothing of the first run may be left in the workspace
+    s2 = libgq.gq_saliency_prepared(grad, g, ws)
+    H2 = torch.zeros_like(H1)
+    libgq.gq_hessian_accumulate(X, s2, H2, ws, flags=flags | libgq.GQ_HESSIAN_S_PREPARED)
+    libgq.gq_check()
+    assert torch.equal(s1, s2)
+    assert torch.equal(H1, H2)
+    check_s(s2, orc.saliency(synth.bf16_bits(grad), g))
+    with pytest.raises(libgq.GQError) as e:
+        libgq.gq_saliency_prepared(grad, g, ws[:8])
+    assert "GQ_ERR_WORKSPACE" in str(e.value)
+
+
 def test_hessian_errors(dev):
     X = torch.zeros((16, 64), dtype=torch.bfloat16, device=dev)
     s = torch.zeros((2, 16), dtype=torch.float32, device=dev)
@@ -171,7 +198,7 @@ def test_hessian_errors(dev):
         libgq.gq_hessian_accumulate(X, s, H, ws[:16])
     assert "GQ_ERR_WORKSPACE" in str(e.value)
     with pytest.raises(libgq.GQError) as e:
-        libgq.gq_hessian_accumulate(X, s, H, ws, flags=2)
+        libgq.gq_hessian_accumulate(X, s, H, ws, flags=4)
     assert "GQ_ERR_INVALID_ARG" in str(e.value)
     Xbad = torch.zeros((16, 68), dtype=torch.bfloat16, device=dev)
     Hbad = torch.zeros((2, 68, 68), dtype=torch.float32, device=dev)
@@ -219,7 +246,8 @@ def test_objective_zero_and_single_entry(dev):
     loss = libgq.gq_objective(W, W.clone(), H, ws)
     libgq.gq_check()
     assert torch.count_nonzero(loss).item() == 0
-    # a single perturbed weight with a value that bf16 cannot hold: the hi/lo split must recover it
+    # a single perturbed weight with a value that neither fp16 nor bf16 holds exactly: the result must still be
+    # inside the objective's tolerance (11 significant bits per factor: 2^-11 at worst)
     What = W.clone()
     What[11, 77] += 0.123456789
     loss = libgq.gq_objective(W, What, H, ws)
@@ -228,7 +256,7 @@ def test_objective_zero_and_single_entry(dev):
     expect = delta * delta * float(H[1, 77, 77])
     got = loss.cpu().numpy()
     assert got[0] == 0.0
-    assert abs(got[1] - expect) <= 1e-4 * expect and abs(got[2] - expect) <= 1e-4 * expect
+    assert abs(got[1] - expect) <= L_RTOL * expect and abs(got[2] - expect) <= L_RTOL * expect
 
 
 # ------------------------------------------------------------------------------------------ whole path
@@ -243,8 +271,8 @@ def run_layer(cfg, dev, n_tokens=None, grad_scale=1.0, seed=0):
     while done < n:
         nt = min(cfg.chunk, n - done)
         X, grad = syn.x_chunk(c, nt), syn.grad_chunk(c, nt)
-        s = libgq.gq_saliency(grad, g, grad_scale)
-        libgq.gq_hessian_accumulate(X, s, H, ws)
+        s = libgq.gq_saliency_prepared(grad, g, ws, grad_scale)          # the two launches per chunk bench.py makes
+        libgq.gq_hessian_accumulate(X, s, H, ws, flags=libgq.GQ_HESSIAN_S_PREPARED)
         xs.append(X), gs.append(grad), ss.append(s)
         done += nt
         c += 1

@@ -31,8 +31,9 @@ def run_path(cfg, xs, gs, W, What, bufs):
     H.zero_()
     for x, gr in zip(xs, gs):
         nt = x.shape[0]
-        libgq.gq_saliency(gr, g, 1.0, s=s_buf[:, :nt])
-        libgq.gq_hessian_accumulate(x, s_buf[:, :nt], H, ws, flags=libgq.GQ_HESSIAN_DETERMINISTIC)
+        libgq.gq_saliency_prepared(gr, g, ws, 1.0, s=s_buf[:, :nt])
+        libgq.gq_hessian_accumulate(x, s_buf[:, :nt], H, ws,
+                                    flags=libgq.GQ_HESSIAN_DETERMINISTIC | libgq.GQ_HESSIAN_S_PREPARED)
     libgq.gq_hessian_finalize(H)
     libgq.gq_objective(W, What, H, ows, loss=loss)
 
@@ -67,7 +68,7 @@ def test_side_stream_and_graph_replay_match_the_default_stream(dev):
     with torch.cuda.graph(graph):
         run_path(cfg, xs, gs, W, What, b2)
     per_step = libgq.gq_launch_count() - launches0
-    assert per_step == 3 * cfg.n_chunks + 4          # saliency, split, Hessian per chunk; mirror, split, dot, reduce
+    assert per_step == 2 * cfg.n_chunks + 5          # saliency, Hessian per chunk; mirror, maximum, fp16, dot, reduce
     for _ in range(2):
         b2[0].fill_(7.0)
         b2[4].zero_()
