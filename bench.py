@@ -46,6 +46,7 @@ NCU_TRAFFIC_BYTES = {"c1_7b_attn": 343.36e6}
 # The oracle sample both the cpu_baseline leg and --impl reference time (one size, so that the oracle's
 # throughput is one number): tokens of chunk 0 for saliency + Hessian, channels per group for the objective.
 ORACLE_SAMPLE_TOKENS, ORACLE_SAMPLE_CHANNELS = 1024, 64
+OBJ_B2B_CALLS = 10           # calls of gq_objective inside one event pair
 SAL_B2B_PASSES = 5           # passes over all chunks in the back-to-back saliency measurement
 OBJECTIVE_KERNELS = ("split_delta", "gram_dot", "reduce")     # the kernels one gq_objective call launches
 CPU_BASELINE_PASSES = 4      # passes of that sample in the cpu_baseline leg (about 10-15 s of host time)
@@ -191,6 +192,81 @@ def run_reference(args, cfg, g):
     print(json.dumps(out), flush=True)
 
 
+def run_token_sharded(libgq, cfg, g, dev, rank, world):
+    """One token-sharded layer on `world` GPUs: rank r accumulates chunks r, r + world, ... of the SAME synthetic layer
+    into its own H (allocated in memory every rank can address), then the partial matrices are added by
+    gq_hessian_reduce_share / gq_hessian_gather_shares with host barriers in between (plain peer loads; no kernel
+    waits for another GPU).  Not part of the timed region of the headline number.  Returns the record for the JSON
+    line (identical on every rank), or {"error": ...} if peer memory could not be set up."""
+    import torch.distributed as dist
+
+    def all_ok(ok):
+        flag = torch.tensor([1 if ok else 0], dtype=torch.int32, device=dev)
+        dist.all_reduce(flag, op=dist.ReduceOp.MIN)
+        return bool(flag.item())
+
+    try:
+        H, ptrs, err = None, None, None
+        try:
+            H, ptrs = shard.allocate_symmetric_hessian(g, cfg.d_in, dev)
+        except Exception as exc:
+            err = repr(exc)[:300]
+        if not all_ok(err is None):                             # every rank takes the same way out
+            return {"error": err or "peer memory could not be set up on another rank"}
+        syn = synth.LayerSynth(cfg, dev, seed=0)
+        ws = libgq.alloc_workspace(libgq.gq_hessian_workspace_bytes(cfg.chunk, cfg.d_in, g), dev)
+        mine = shard.chunks_for_rank(cfg.n_chunks, rank, world)
+        xs = [syn.x_chunk(c) for c in mine]
+        gs = [syn.grad_chunk(c) for c in mine]
+        rank_ptrs = [H if r == rank else ptrs[r] for r in range(world)]
+
+        def accumulate(Hbuf, xs_, gs_):
+            for x, gr in zip(xs_, gs_):
+                sb = libgq.gq_saliency_prepared(gr, g, ws, 1.0)
+                libgq.gq_hessian_accumulate(x, sb, Hbuf, ws, flags=libgq.GQ_HESSIAN_S_PREPARED)
+
+        accumulate(H, xs, gs)                                   # warm-up of kernels and peer mappings
+        shard.exchange_hessian(H, rank_ptrs, rank)
+        torch.cuda.synchronize()
+        dist.barrier()
+        H.zero_()
+        torch.cuda.synchronize()
+        dist.barrier()
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record()
+        accumulate(H, xs, gs)
+        e[1].record()
+        shard.exchange_hessian(H, rank_ptrs, rank)
+        e[2].record()
+        torch.cuda.synchronize()
+        libgq.gq_check()
+        ms_acc, ms_ex = e[0].elapsed_time(e[1]), e[1].elapsed_time(e[2])
+        # every rank must hold the same bits: compare a checksum of the bit patterns
+        bits = H.view(torch.int32).to(torch.int64)
+        checksum = torch.stack([bits.sum(), (bits * (torch.arange(bits.numel(), device=dev).view_as(bits) % 1021)).sum()])
+        sums = [torch.zeros_like(checksum) for _ in range(world)]
+        dist.all_gather(sums, checksum)
+        bit_equal = all(bool(torch.equal(t, sums[0])) for t in sums)
+        # rank 0 also builds the layer unsharded and compares (summation order differs)
+        rel = torch.zeros(1, dtype=torch.float64, device=dev)
+        if rank == 0:
+            H1 = torch.zeros_like(H)
+            accumulate(H1, [syn.x_chunk(c) for c in range(cfg.n_chunks)], [syn.grad_chunk(c) for c in range(cfg.n_chunks)])
+            libgq.gq_hessian_finalize(H1)
+            libgq.gq_check()
+            rel[0] = ((H.double() - H1.double()).norm() / H1.double().norm()).item()
+            del H1
+        dist.broadcast(rel, 0)
+        ms_acc, ms_ex = shard.max_over_ranks([ms_acc, ms_ex], device=dev)
+        nvl = shard.exchange_bytes_per_rank(cfg.d_in, g, world)
+        return {"ms_accumulate": ms_acc, "ms_exchange": ms_ex, "bytes_over_nvlink": nvl,
+                "exchange_gbs_per_rank": nvl / (ms_ex * 1e-3) / 1e9 if ms_ex > 0 else None,
+                "all_ranks_bit_equal": bit_equal, "max_rel_vs_rank0_unsharded": float(rel.item()),
+                "chunks_per_rank": len(mine), "note": "exchange time includes its three host barriers and the mirror step"}
+    except Exception as exc:      # peer memory unavailable etc.: the headline numbers stand, the leg reports why it did not run
+        return {"error": repr(exc)[:300]}
+
+
 def run_ours(args, cfg, g):
     from paper_2505_07004_b200 import api as libgq
     rank, local_rank, world = dist_env()
@@ -264,20 +340,42 @@ def run_ours(args, cfg, g):
     if not np.all(np.isfinite(loss_host)) or loss_host[g] <= 0:
         raise RuntimeError("objective is not finite/positive: %s" % loss_host)
 
-    # ---- saliency alone, back to back over all chunks (no per-launch event pair in the way)
+    # ---- saliency alone: all chunks' launches captured into one CUDA graph (no host time between launches, no
+    # per-launch event pair), replayed SAL_B2B_PASSES times inside one event pair
     sal_b2b_gbs = None
     if n_chunks * cfg.chunk * cfg.d_out * 2 > 200e6:                    # only meaningful when a pass exceeds L2
-        for c in range(n_chunks):
-            libgq.gq_saliency(gs[c], g, 1.0, s=s_buf[:, :gs[c].shape[0]])
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for c in range(n_chunks):
+                libgq.gq_saliency_prepared(gs[c], g, ws, 1.0, s=s_buf[:, :gs[c].shape[0]])
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for c in range(n_chunks):
+                libgq.gq_saliency_prepared(gs[c], g, ws, 1.0, s=s_buf[:, :gs[c].shape[0]])
+        graph.replay()
         torch.cuda.synchronize()
         b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         b0.record()
         for _ in range(SAL_B2B_PASSES):
-            for c in range(n_chunks):
-                libgq.gq_saliency(gs[c], g, 1.0, s=s_buf[:, :gs[c].shape[0]])
+            graph.replay()
         b1.record()
         torch.cuda.synchronize()
         sal_b2b_gbs = SAL_B2B_PASSES * sum(x.shape[0] * (2 * cfg.d_out + 4 * g) for x in gs) / (b0.elapsed_time(b1) * 1e-3) / 1e9
+        del graph
+
+    # ---- the objective alone: OBJ_B2B_CALLS calls inside one event pair (its inputs, W, W_hat and H, exceed L2)
+    libgq.gq_objective(W, What, H, ows, loss=loss)
+    torch.cuda.synchronize()
+    o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    o0.record()
+    for _ in range(OBJ_B2B_CALLS):
+        libgq.gq_objective(W, What, H, ows, loss=loss)
+    o1.record()
+    torch.cuda.synchronize()
+    obj_b2b_ms = o0.elapsed_time(o1) / OBJ_B2B_CALLS
+    libgq.gq_check()
 
     # ---- end to end from pinned host memory through the host-buffer entry point
     e2e_s, e2e_steps, h2d, d2h = float('nan'), 0, 0, 0
@@ -309,6 +407,12 @@ def run_ours(args, cfg, g):
             raise RuntimeError("host-buffer path and device path disagree: %r vs %r" % (loss_h[g].item(), loss_host[g]))
         h2d = Xh.numel() * 2 + Gh.numel() * 2 + Wh.numel() * 4 + Whh.numel() * 4
         d2h = (g + 1) * 8
+
+    # ---- N > 1 only: ONE layer (seed of rank 0) with its token chunks dealt to the ranks, partial matrices added
+    # by the library's exchange kernels over peer memory (Algorithm 1, Hessian step: H is a sum over tokens)
+    token_sharded = None
+    if world > 1 and not args.no_token_sharded:
+        token_sharded = run_token_sharded(libgq, cfg, g, dev, rank, world)
 
     # ---- max over ranks
     ms_total, e2e_ms = shard.max_over_ranks([ms_total, e2e_s * 1e3], device=dev)
@@ -356,25 +460,28 @@ def run_ours(args, cfg, g):
         }
         sal_gbs = (sal_bytes / (sal_ms / max(1, sal_n) * 1e-3) / 1e9) if sal_n else None
         saliency_roofline = {
-            "kernel": "saliency_kernel (gq_saliency)", "bound": "hbm", "unit": "GB/s", "peak": peaks["hbm_gbs"],
+            "kernel": "saliency_kernel (gq_saliency_prepared)", "bound": "hbm", "unit": "GB/s", "peak": peaks["hbm_gbs"],
             "bytes_per_launch": sal_bytes,
-            "achieved": sal_gbs, "frac": frac(sal_gbs, peaks["hbm_gbs"]),
-            "timing": "event pair around each launch inside the step (a %d MB launch lasts ~10-20 us: the pair's own "
-                      "cost is part of this figure)" % (sal_bytes // 1000000),
-            "achieved_back_to_back": sal_b2b_gbs, "frac_back_to_back": frac(sal_b2b_gbs, peaks["hbm_gbs"]),
-            "timing_back_to_back": "one event pair around %d passes over all %d chunks (%.2f GB per pass, larger than L2)"
-                                   % (SAL_B2B_PASSES, n_chunks, n_chunks * sal_bytes / 1e9),
+            "achieved": sal_b2b_gbs, "frac": frac(sal_b2b_gbs, peaks["hbm_gbs"]),
+            "timing": "one event pair around %d replays of a CUDA graph holding the launches of all %d chunks "
+                      "(%.2f GB per replay, larger than L2)" % (SAL_B2B_PASSES, n_chunks, n_chunks * sal_bytes / 1e9),
+            "achieved_per_launch_events": sal_gbs, "frac_per_launch_events": frac(sal_gbs, peaks["hbm_gbs"]),
+            "timing_per_launch_events": "event pair around each launch inside the step (a %d MB launch lasts ~12 us: the "
+                                        "pair's own cost is part of this figure)" % (sal_bytes // 1000000),
         }
         objective_roofline = None
         if kern["gram_dot"][1]:
             calls = kern["gram_dot"][1]
-            obj_ms = sum(kern[k][0] for k in OBJECTIVE_KERNELS) / calls
+            obj_events_ms = sum(kern[k][0] for k in OBJECTIVE_KERNELS) / calls
+            obj_ms = obj_b2b_ms
             obj_bytes = 2.0 * g * cfg.d_in * (cfg.d_in + 1) + 8.0 * cfg.d_in * cfg.d_out     # upper triangle of H (fp32) + W, W_hat
             obj_flops_sym = float(cfg.d_in) * cfg.d_in * cfg.d_out                           # 2 d_in^2 d_out, halved by symmetry
             t_bytes = obj_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
             t_flops = obj_flops_sym / (peaks["bf16_tflops"] * 1e12) * 1e3
             objective_roofline = {
                 "kernel": "gq_objective (all of its kernels)", "ms_per_call": obj_ms,
+                "timing": "one event pair around %d back-to-back calls" % OBJ_B2B_CALLS,
+                "ms_per_call_kernel_events": obj_events_ms,
                 "bound": "tensor" if t_flops >= t_bytes else "hbm",
                 "algorithmic_bytes": obj_bytes, "symmetric_flops": obj_flops_sym,
                 "ms_at_hbm_peak": t_bytes, "ms_at_tensor_burst_peak": t_flops,
@@ -403,6 +510,8 @@ def run_ours(args, cfg, g):
             "clocks": clocks,
             "loss_total": float(loss_host[g]),
         }
+        if token_sharded is not None:
+            out["token_sharded"] = token_sharded
         if world == 1 and not args.no_cpu_baseline:
             from oracle import gq_oracle as orc
             orc.build()
@@ -436,6 +545,7 @@ def main():
     ap.add_argument("--ref-channels", type=int, default=ORACLE_SAMPLE_CHANNELS)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-token-sharded", action="store_true", help="N > 1: skip the token-sharded layer with the peer-memory exchange")
     ap.add_argument("--tokens", type=int, default=0, help="use only the first TOKENS tokens (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -83,6 +83,28 @@ int32_t gq_saliency_prepared(const void *grad, int64_t n, int64_t d_out, int64_t
                              size_t workspace_bytes, void *stream);
 
 /*
+ * Saliency at the source (Algorithm 1, saliency step; Section 3.2: of the end-loss gradients only the averaged
+ * squares are kept, O(n g) numbers per layer): the same reduction for dl/dZ in the dtype and layout a backward
+ * pass hands it over, written straight into the caller's calibration-wide s, so that a backward hook keeps nothing
+ * but s.
+ *
+ *   grad        [batch, seq, d_out] with element strides (stride_b, stride_t, 1); token i = b * seq + t.
+ *               16-byte aligned; stride_t >= d_out; both strides multiples of 16 bytes (8 elements for the 16-bit
+ *               types, 4 for fp32); sequences must not overlap
+ *   dtype       GQ_DTYPE_BF16, GQ_DTYPE_FP16 (IEEE half) or GQ_DTYPE_FP32
+ *   s           fp32 [g, ld_s], ld_s >= batch * seq; s[k * ld_s + i] is written (pass s + offset of the first token
+ *               and the leading dimension of the whole buffer to fill a slice of a larger array)
+ * Other rules as for gq_saliency: d_out % g == 0, (d_out / g) % 8 == 0, batch * seq * g < 2^31, grad_scale finite.
+ * Values are widened to fp32 exactly; squares and sums are fp32.
+ * (There is no accumulating form: squares of partial gradients do not add up to the square of their sum, so
+ * the gradient of a token has to be complete when it is reduced.)
+ */
+enum gq_dtype { GQ_DTYPE_BF16 = 0, GQ_DTYPE_FP16 = 1, GQ_DTYPE_FP32 = 2 };
+int32_t gq_saliency_strided(const void *grad, int32_t dtype, int64_t batch, int64_t seq, int64_t d_out,
+                            int64_t stride_b, int64_t stride_t, int32_t g, float grad_scale, float *s,
+                            int64_t ld_s, void *stream);
+
+/*
  * Guided Hessian, one token chunk: Algorithm 1, Hessian step, streamed,
  *     H[k][a][b] += sum_{i < n} s[k * ld_s + i] * X[i * ld_x + a] * X[i * ld_x + b]
  * for every group k and every a <= b (the upper triangle including the diagonal).  No 1/n factor.

@@ -54,6 +54,53 @@ int gq_oracle_saliency(const uint16_t *grad, int64_t n, int64_t d_out, int64_t l
 }
 
 /*
+ * The same saliency for a gradient as a backward pass hands it over (Section 3.2: only the averaged squared
+ * gradients of a layer are kept): a [batch][seq][d_out] array with element strides (stride_b, stride_t, 1),
+ * stored as bf16 (dtype 0), IEEE half (dtype 1) or fp32 (dtype 2); token i = b * seq + t.  Every input value
+ * widens to fp64 without rounding.  s: [g][ld_s] fp64.  Returns 0, or -1 on bad sizes / an unknown dtype.
+ */
+static double half_to_f64(uint16_t h)
+{
+    const int sign = (h >> 15) & 1, expo = (h >> 10) & 0x1f, frac = h & 0x3ff;
+    double v;
+    if (expo == 0) v = (double)frac / 1024.0 / 16384.0;                       /* subnormal: frac * 2^-24 */
+    else if (expo == 31) v = frac ? (0.0 / 0.0) : (1.0 / 0.0);
+    else {
+        v = 1.0 + (double)frac / 1024.0;
+        for (int e = expo; e > 15; --e) v *= 2.0;
+        for (int e = expo; e < 15; ++e) v *= 0.5;
+    }
+    return sign ? -v : v;
+}
+
+int gq_oracle_saliency_strided(const void *grad, int32_t dtype, int64_t batch, int64_t seq, int64_t d_out,
+                               int64_t stride_b, int64_t stride_t, int32_t g, double grad_scale, double *s,
+                               int64_t ld_s)
+{
+    if (g < 1 || d_out < 1 || d_out % g != 0 || batch < 0 || seq < 0 || ld_s < batch * seq) return -1;
+    if (dtype < 0 || dtype > 2) return -1;
+    const int64_t m = d_out / g;
+    for (int32_t k = 0; k < g; ++k) {
+#pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < batch * seq; ++i) {
+            const int64_t b = i / seq, t = i % seq;
+            const int64_t base = b * stride_b + t * stride_t;
+            double acc = 0.0;
+            for (int64_t j = m * k; j < m * (k + 1); ++j) {
+                double v;
+                if (dtype == 0) v = bf16_to_f64(((const uint16_t *)grad)[base + j]);
+                else if (dtype == 1) v = half_to_f64(((const uint16_t *)grad)[base + j]);
+                else v = (double)((const float *)grad)[base + j];
+                const double gij = grad_scale * v;
+                acc += gij * gij;
+            }
+            s[(int64_t)k * ld_s + i] = acc / (double)m;
+        }
+    }
+    return 0;
+}
+
+/*
  * Algorithm 1, Hessian step:  H_k = X^T Diag(s_k) X, i.e.
  *   H_k[a][b] (+)= sum_{i=1..n} s_k[i] * X[i][a] * X[i][b]      for all a, b.
  * No 1/n factor (Section 3.2 writes the unguided case as H = X^T X).

@@ -49,6 +49,8 @@ def _c():
         lib.gq_oracle_saliency.argtypes = [vp, i64, i64, i64, i32, dbl, vp, i64]
         lib.gq_oracle_hessian_accumulate.argtypes = [vp, i64, i64, i64, vp, i64, i32, vp]
         lib.gq_oracle_objective.argtypes = [vp, vp, i64, i64, vp, i32, vp]
+        lib.gq_oracle_saliency_strided.argtypes = [vp, i32, i64, i64, i64, i64, i64, i32, dbl, vp, i64]
+        lib.gq_oracle_saliency_strided.restype = ctypes.c_int
         lib.gq_oracle_hessian_diag.argtypes = [vp, i64, i64, i64, vp, i64, i32, vp]
         lib.gq_oracle_hessian_apply.argtypes = [vp, i64, i64, i64, vp, i64, i32, vp, i32, vp]
         for f in (lib.gq_oracle_saliency, lib.gq_oracle_hessian_accumulate, lib.gq_oracle_objective,
@@ -92,6 +94,36 @@ def saliency(grad_bits: np.ndarray, g: int, grad_scale: float = 1.0, impl: str =
     rc = _c().gq_oracle_saliency(_ptr(grad_bits), n, d_out, d_out, g, float(grad_scale), _ptr(s), n)
     if rc:
         raise RuntimeError("gq_oracle_saliency rc=%d" % rc)
+    return s
+
+
+DTYPE_CODES = {"bf16": 0, "fp16": 1, "fp32": 2}
+
+
+def saliency_strided(grad: np.ndarray, dtype: str, g: int, grad_scale: float = 1.0, impl: str = "c") -> np.ndarray:
+    """Algorithm 1's saliency for a gradient as autograd hands it over: ``grad`` is ``[batch, seq, d_out]`` with a
+    contiguous last dimension and arbitrary (non-negative) strides of the first two, holding bf16 bit patterns
+    (``uint16``, dtype "bf16"), IEEE half (``float16``, "fp16") or ``float32`` ("fp32").  Token ``i = b * seq + t``.
+    Returns fp64 ``[g, batch * seq]``."""
+    if grad.ndim != 3 or (grad.shape[2] > 1 and grad.strides[2] != grad.itemsize):
+        raise ValueError("grad must be [batch, seq, d_out] with a contiguous last dimension")
+    want = {"bf16": np.uint16, "fp16": np.float16, "fp32": np.float32}[dtype]
+    if grad.dtype != want:
+        raise ValueError("dtype %s needs a %s array" % (dtype, want))
+    batch, seq, d_out = grad.shape
+    if g < 1 or d_out % g:
+        raise ValueError("d_out must be divisible by g")
+    n = batch * seq
+    if impl == "numpy":
+        wide = bf16_bits_to_f64(np.ascontiguousarray(grad)).reshape(grad.shape) if dtype == "bf16" else grad.astype(np.float64)
+        gr = wide.reshape(n, g, d_out // g) * float(grad_scale)
+        return np.ascontiguousarray((gr * gr).mean(axis=2).T)
+    s = np.zeros((g, n), dtype=np.float64)
+    sb, st = grad.strides[0] // grad.itemsize, grad.strides[1] // grad.itemsize
+    rc = _c().gq_oracle_saliency_strided(ctypes.c_void_p(grad.ctypes.data), DTYPE_CODES[dtype], batch, seq, d_out, sb, st, g,
+                                         float(grad_scale), _ptr(s), n)
+    if rc:
+        raise RuntimeError("gq_oracle_saliency_strided rc=%d" % rc)
     return s
 
 

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libgq.so")
 _lib = None
 
 EXPORTS = (
-    "gq_version", "gq_status_string", "gq_last_cuda_error", "gq_saliency", "gq_saliency_prepared", "gq_hessian_accumulate",
+    "gq_version", "gq_status_string", "gq_last_cuda_error", "gq_saliency", "gq_saliency_prepared", "gq_saliency_strided", "gq_hessian_accumulate",
     "gq_hessian_workspace_bytes", "gq_hessian_finalize", "gq_objective", "gq_objective_workspace_bytes",
     "gq_layer_objective_host", "gq_layer_host_arena_bytes", "gq_check", "gq_launch_count",
     "gq_kernel_timing_enable", "gq_kernel_timing_read", "gq_objective_noalloc", "gq_cd_cycles", "gq_cd_workspace_bytes",
@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.gq_saliency.argtypes = [vp, i64, i64, i64, i32, f32, vp, i64, vp]
         L.gq_saliency_prepared.restype = i32
         L.gq_saliency_prepared.argtypes = [vp, i64, i64, i64, i32, f32, vp, i64, vp, sz, vp]
+        L.gq_saliency_strided.restype = i32
+        L.gq_saliency_strided.argtypes = [vp, i32, i64, i64, i64, i64, i64, i32, f32, vp, i64, vp]
         L.gq_hessian_workspace_bytes.restype = sz
         L.gq_hessian_workspace_bytes.argtypes = [i64, i64, i32, u32]
         L.gq_hessian_accumulate.restype = i32
@@ -215,6 +217,36 @@ def gq_saliency_prepared(grad: torch.Tensor, g: int, hessian_workspace: torch.Te
                                         hessian_workspace.numel() * hessian_workspace.element_size(), st)
     if rc:
         raise GQError("gq_saliency_prepared", rc)
+    return s
+
+
+_DTYPE_CODES = {torch.bfloat16: 0, torch.float16: 1, torch.float32: 2}
+
+
+def gq_saliency_strided(grad: torch.Tensor, g: int, grad_scale: float = 1.0, s: Optional[torch.Tensor] = None,
+                        stream=None) -> torch.Tensor:
+    """Saliency of a ``[batch, seq, d_out]`` gradient in bf16, fp16 or fp32 with arbitrary batch / sequence strides
+    (a contiguous last dimension), e.g. the ``grad_output`` of a backward hook.  Writes ``s[k, b * seq + t]``;
+    pass a view ``s_all[:, offset:offset + batch * seq]`` to fill a slice of a calibration-wide buffer in place."""
+    if not grad.is_cuda or grad.dtype not in _DTYPE_CODES:
+        raise ValueError("grad must be a CUDA tensor of dtype bfloat16, float16 or float32")
+    if grad.dim() != 3 or (grad.shape[2] > 1 and grad.stride(2) != 1):
+        raise ValueError("grad must be [batch, seq, d_out] with a contiguous last dimension")
+    batch, seq, d_out = grad.shape
+    n = batch * seq
+    if s is None:
+        s = torch.empty((g, n), dtype=torch.float32, device=grad.device)
+    _dev(s, torch.float32, "s")
+    _, s_n, ld_s = _rows(s, "s")
+    if s.shape[0] != g or s_n < n:
+        raise ValueError("s must be [g, >= batch * seq]")
+    stride_b = grad.stride(0) if batch > 1 else max(grad.stride(0), seq * grad.stride(1))
+    stride_t = grad.stride(1) if seq > 1 else max(grad.stride(1), d_out)
+    with _on(_same_device(("grad", grad), ("s", s)), stream) as st:
+        rc = lib().gq_saliency_strided(grad.data_ptr(), _DTYPE_CODES[grad.dtype], batch, seq, d_out, stride_b, stride_t, g,
+                                       float(grad_scale), s.data_ptr(), ld_s, st)
+    if rc:
+        raise GQError("gq_saliency_strided", rc)
     return s
 
 

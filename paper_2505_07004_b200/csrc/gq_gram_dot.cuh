@@ -28,15 +28,15 @@
 // row, tensor memory dictates lane = row, so a warp's 32-byte load is 32 separate sector requests).  So the
 // requests are spread over the whole time the tile is being computed: as soon as an epilogue warp has finished a
 // tile it requests the four 32 x 32 blocks of its next tile into registers (128 KB per CTA: with that the eight
-// epilogue warps hold all of the CTA's share), and they have a full unit of MMAs (4 - 7 us) to arrive.  Warp 3
-// of each CTA additionally asks for those rows one unit earlier with cp.async.bulk.prefetch.L2 (one request per
-// row segment), so that the register loads are served from L2.  Once the accumulator is complete the contraction
-// itself takes well under a microsecond: tensor-memory columns of block j + 1 are requested before block j is
-// used, blocks above the diagonal take a branch without per-entry weights, and the accumulator is handed back as
-// soon as its last block sits in registers.
+// epilogue warps hold all of the CTA's share), and they have a full unit of MMAs (4 - 7 us) to arrive.  (An extra
+// warp that asked for the same rows earlier still with bulk L2 prefetches changed nothing measurable on any of
+// the layer shapes and was taken out again.)  Once the accumulator is complete the contraction itself takes well
+// under a microsecond: tensor-memory columns of block j + 1 are requested before block j is used, blocks above
+// the diagonal take a branch without per-entry weights, and the accumulator is handed back as soon as its last
+// block sits in registers.
 //
 // Roles: warp 0 (one lane) TMA producer, warp 1 (one lane, first CTA) MMA issuer, warp 2 TMEM allocation,
-// warp 3 L2 prefetch of H, warps 4..11 epilogue (registers: the service warpgroup gives up all but 40, the two
+// warp 3 idle, warps 4..11 epilogue (registers: the service warpgroup gives up all but 40, the two
 // epilogue warpgroups take 232).  Whole units only: one fp64 partial per (unit, CTA, warp), reduced in a fixed
 // order, so the result is reproducible.  Every mbarrier wait is bounded (gq_pipeline.cuh).
 #pragma once
@@ -85,11 +85,6 @@ struct GramDotParams {
 __host__ __device__ constexpr uint32_t umma_idesc_f16_mn(uint32_t m, uint32_t n)
 {
     return (1u << 4) | (1u << 15) | (1u << 16) | ((n >> 3) << 17) | ((m >> 4) << 24);
-}
-
-__device__ __forceinline__ void prefetch_l2_bulk(const void *p, uint32_t bytes)
-{
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
 
 // Eight consecutive floats (32 bytes, 32-byte aligned) that are read once: no L1 allocation.
@@ -364,41 +359,6 @@ gram_dot_kernel(const __grid_constant__ CUtensorMap mapD, const GramDotParams p)
                 umma_commit_local(smem_u32(&bar_drain));
                 const uint64_t t0 = global_timer_ns();
                 while (!mbar_try_wait(smem_u32(&bar_drain), 0u) && global_timer_ns() - t0 < 5000000ull) {}
-            }
-        } else if (warp == 3) {
-            // -------------------------------------------------------------- L2 prefetch of this CTA's rows of H
-            // One request per row of the tile: the part of the row segment on or above the diagonal, rounded down
-            // to whole 32-byte sectors.  Requests only move data into L2; nothing waits for them.  They are paced:
-            // the rows of unit `it` are requested when the MMAs of unit it - 2 have finished, i.e. about one unit
-            // of MMAs before the epilogue warps ask for them; running further ahead would push the operands and
-            // earlier requests out of L2 again.
-            uint32_t pf_ph[2] = {0u, 0u};
-            WorkItem w;
-            for (int it = 0; work_item(p.sched, pair, it, w); ++it) {
-                const int buf = it & 1;
-                if (it >= 2) {
-                    // a soft wait: prefetching is only a hint, so running out of patience here is not an error
-                    if (lane == 0) {
-                        const uint64_t t0 = global_timer_ns();
-                        while (!mbar_try_wait_suspend(smem_u32(&bar_acc_full[buf]), pf_ph[buf], 2000u) && !*wc.abort_flag &&
-                               global_timer_ns() - t0 < 200000ull) {}
-                    }
-                    __syncwarp();
-                    if (*wc.abort_flag) break;
-                    pf_ph[buf] ^= 1u;
-                }
-                const GramUnit u = gram_unit(p, w.unit);
-                const int row_base = u.ti * TILE_M + static_cast<int>(rank) * CTA_ROWS;
-                const int col0 = u.tj * TILE_N;
-                const int col1 = (col0 + TILE_N < p.d) ? col0 + TILE_N : p.d;
-                for (int r = lane; r < CTA_ROWS; r += 32) {
-                    const int row = row_base + r;
-                    if (row >= p.d) break;
-                    const int c = (row > col0) ? (row & ~7) : col0;
-                    if (c >= col1) continue;
-                    const float *src = p.H + (static_cast<size_t>(u.k) * p.d + row) * static_cast<size_t>(p.d) + c;
-                    prefetch_l2_bulk(src, static_cast<uint32_t>(col1 - c) * 4u);
-                }
             }
         }
     } else {

@@ -3,6 +3,7 @@
 // SM count.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -117,6 +118,64 @@ saliency_kernel(const __nv_bfloat16 *__restrict__ grad, unsigned n, int m, long 
             if ((k & 1) == 0 && k + 1 == g) w[1] = 0u;
         }
     }
+}
+
+// ------------------------------------------------------------------------------------------------
+// The saliency step for a gradient as a backward pass hands it over (Section 3.2: only the averaged squared
+// gradients of a layer are kept): dl/dZ as [batch][seq][d_out] with element strides (stride_b, stride_t, 1) in
+// bf16, IEEE half or fp32; token i = b * seq + t lands in s[k][i].  Same warp-per-segment scheme and the same
+// fp32 arithmetic as saliency_kernel (a 16-byte load holds 8 sixteen-bit or 4 fp32 values).
+enum { SAL_BF16 = 0, SAL_FP16 = 1, SAL_FP32 = 2 };
+
+template <int DTYPE>
+__device__ __forceinline__ float sum_sq_vec16(const uint4 &v, float acc)
+{
+    if (DTYPE == SAL_BF16) return sum_sq_bf16x8(v, acc);
+    if (DTYPE == SAL_FP16) {
+        const __half2 *h = reinterpret_cast<const __half2 *>(&v);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 t = __half22float2(h[e]);
+            acc = fmaf(t.x, t.x, acc);
+            acc = fmaf(t.y, t.y, acc);
+        }
+        return acc;
+    }
+    const float *f = reinterpret_cast<const float *>(&v);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) acc = fmaf(f[e], f[e], acc);
+    return acc;
+}
+
+template <int DTYPE>
+__global__ void __launch_bounds__(256)
+saliency_strided_kernel(const void *__restrict__ grad, unsigned n, unsigned seq, int m, long long stride_b, long long stride_t,
+                        int g, float coef, float *__restrict__ s, long long ld_s)
+{
+    constexpr int PER_VEC = (DTYPE == SAL_FP32) ? 4 : 8;          // values per 16-byte load
+    constexpr int ELEM = (DTYPE == SAL_FP32) ? 4 : 2;
+    const int lane = threadIdx.x & 31;
+    const unsigned seg = blockIdx.x * 8u + (threadIdx.x >> 5);
+    if (seg >= n * static_cast<unsigned>(g)) return;
+    const unsigned i = seg / static_cast<unsigned>(g);
+    const int k = static_cast<int>(seg - i * static_cast<unsigned>(g));
+    const unsigned b = i / seq, t = i - b * seq;
+    const int vecs = m / PER_VEC;
+    const long long first = static_cast<long long>(b) * stride_b + static_cast<long long>(t) * stride_t + static_cast<long long>(k) * m;
+    const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const char *>(grad) + first * ELEM);
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int v = lane; v < vecs; v += 128) {             // four loads in flight, predicated off past the end
+        uint4 x[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            x[u] = (v + 32 * u < vecs) ? ld_once_16(src + v + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) acc[u] = sum_sq_vec16<DTYPE>(x[u], acc[u]);
+    }
+    float sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+    if (lane == 0) s[static_cast<long long>(k) * ld_s + i] = sum * coef;
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -437,6 +437,48 @@ int32_t gq_saliency_prepared(const void *grad, int64_t n, int64_t d_out, int64_t
     return saliency_impl(grad, n, d_out, ld_grad, g, grad_scale, s, ld_s, true, hessian_workspace, workspace_bytes, stream);
 }
 
+int32_t gq_saliency_strided(const void *grad, int32_t dtype, int64_t batch, int64_t seq, int64_t d_out, int64_t stride_b,
+                            int64_t stride_t, int32_t g, float grad_scale, float *s, int64_t ld_s, void *stream)
+{
+    if (batch < 0 || seq < 0 || g < 1 || d_out < 1 || d_out % g != 0 || stride_t < d_out || stride_b < 0 ||
+        (dtype != GQ_DTYPE_BF16 && dtype != GQ_DTYPE_FP16 && dtype != GQ_DTYPE_FP32) ||
+        !(grad_scale == grad_scale) || grad_scale - grad_scale != 0.0f)
+        return GQ_ERR_INVALID_ARG;
+    if (batch > (1ll << 31) || seq > (1ll << 31)) return GQ_ERR_UNSUPPORTED_SHAPE;
+    const int64_t n = batch * seq;
+    if (ld_s < n) return GQ_ERR_INVALID_ARG;
+    if (batch > 1 && stride_b < (seq - 1) * stride_t + d_out) return GQ_ERR_INVALID_ARG;      // sequences overlap
+    if ((d_out / g) % 8 != 0 || g > 1024 || d_out > (1ll << 24) || n * g >= (1ll << 31)) return GQ_ERR_UNSUPPORTED_SHAPE;
+    const int64_t per16 = (dtype == GQ_DTYPE_FP32) ? 4 : 8;                    // elements per 16 bytes
+    if (stride_t % per16 != 0 || stride_b % per16 != 0) return GQ_ERR_ALIGNMENT;
+    if (n == 0) return GQ_OK;
+    if (!grad || !s) return GQ_ERR_INVALID_ARG;
+    if (!aligned(grad, 16) || !aligned(s, 4)) return GQ_ERR_ALIGNMENT;
+    const size_t elem = (dtype == GQ_DTYPE_FP32) ? 4 : 2;
+    const size_t g_bytes = (static_cast<size_t>(batch - 1) * stride_b + static_cast<size_t>(seq - 1) * stride_t + d_out) * elem;
+    if (overlaps(grad, g_bytes, s, span_bytes(g, n, ld_s, 4))) return GQ_ERR_INVALID_ARG;
+    DeviceInfo *di;
+    if (int32_t rc = device_info(&di)) return rc;
+    const int m = static_cast<int>(d_out / g);
+    const float coef = grad_scale * grad_scale / static_cast<float>(m);
+    const unsigned grid = static_cast<unsigned>((n * g + 7) / 8);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    {
+        LaunchScope scope(GQ_KERNEL_SALIENCY, st);
+        if (dtype == GQ_DTYPE_BF16)
+            gq::saliency_strided_kernel<gq::SAL_BF16><<<grid, 256, 0, st>>>(grad, static_cast<unsigned>(n), static_cast<unsigned>(seq), m,
+                                                                         stride_b, stride_t, g, coef, s, ld_s);
+        else if (dtype == GQ_DTYPE_FP16)
+            gq::saliency_strided_kernel<gq::SAL_FP16><<<grid, 256, 0, st>>>(grad, static_cast<unsigned>(n), static_cast<unsigned>(seq), m,
+                                                                         stride_b, stride_t, g, coef, s, ld_s);
+        else
+            gq::saliency_strided_kernel<gq::SAL_FP32><<<grid, 256, 0, st>>>(grad, static_cast<unsigned>(n), static_cast<unsigned>(seq), m,
+                                                                         stride_b, stride_t, g, coef, s, ld_s);
+    }
+    GQ_CUDA(cudaGetLastError());
+    return GQ_OK;
+}
+
 size_t gq_hessian_workspace_bytes(int64_t n_max, int64_t d_in, int32_t g, uint32_t flags)
 {
     if ((flags & ~static_cast<uint32_t>(GQ_HESSIAN_DETERMINISTIC | GQ_HESSIAN_S_PREPARED)) != 0 || n_max < 0 ||

@@ -58,22 +58,35 @@ def allocate_symmetric_hessian(g: int, d_in: int, device, group=None):
     return H, [int(p) for p in handle.buffer_ptrs]
 
 
-def exchange_hessian(H: torch.Tensor, rank_ptrs: Sequence, rank: int, group=None) -> torch.Tensor:
+def exchange_hessian(H: torch.Tensor, rank_ptrs: Sequence, rank: int, group=None, ops=None) -> torch.Tensor:
     """After every rank has accumulated its chunks into its H: make every rank's H the full sum and complete
-    it (finalize).  `rank_ptrs[r]` is rank r's H as addressable from this GPU (`rank_ptrs[rank]` is `H`)."""
-    from . import api
+    it (finalize).  `rank_ptrs[r]` is rank r's H as addressable from this GPU (`rank_ptrs[rank]` is `H`).
+    `ops` supplies gq_hessian_reduce_share / gq_hessian_gather_shares / gq_hessian_finalize (default: the
+    library binding); the sequence of calls and meeting points is what this function owns."""
+    if ops is None:
+        from . import api as ops
     g, d_in = int(H.shape[0]), int(H.shape[1])
 
     def meet():
-        torch.cuda.current_stream().synchronize()
+        if H.is_cuda:
+            torch.cuda.current_stream(H.device).synchronize()
         if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
             dist.barrier(group)
 
     if len(rank_ptrs) > 1:
         meet()                                            # all partial matrices are complete
-        api.gq_hessian_reduce_share(rank_ptrs, rank, d_in, g)
+        ops.gq_hessian_reduce_share(rank_ptrs, rank, d_in, g)
         meet()                                            # all shares are reduced
-        api.gq_hessian_gather_shares(rank_ptrs, rank, d_in, g)
+        ops.gq_hessian_gather_shares(rank_ptrs, rank, d_in, g)
         meet()                                            # nobody reads this rank's H any more
-    api.gq_hessian_finalize(H)
+    ops.gq_hessian_finalize(H)
     return H
+
+
+def exchange_bytes_per_rank(d_in: int, g: int, world: int, block: int = 128) -> int:
+    """Bytes one rank reads from its peers in the two steps of `exchange_hessian` together: in the reduce step its
+    own share of the 128 x 128 blocks of the upper triangle from the other world - 1 matrices, in the gather step
+    the other ranks' shares; each is (world - 1) / world of the blocks."""
+    nb = (int(d_in) + block - 1) // block
+    blocks = int(g) * nb * (nb + 1) // 2
+    return 2 * (blocks * (int(world) - 1) // int(world)) * block * block * 4

@@ -82,6 +82,13 @@ def test_host_side_validation_needs_no_gpu(L):
     assert L.gq_saliency(p16 + 2, 4, 64, 64, 2, 1.0, p16, 4, None) == ALIGN
     assert L.gq_saliency(None, 4, 64, 64, 2, 1.0, p16, 4, None) == INVALID
     assert L.gq_saliency(None, 0, 64, 64, 2, 1.0, None, 0, None) == 0          # empty call: no-op
+    # saliency from a [batch, seq, d_out] gradient in another dtype
+    assert L.gq_saliency_strided(p16, 3, 2, 4, 64, 256, 64, 2, 1.0, p16 + 4096, 8, None) == INVALID   # unknown dtype
+    assert L.gq_saliency_strided(p16, 1, 2, 4, 64, 256, 32, 2, 1.0, p16 + 4096, 8, None) == INVALID   # stride_t < d_out
+    assert L.gq_saliency_strided(p16, 1, 2, 4, 64, 128, 64, 2, 1.0, p16 + 4096, 8, None) == INVALID   # sequences overlap
+    assert L.gq_saliency_strided(p16, 2, 2, 4, 64, 264, 66, 2, 1.0, p16 + 4096, 8, None) == ALIGN     # 66 floats: not 16 bytes
+    assert L.gq_saliency_strided(p16, 1, 2, 4, 64, 256, 64, 2, 1.0, p16 + 4096, 7, None) == INVALID   # ld_s < batch * seq
+    assert L.gq_saliency_strided(None, 1, 0, 4, 64, 256, 64, 2, 1.0, None, 0, None) == 0              # empty call
     # hessian
     assert L.gq_hessian_accumulate(p16, 4, 64, 64, p16, 4, 2, p16, 4, p16, 4096, None) == INVALID   # flags
     assert L.gq_hessian_accumulate(p16, 4, 60, 64, p16, 4, 2, p16, 0, p16, 4096, None) == SHAPE     # d_in % 8

@@ -111,6 +111,42 @@ def test_saliency_empty_and_errors(dev):
     assert "GQ_ERR_INVALID_ARG" in str(e.value)
 
 
+@pytest.mark.parametrize("dtype,np_dtype,name", [(torch.bfloat16, np.uint16, "bf16"), (torch.float16, np.float16, "fp16"),
+                                                 (torch.float32, np.float32, "fp32")])
+@pytest.mark.parametrize("batch,seq,d_out,g,pad,bstep", [(3, 37, 512, 4, 0, 1), (2, 65, 688, 2, 40, 2), (1, 1, 8, 1, 0, 1),
+                                                          (4, 19, 11008, 16, 0, 1), (2, 8, 2560, 2, 8, 3)])
+def test_saliency_strided_parity(dev, dtype, np_dtype, name, batch, seq, d_out, g, pad, bstep):
+    """gq_saliency_strided on [batch, seq, d_out] views (padded rows, every bstep-th slab of a larger buffer) in the
+    three gradient dtypes, written into a slice of a wider s buffer, against the oracle on the same bits."""
+    gen = torch.Generator(device=dev).manual_seed(batch * 1000 + seq + d_out)
+    base = (torch.randn(batch * bstep, seq, d_out + pad, generator=gen, device=dev) * 3e-3)
+    base = (base * torch.exp(torch.randn(batch * bstep, seq, 1, generator=gen, device=dev))).to(dtype)
+    view = base[::bstep, :, :d_out]
+    n, off = batch * seq, 24
+    s_all = torch.full((g, n + 48), -1.0, device=dev)
+    libgq.gq_saliency_strided(view, g, 2.0, s=s_all[:, off:off + n])
+    libgq.gq_check()
+    host = base.cpu()
+    host_np = host.view(torch.int16).numpy().view(np.uint16) if dtype == torch.bfloat16 else host.numpy()
+    s_ref = orc.saliency_strided(host_np[::bstep, :, :d_out], name, g, 2.0)
+    check_s(s_all[:, off:off + n], s_ref)
+    assert torch.all(s_all[:, :off] == -1.0) and torch.all(s_all[:, off + n:] == -1.0)      # nothing else is touched
+    if dtype == torch.bfloat16 and pad == 0 and bstep == 1:
+        s_plain = libgq.gq_saliency(view.reshape(n, d_out), g, 2.0)
+        assert torch.equal(s_plain, s_all[:, off:off + n])                                  # same arithmetic, same bits
+
+
+def test_saliency_strided_errors(dev):
+    grad = torch.zeros((2, 4, 68), dtype=torch.float16, device=dev)
+    with pytest.raises(libgq.GQError) as e:
+        libgq.gq_saliency_strided(grad[:, :, :64], 2)            # row stride 68 is not a multiple of 16 bytes
+    assert "GQ_ERR_ALIGNMENT" in str(e.value)
+    with pytest.raises(ValueError):
+        libgq.gq_saliency_strided(torch.zeros((2, 4, 64), dtype=torch.float64, device=dev), 2)
+    s = libgq.gq_saliency_strided(torch.zeros((0, 4, 64), dtype=torch.float32, device=dev), 2)
+    assert tuple(s.shape) == (2, 0)
+
+
 # ------------------------------------------------------------------------------------------ Hessian
 @pytest.mark.parametrize("flags", [0, libgq.GQ_HESSIAN_DETERMINISTIC])
 @pytest.mark.parametrize("n,d_in,g,chunks", [

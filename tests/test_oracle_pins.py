@@ -277,6 +277,42 @@ def test_objective_edge_cases(impl):
     np.testing.assert_allclose(loss[1], np.linalg.norm(x @ W.astype(np.float64).T, "fro") ** 2, rtol=1e-12)
 
 
+# ------------------------------------------------------------- saliency from other dtypes and layouts
+@pytest.mark.parametrize("impl", IMPLS)
+def test_strided_typed_saliency(impl):
+    """saliency_strided: the hand example in every dtype, equality with saliency() on bf16 rows, brute force in
+    pure Python on a tiny strided fp16 / fp32 case (values widened exactly), a view with padded rows and a
+    batch stride, half-precision subnormals and the gradient scale."""
+    fx = read_fixture(os.path.join(GOLDEN, "hand_example.txt"))
+    for dtype, arr in (("bf16", orc.f64_to_bf16_bits(fx["grad"])), ("fp16", fx["grad"].astype(np.float16)),
+                       ("fp32", fx["grad"].astype(np.float32))):
+        s2 = orc.saliency_strided(arr.reshape(1, 2, 2), dtype, 2, impl=impl)
+        np.testing.assert_array_equal(s2, fx["g2_s"])
+        s1 = orc.saliency_strided(arr.reshape(2, 1, 2), dtype, 1, impl=impl)
+        np.testing.assert_array_equal(s1[0], fx["g1_s"])
+    rng = np.random.default_rng(31)
+    gb, _ = bf16_exact(rng, (24, 48), 1e-2)
+    np.testing.assert_array_equal(orc.saliency_strided(gb.reshape(4, 6, 48), "bf16", 3, 2.0, impl=impl),
+                                  orc.saliency(gb, 3, 2.0, impl="c"))
+    for dtype, np_t in (("fp16", np.float16), ("fp32", np.float32)):
+        wide = (rng.standard_normal((3, 5, 40)) * 1e-2).astype(np_t)          # [batch, seq, padded row]
+        wide[0, 0, :4] = np.array([6e-8, -6e-8, 3e-5, 0.0]).astype(np_t)       # half subnormals (exact in fp32 too)
+        view = wide[::2, :, :32]                          # rows padded from 32 to 40 elements, batch stride of two slabs
+        got = orc.saliency_strided(view, dtype, 4, 3.0, impl=impl)
+        assert got.shape == (4, 2 * 5)
+        for b in range(2):
+            for t in range(5):
+                for k in range(4):
+                    acc = 0.0
+                    for j in range(8 * k, 8 * k + 8):
+                        acc += (3.0 * float(view[b, t, j])) ** 2
+                    assert abs(got[k, b * 5 + t] - acc / 8.0) <= 1e-15 * max(acc, 1e-300) + 1e-300
+    with pytest.raises(ValueError):
+        orc.saliency_strided(np.zeros((2, 2, 9), np.float32), "fp32", 2)
+    with pytest.raises(ValueError):
+        orc.saliency_strided(np.zeros((2, 2, 8), np.float32), "fp16", 2)
+
+
 # ------------------------------------------------------------- C loops vs numpy
 def test_c_loops_match_numpy_definitions():
     rng = np.random.default_rng(11)

@@ -90,3 +90,73 @@ def test_chunks_for_rank_partitions():
         for world in (1, 2, 3, 8):
             got = sorted(c for r in range(world) for c in shard.chunks_for_rank(n_chunks, r, world))
             assert got == list(range(n_chunks))
+
+
+class _CpuExchangeOps:
+    """CPU stand-ins for the three library calls exchange_hessian makes.  The ranks are separate processes without
+    shared memory, so "reading a peer's matrix" is an all-gather here; shares are row ranges.  What is under test
+    is exchange_hessian's own sequence: reduce only after every partial matrix is complete, gather only after
+    every share is reduced, finalize last."""
+
+    def __init__(self, H, world):
+        self.H, self.world, self.log = H, world, []
+
+    def _all(self):
+        mats = [torch.empty_like(self.H) for _ in range(self.world)]
+        dist.all_gather(mats, self.H)
+        return mats
+
+    def _rows(self, r):
+        d = self.H.shape[1]
+        return slice(d * r // self.world, d * (r + 1) // self.world)
+
+    def gq_hessian_reduce_share(self, ptrs, rank, d_in, g):
+        self.log.append("reduce")
+        mats = self._all()
+        acc = torch.zeros_like(self.H[:, self._rows(rank)])
+        for m in mats:                                   # rank order: the same bits on whichever rank adds them
+            acc += m[:, self._rows(rank)]
+        self.H[:, self._rows(rank)] = acc
+
+    def gq_hessian_gather_shares(self, ptrs, rank, d_in, g):
+        self.log.append("gather")
+        mats = self._all()
+        for r in range(self.world):
+            if r != rank:
+                self.H[:, self._rows(r)] = mats[r][:, self._rows(r)]
+
+    def gq_hessian_finalize(self, H):
+        self.log.append("finalize")
+        up = torch.triu(H)
+        H.copy_(up + torch.triu(H, 1).transpose(1, 2))
+
+
+def _exchange_worker(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        gen = torch.Generator().manual_seed(100 + rank)
+        H = torch.triu(torch.randn(2, 12, 12, generator=gen, dtype=torch.float64))      # this rank's partial sums
+        partial = H.clone()
+        ops = _CpuExchangeOps(H, world)
+        shard.exchange_hessian(H, [None] * world, rank, ops=ops)
+        torch.save({"H": H, "partial": partial, "log": ops.log}, os.path.join(out_dir, "x%d.pt" % rank))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_exchange_hessian_sequence_with_cpu_stand_ins(tmp_path):
+    world, port = 2, _free_port()
+    mp.spawn(_exchange_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    r = [torch.load(os.path.join(tmp_path, "x%d.pt" % i)) for i in range(world)]
+    total = r[0]["partial"] + r[1]["partial"]
+    expect = total + torch.triu(total, 1).transpose(1, 2)
+    for i in range(world):
+        assert r[i]["log"] == ["reduce", "gather", "finalize"]
+        assert torch.equal(r[i]["H"], expect)                       # every rank ends with the same full matrix
+    # one rank: no exchange, only finalize
+    H = torch.triu(torch.randn(1, 6, 6, dtype=torch.float64))
+    ops = _CpuExchangeOps(H, 1)
+    shard.exchange_hessian(H, [None], 0, ops=ops)
+    assert ops.log == ["finalize"] and torch.equal(H, H.transpose(1, 2))
+    assert shard.exchange_bytes_per_rank(4096, 4, 8) == 2 * (4 * 32 * 33 // 2 * 7 // 8) * 128 * 128 * 4
