@@ -427,12 +427,12 @@ def run_ours(args, cfg, g):
         ms_per_launch = ga_ms / max(1, ga_n)
         achieved = flops_per_launch / (ms_per_launch * 1e-3) / 1e12 if ga_n else None
         issued = issued_per_launch / (ms_per_launch * 1e-3) / 1e12 if ga_n else None
-        # Which measured tensor peak applies: the burst figure when the timed region is short or the clock
-        # stayed near its maximum (the kernel ran as in a burst), the sustained one when the run sat at the
-        # power cap with the clock pulled down.  Both fractions are printed either way.
+        # Which measured tensor peak applies: the burst figure when the sampled SM clock stayed near its maximum (the
+        # kernel ran as in a burst), the sustained one when the run sat at the power cap with the clock pulled
+        # down.  Both fractions are printed either way.
         sm, sm_max = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
         near_max = bool(sm and sm_max and sm >= 0.9 * sm_max)
-        burst = near_max or ms_total < 1000.0
+        burst = near_max if (sm and sm_max) else ms_total < 1000.0          # no clock samples: go by the duration
         peak = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
         kernel_ms = sum(v[0] for v in kern.values())
         kernels = {k: {"launches": v[1], "ms_total": round(v[0], 4), "share": round(v[0] / kernel_ms, 4) if kernel_ms else None}
@@ -446,8 +446,8 @@ def run_ours(args, cfg, g):
             "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
             "peak_source": ("bf16_tflops (burst), " if burst else "bf16_tflops_sustained, ") + peaks["source"],
             "peak_regime": ("burst: %s" % ("median SM clock %.0f of %.0f MHz" % (sm, sm_max) if near_max
-                                           else "timed region of %.2f s" % (ms_total * 1e-3))) if burst
-                           else "sustained: timed region of %.1f s at a median SM clock of %s of %s MHz" % (ms_total * 1e-3, sm, sm_max),
+                                           else "no clock samples, timed region of %.2f s" % (ms_total * 1e-3))) if burst
+                           else "sustained: timed region of %.2f s at a median SM clock of %s of %s MHz" % (ms_total * 1e-3, sm, sm_max),
             "frac_of_burst_peak": frac(achieved, peaks["bf16_tflops"]),
             "frac_of_sustained_peak": frac(achieved, peaks["bf16_tflops_sustained"]),
             "frac_of_nominal_peak": frac(achieved, NOMINAL_BF16_TFLOPS),
