@@ -409,6 +409,55 @@ def test_full_shapes_sampled(dev, name, g, n_tokens, _unused):
     torch.cuda.empty_cache()
 
 
+# ------------------------------------------------------------------------------------------ extreme sizes
+def test_largest_feature_count(dev):
+    """d_in = 65536, the largest the interface accepts (H is 17 GB, 32896 tiles): index arithmetic beyond 2^31
+    elements.  The oracle is run on sampled features (which are the same entries of the full H), on the diagonal of
+    all features, and the objective on a weight error confined to the sampled features."""
+    d_in, n, g, d_out = 65536, 96, 1, 16
+    gen = torch.Generator(device=dev).manual_seed(65536)
+    X = (torch.randn(n, d_in, generator=gen, device=dev) * torch.exp(0.5 * torch.randn(d_in, generator=gen, device=dev)))
+    X = X.to(torch.bfloat16)
+    s = torch.rand(g, n, generator=gen, device=dev) + 0.1
+    H = gpu_hessian([X], [s], d_in, g, dev)
+    rng = np.random.default_rng(1)
+    F = np.unique(np.concatenate([rng.choice(d_in, 60, replace=False), [0, 255, 256, 32767, 32768, 65280, 65535]]))
+    Ft = torch.from_numpy(F).to(dev)
+    s64 = s.cpu().numpy().astype(np.float64)
+    H_ref = orc.hessian(synth.bf16_bits(X[:, Ft].contiguous()), s64)
+    check_H(H[:, Ft][:, :, Ft], H_ref)
+    diag = orc.hessian_diag(synth.bf16_bits(X), s64)
+    d_gpu = torch.diagonal(H[0]).double().cpu().numpy()
+    assert np.all(np.abs(d_gpu - diag[0]) <= H_ENTRY * diag[0] + 1e-30)
+    corner = H[0, 65000:, 65000:].cpu()
+    assert torch.equal(corner, corner.T)
+    W = 0.02 * torch.randn(d_out, d_in, generator=gen, device=dev)
+    What = W.clone()
+    What[:, Ft] += 0.01 * torch.randn(d_out, len(F), generator=gen, device=dev)
+    ows = libgq.alloc_workspace(libgq.gq_objective_workspace_bytes(d_in, d_out, g), dev)
+    loss = libgq.gq_objective(W, What, H, ows)
+    libgq.gq_check()
+    loss_ref = orc.objective(W[:, Ft].contiguous().cpu().numpy(), What[:, Ft].contiguous().cpu().numpy(),
+                             H[:, Ft][:, :, Ft].double().cpu().numpy())
+    check_loss(loss, loss_ref)
+    del H, X, W, What, ows
+    torch.cuda.empty_cache()
+
+
+def test_largest_group_count(dev):
+    """g = 1024 groups of 8 channels, the most the interface accepts: 512 pairs of groups per tile."""
+    n, d_in, g = 300, 264, 1024
+    cfg = synth.LayerConfig("g1024", n, 128, d_in, 8 * g, (g,), "lognormal", 0.01, 20.0)
+    xs, gs, ss, H, W, What, loss = run_layer(cfg, dev)
+    xb = np.concatenate([synth.bf16_bits(x) for x in xs])
+    gb = np.concatenate([synth.bf16_bits(x) for x in gs])
+    s_ref = orc.saliency(gb, g)
+    check_s(torch.cat(ss, dim=1), s_ref)
+    H_ref = orc.hessian(xb, s_ref)
+    check_H(H, H_ref)
+    check_loss(loss, orc.objective(W.cpu().numpy(), What.cpu().numpy(), H_ref))
+
+
 # ------------------------------------------------------------------------------------------ failure detection
 def test_device_wait_timeout_is_reported_and_context_survives(dev):
     """A pipeline wait that runs out of its time budget makes the kernel return (no trap, no hang), the status
