@@ -11,8 +11,11 @@ two passes over the same calibration batches in the same order:
         for batch in batches: model(batch)
     H = cap.finalize()                   # {name: [g, d_in, d_in] fp32}, complete symmetric matrices
 
-No arithmetic of the method happens here: the hooks flatten tokens, cast to bf16 (the library's input type)
-and call gq_saliency / gq_hessian_accumulate / gq_hessian_finalize on the tensors' own device and stream."""
+No arithmetic of the method happens here.  The backward hook hands the gradient over as autograd produced it
+(``[batch, seq, d_out]`` in bf16, fp16 or fp32, any batch / sequence strides) to gq_saliency_strided, so no cast
+and no contiguous copy of it is ever made; other layouts are flattened and cast to bf16 for gq_saliency.  The
+forward hook flattens the layer input to bf16 tokens (the Hessian kernel's input type) and calls
+gq_hessian_accumulate; finalize() calls gq_hessian_finalize.  All on the tensors' own device and stream."""
 from __future__ import annotations
 
 import contextlib
@@ -43,8 +46,12 @@ class GuidedHessianCapture:
         handles = []
         for name, mod in self.layers.items():
             def hook(_mod, _grad_in, grad_out, name=name):
-                grad = self._tokens(grad_out[0].detach())
-                self.s[name].append(api.gq_saliency(grad, self.g, self.grad_scale))
+                grad = grad_out[0].detach()
+                if (grad.dim() == 3 and grad.dtype in (torch.bfloat16, torch.float16, torch.float32)
+                        and (grad.shape[2] == 1 or grad.stride(2) == 1)):
+                    self.s[name].append(api.gq_saliency_strided(grad, self.g, self.grad_scale))
+                else:
+                    self.s[name].append(api.gq_saliency(self._tokens(grad), self.g, self.grad_scale))
             handles.append(mod.register_full_backward_hook(hook))
         try:
             yield self

@@ -1,6 +1,7 @@
 """The two-pass capture (backward hooks -> saliency, forward hooks -> guided Hessians) on a small random
-PyTorch model against the oracle, which gets the same bf16 bit patterns of the gradients and inputs that the
-hooks see (recorded by independent hooks of the test)."""
+PyTorch model against the oracle, which gets the fp32 gradients and the bf16 bit patterns of the inputs that
+the hooks see (recorded by independent hooks of the test).  The gradients reach the library in autograd's own
+dtype and layout (gq_saliency_strided), so the oracle reads the same fp32 values."""
 import numpy as np
 import pytest
 import torch
@@ -12,14 +13,15 @@ from paper_2505_07004_b200.capture import GuidedHessianCapture
 pytestmark = pytest.mark.gpu
 
 
-def test_capture_matches_oracle():
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["fp32", "bf16"])
+def test_capture_matches_oracle(dtype):
     assert torch.cuda.is_available()
     dev = torch.device("cuda:0")
     torch.manual_seed(0)
-    model = torch.nn.Sequential(torch.nn.Linear(64, 128), torch.nn.GELU(), torch.nn.Linear(128, 64)).to(dev)
+    model = torch.nn.Sequential(torch.nn.Linear(64, 128), torch.nn.GELU(), torch.nn.Linear(128, 64)).to(dev).to(dtype)
     layers = {"fc1": model[0], "fc2": model[2]}
     g, scale = 4, 1e3
-    batches = [torch.randn(3, 50, 64, device=dev), torch.randn(2, 37, 64, device=dev)]
+    batches = [torch.randn(3, 50, 64, device=dev).to(dtype), torch.randn(2, 37, 64, device=dev).to(dtype)]
     target = [torch.randint(0, 64, (3, 50), device=dev), torch.randint(0, 64, (2, 37), device=dev)]
 
     seen_x = {k: [] for k in layers}
@@ -29,13 +31,13 @@ def test_capture_matches_oracle():
         spies.append(mod.register_forward_pre_hook(
             lambda m, inp, name=name: seen_x[name].append(inp[0].detach().reshape(-1, inp[0].shape[-1]).to(torch.bfloat16))))
         spies.append(mod.register_full_backward_hook(
-            lambda m, gi, go, name=name: seen_g[name].append(go[0].detach().reshape(-1, go[0].shape[-1]).to(torch.bfloat16))))
+            lambda m, gi, go, name=name: seen_g[name].append(go[0].detach().clone())))
 
     cap = GuidedHessianCapture(layers, g, grad_scale=scale)
     with cap.saliency_pass():
         for x, t in zip(batches, target):
             out = model(x)
-            torch.nn.functional.cross_entropy(out.reshape(-1, 64), t.reshape(-1), reduction="sum").backward()
+            torch.nn.functional.cross_entropy(out.reshape(-1, 64).float(), t.reshape(-1), reduction="sum").backward()
     for k in seen_x:
         seen_x[k].clear()
     with cap.hessian_pass():
@@ -47,9 +49,13 @@ def test_capture_matches_oracle():
         h.remove()
 
     for name in layers:
-        gb = np.concatenate([synth.bf16_bits(t.cpu()) for t in seen_g[name]])
         xb = np.concatenate([synth.bf16_bits(t.cpu()) for t in seen_x[name]])
-        s_o = orc.saliency(gb, g, scale)
+        assert all(t.dim() == 3 and t.dtype == dtype for t in seen_g[name])
+        if dtype == torch.float32:
+            s_o = np.concatenate([orc.saliency_strided(t.cpu().numpy(), "fp32", g, scale) for t in seen_g[name]], axis=1)
+        else:
+            s_o = np.concatenate([orc.saliency_strided(synth.bf16_bits(t.cpu()).reshape(tuple(t.shape)), "bf16", g, scale)
+                                  for t in seen_g[name]], axis=1)
         s_g = torch.cat(cap.s[name], dim=1).cpu().numpy().astype(np.float64)
         assert np.all(np.abs(s_g - s_o) <= 1e-4 * np.abs(s_o) + 1e-30)
         H_o = orc.hessian(xb, s_o)
