@@ -3,9 +3,10 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
-One "step" is one pass of the whole path over one synthetic layer: for every token chunk
-gq_saliency_prepared + gq_hessian_accumulate (two launches), then gq_hessian_finalize and gq_objective (H is
-zeroed at the start of the step).  The default workload is the Llama-2-7B attention-projection shape
+One "step" is one pass of the whole path over one synthetic layer: gq_saliency_prepared for the first token
+chunk, then one gq_hessian_accumulate_ahead per chunk (the Hessian step of that chunk and, on the warps it leaves
+idle, the saliency step of the next one), then gq_hessian_finalize and gq_objective (H is zeroed at the start of
+the step).  `--two-launch-chunks` runs gq_saliency_prepared + gq_hessian_accumulate per chunk instead.  The default workload is the Llama-2-7B attention-projection shape
 (131072 tokens in 16 chunks of 8192, d_in = d_out = 4096, g = 4).  All inputs are seeded and
 synthetic and stay resident in HBM for the device-timed number; the `e2e` number goes through
 gq_layer_objective_host with pinned host buffers (host->device copies inside the timed region).
@@ -42,7 +43,8 @@ KERNEL_TIMING_EVERY = 8      # steps between two steps whose launches are timed 
 NOMINAL_BF16_TFLOPS = 2250.0     # B200 dense bf16 / fp16 tensor peak (vendor figure), for context beside the measured peaks
 # DRAM bytes (read + write) per launch of the dominant kernel, from an ncu capture of one launch of that
 # workload; None where no capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {"c1_7b_attn": 343.36e6}
+# Keyed by (workload, chunk loop): a launch of the look-ahead loop also reads the next chunk's gradients.
+NCU_TRAFFIC_BYTES = {("c1_7b_attn", "ahead"): 415.59e6, ("c1_7b_attn", "two_launch"): 347.50e6}
 # The oracle sample both the cpu_baseline leg and --impl reference time (one size, so that the oracle's
 # throughput is one number): tokens of chunk 0 for saliency + Hessian, channels per group for the objective.
 ORACLE_SAMPLE_TOKENS, ORACLE_SAMPLE_CHANNELS = 1024, 64
@@ -288,11 +290,13 @@ def run_ours(args, cfg, g):
     W, What = syn.weights()
     H = torch.empty((g, cfg.d_in, cfg.d_in), dtype=torch.float32, device=dev)
     s_buf = torch.empty((g, cfg.chunk), dtype=torch.float32, device=dev)
+    s_alt = torch.empty((g, cfg.chunk), dtype=torch.float32, device=dev)
     ws = libgq.alloc_workspace(libgq.gq_hessian_workspace_bytes(cfg.chunk, cfg.d_in, g), dev)
+    ws_alt = libgq.alloc_workspace(libgq.gq_hessian_workspace_bytes(cfg.chunk, cfg.d_in, g), dev)
     ows = libgq.alloc_workspace(libgq.gq_objective_workspace_bytes(cfg.d_in, cfg.d_out, g), dev)
     loss = torch.empty(g + 1, dtype=torch.float64, device=dev)
 
-    def step():
+    def step_two_launch_chunks():
         H.zero_()
         for c in range(n_chunks):
             nt = xs[c].shape[0]
@@ -300,6 +304,23 @@ def run_ours(args, cfg, g):
             libgq.gq_hessian_accumulate(xs[c], s_buf[:, :nt], H, ws, flags=libgq.GQ_HESSIAN_S_PREPARED)
         libgq.gq_hessian_finalize(H)
         libgq.gq_objective(W, What, H, ows, loss=loss)
+
+    def step_ahead():
+        # two saliency buffers / scratch blocks in turn: chunk c reads one pair while chunk c + 1's is written
+        sb, wb = (s_buf, s_alt), (ws, ws_alt)
+        H.zero_()
+        libgq.gq_saliency_prepared(gs[0], g, wb[0], 1.0, s=sb[0][:, :gs[0].shape[0]])
+        for c in range(n_chunks):
+            nt = xs[c].shape[0]
+            if c + 1 < n_chunks:
+                libgq.gq_hessian_accumulate_ahead(xs[c], sb[c & 1][:, :nt], H, wb[c & 1], gs[c + 1], wb[(c + 1) & 1], 1.0,
+                                                  sb[(c + 1) & 1][:, :gs[c + 1].shape[0]], flags=libgq.GQ_HESSIAN_S_PREPARED)
+            else:
+                libgq.gq_hessian_accumulate(xs[c], sb[c & 1][:, :nt], H, wb[c & 1], flags=libgq.GQ_HESSIAN_S_PREPARED)
+        libgq.gq_hessian_finalize(H)
+        libgq.gq_objective(W, What, H, ows, loss=loss)
+
+    step = step_two_launch_chunks if args.two_launch_chunks else step_ahead
 
     def barrier():
         if world > 1:
@@ -339,6 +360,22 @@ def run_ours(args, cfg, g):
     loss_host = loss.cpu().numpy()
     if not np.all(np.isfinite(loss_host)) or loss_host[g] <= 0:
         raise RuntimeError("objective is not finite/positive: %s" % loss_host)
+
+    # ---- the Hessian kernel without the look-ahead work: two passes of the two-launch chunk loop right after the
+    # timed region (same clocks, same cache state), an event pair around every launch
+    plain_hessian = None
+    if not args.two_launch_chunks:
+        step_two_launch_chunks()
+        libgq.gq_kernel_timing_read()
+        libgq.gq_kernel_timing_enable(True)
+        for _ in range(2):
+            step_two_launch_chunks()
+        libgq.gq_kernel_timing_enable(False)
+        torch.cuda.synchronize()
+        k2 = libgq.gq_kernel_timing_read()
+        if k2["hessian"][1]:
+            plain_hessian = k2["hessian"][0] / k2["hessian"][1]
+        libgq.gq_check()
 
     # ---- saliency alone: all chunks' launches captured into one CUDA graph (no host time between launches, no
     # per-launch event pair), replayed SAL_B2B_PASSES times inside one event pair
@@ -441,9 +478,11 @@ def run_ours(args, cfg, g):
         sal_bytes = cfg.chunk * (2 * cfg.d_out + 4 * g)
         frac = lambda a, p: (a / p) if (a is not None and p) else None
         roofline = {
-            "kernel": "hessian_kernel (gq_hessian_accumulate)", "bound": "tensor",
+            "kernel": "hessian_kernel (gq_hessian_accumulate)" if args.two_launch_chunks else
+                      "hessian_kernel (gq_hessian_accumulate_ahead: the launch also computes the next chunk's saliency; "
+                      "only the Hessian flops are counted)", "bound": "tensor",
             "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": frac(achieved, peak),
-            "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
+            "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, "two_launch" if args.two_launch_chunks else "ahead")),
             "peak_source": ("bf16_tflops (burst), " if burst else "bf16_tflops_sustained, ") + peaks["source"],
             "peak_regime": ("burst: %s" % ("median SM clock %.0f of %.0f MHz" % (sm, sm_max) if near_max
                                            else "no clock samples, timed region of %.2f s" % (ms_total * 1e-3))) if burst
@@ -458,9 +497,20 @@ def run_ours(args, cfg, g):
             "issued_frac_of_nominal_peak": frac(issued, NOMINAL_BF16_TFLOPS),
             "target": "60 %% of the nominal peak: %s" % ("met" if (achieved or 0) >= 0.6 * NOMINAL_BF16_TFLOPS else "not met"),
         }
+        if plain_hessian:
+            tf = flops_per_launch / (plain_hessian * 1e-3) / 1e12
+            roofline["without_look_ahead"] = {
+                "ms_per_launch": plain_hessian, "achieved": tf, "frac_of_burst_peak": frac(tf, peaks["bf16_tflops"]),
+                "frac_of_sustained_peak": frac(tf, peaks["bf16_tflops_sustained"]), "frac_of_nominal_peak": frac(tf, NOMINAL_BF16_TFLOPS),
+                "timing": "event pairs around the gq_hessian_accumulate launches of two passes of the two-launch chunk loop, "
+                          "run directly after the timed region (the launches of the timed region also compute the next "
+                          "chunk's saliency)"}
         sal_gbs = (sal_bytes / (sal_ms / max(1, sal_n) * 1e-3) / 1e9) if sal_n else None
         saliency_roofline = {
-            "kernel": "saliency_kernel (gq_saliency_prepared)", "bound": "hbm", "unit": "GB/s", "peak": peaks["hbm_gbs"],
+            "kernel": "saliency_kernel (gq_saliency_prepared) as a launch of its own" +
+                      ("" if args.two_launch_chunks else "; in the step only the first chunk's saliency is such a launch, "
+                       "the others run inside the Hessian launches"),
+            "bound": "hbm", "unit": "GB/s", "peak": peaks["hbm_gbs"],
             "bytes_per_launch": sal_bytes,
             "achieved": sal_b2b_gbs, "frac": frac(sal_b2b_gbs, peaks["hbm_gbs"]),
             "timing": "one event pair around %d replays of a CUDA graph holding the launches of all %d chunks "
@@ -507,6 +557,8 @@ def run_ours(args, cfg, g):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "api": "gq_layer_objective_host (pinned host buffers)"},
             "gpu_launches": int(launches),
+            "chunk_loop": ("gq_saliency_prepared + gq_hessian_accumulate per chunk" if args.two_launch_chunks else
+                           "gq_hessian_accumulate_ahead: the saliency step of chunk c + 1 runs inside the Hessian launch of chunk c"),
             "clocks": clocks,
             "loss_total": float(loss_host[g]),
         }
@@ -546,6 +598,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-token-sharded", action="store_true", help="N > 1: skip the token-sharded layer with the peer-memory exchange")
+    ap.add_argument("--two-launch-chunks", action="store_true",
+                    help="per chunk gq_saliency_prepared + gq_hessian_accumulate instead of gq_hessian_accumulate_ahead")
     ap.add_argument("--tokens", type=int, default=0, help="use only the first TOKENS tokens (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

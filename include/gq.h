@@ -140,6 +140,36 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
                               int64_t ld_s, int32_t g, float *H, uint32_t flags, void *workspace,
                               size_t workspace_bytes, void *stream);
 
+/*
+ * gq_hessian_accumulate for this chunk and, in the same launch, gq_saliency_prepared for the NEXT chunk
+ * (Algorithm 1: the saliency step of a chunk uses nothing that the Hessian step of another chunk writes, so the
+ * two are independent).  The Hessian kernel is bound by the tensor cores and leaves two warps per CTA without
+ * work; those warps stream the next chunk's gradients meanwhile, so the saliency step costs no time of its own
+ * as long as it ends before the Hessian step does (the launch lasts as long as the longer of the two).
+ *
+ *   X, n, d_in, ld_x, s, ld_s, g, H, flags, workspace, workspace_bytes
+ *               exactly as for gq_hessian_accumulate (this chunk)
+ *   next_grad, next_n, d_out, ld_grad, grad_scale, next_s, next_ld_s, next_workspace, next_workspace_bytes
+ *               exactly as grad, n, d_out, ld_grad, grad_scale, s, ld_s, hessian_workspace, workspace_bytes of
+ *               gq_saliency_prepared (the next chunk; same g).  next_workspace is a second scratch block:
+ *               neither it nor next_s may share memory with X, s, H or workspace, and next_grad must not share
+ *               memory with H or workspace.  (s and next_s may be two disjoint column ranges of one [g, ld]
+ *               buffer that holds the saliency of all chunks: with equal leading dimensions the check is exact.)  The next call passes next_workspace as its workspace together
+ *               with GQ_HESSIAN_S_PREPARED.
+ * next_s and next_workspace receive the same bits as a gq_saliency_prepared call would write.
+ * The spare warps stream about 1 TB/s.  Where the next chunk's gradients would take longer than this chunk's
+ * Hessian work (few groups and d_out large against d_in: roughly 3000 * d_out * next_n > g * d_in^2 * n) the
+ * call runs the saliency step as a kernel of its own before the Hessian kernel instead; results are the same.
+ * next_n == 0: the call is gq_hessian_accumulate.  n == 0: the call is gq_saliency_prepared for the next chunk
+ * (after the arguments of this chunk have been checked).
+ * The caller runs the saliency step of the very first chunk with gq_saliency_prepared.
+ */
+int32_t gq_hessian_accumulate_ahead(const void *X, int64_t n, int64_t d_in, int64_t ld_x, const float *s,
+                                    int64_t ld_s, int32_t g, float *H, uint32_t flags, void *workspace,
+                                    size_t workspace_bytes, const void *next_grad, int64_t next_n, int64_t d_out,
+                                    int64_t ld_grad, float grad_scale, float *next_s, int64_t next_ld_s,
+                                    void *next_workspace, size_t next_workspace_bytes, void *stream);
+
 /* Scratch bytes gq_hessian_accumulate needs for chunks of up to n_max tokens (0 on bad arguments). */
 size_t gq_hessian_workspace_bytes(int64_t n_max, int64_t d_in, int32_t g, uint32_t flags);
 

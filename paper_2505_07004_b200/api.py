@@ -20,6 +20,7 @@ _lib = None
 
 EXPORTS = (
     "gq_version", "gq_status_string", "gq_last_cuda_error", "gq_saliency", "gq_saliency_prepared", "gq_saliency_strided", "gq_hessian_accumulate",
+    "gq_hessian_accumulate_ahead",
     "gq_hessian_workspace_bytes", "gq_hessian_finalize", "gq_objective", "gq_objective_workspace_bytes",
     "gq_layer_objective_host", "gq_layer_host_arena_bytes", "gq_check", "gq_launch_count",
     "gq_kernel_timing_enable", "gq_kernel_timing_read", "gq_objective_noalloc", "gq_cd_cycles", "gq_cd_workspace_bytes",
@@ -68,6 +69,9 @@ def lib() -> ctypes.CDLL:
         L.gq_hessian_workspace_bytes.argtypes = [i64, i64, i32, u32]
         L.gq_hessian_accumulate.restype = i32
         L.gq_hessian_accumulate.argtypes = [vp, i64, i64, i64, vp, i64, i32, vp, u32, vp, sz, vp]
+        L.gq_hessian_accumulate_ahead.restype = i32
+        L.gq_hessian_accumulate_ahead.argtypes = [vp, i64, i64, i64, vp, i64, i32, vp, u32, vp, sz,
+                                                  vp, i64, i64, i64, f32, vp, i64, vp, sz, vp]
         L.gq_hessian_finalize.restype = i32
         L.gq_hessian_finalize.argtypes = [vp, i64, i32, vp]
         for f in (L.gq_hessian_reduce_share, L.gq_hessian_gather_shares):
@@ -273,6 +277,40 @@ def gq_hessian_accumulate(X: torch.Tensor, s: torch.Tensor, H: torch.Tensor, wor
     if rc:
         raise GQError("gq_hessian_accumulate", rc)
     return H
+
+
+def gq_hessian_accumulate_ahead(X: torch.Tensor, s: torch.Tensor, H: torch.Tensor, workspace: torch.Tensor,
+                                next_grad: torch.Tensor, next_workspace: torch.Tensor, grad_scale: float = 1.0,
+                                next_s: Optional[torch.Tensor] = None, flags: int = 0, stream=None) -> torch.Tensor:
+    """:func:`gq_hessian_accumulate` for this chunk and, in the same launch, :func:`gq_saliency_prepared` for the
+    next one (``next_grad`` -> ``next_s`` and ``next_workspace``).  Returns ``next_s``."""
+    _dev(X, torch.bfloat16, "X")
+    _dev(s, torch.float32, "s")
+    _dev(H, torch.float32, "H")
+    _dev(next_grad, torch.bfloat16, "next_grad")
+    n, d_in, ld_x = _rows(X, "X")
+    g, s_n, ld_s = _rows(s, "s")
+    if s_n < n:
+        raise ValueError("s must be [g, >= n]")
+    if tuple(H.shape) != (g, d_in, d_in) or not H.is_contiguous():
+        raise ValueError("H must be a contiguous [g, d_in, d_in] tensor")
+    next_n, d_out, ld_grad = _rows(next_grad, "next_grad")
+    if next_s is None:
+        next_s = torch.empty((g, next_n), dtype=torch.float32, device=next_grad.device)
+    _dev(next_s, torch.float32, "next_s")
+    _, ns_n, next_ld_s = _rows(next_s, "next_s")
+    if next_s.shape[0] != g or ns_n < next_n:
+        raise ValueError("next_s must be [g, >= next_n]")
+    with _on(_same_device(("X", X), ("s", s), ("H", H), ("workspace", workspace), ("next_grad", next_grad),
+                          ("next_s", next_s), ("next_workspace", next_workspace)), stream) as st:
+        rc = lib().gq_hessian_accumulate_ahead(
+            X.data_ptr(), n, d_in, ld_x, s.data_ptr(), ld_s, g, H.data_ptr(), flags, workspace.data_ptr(),
+            workspace.numel() * workspace.element_size(), next_grad.data_ptr(), next_n, d_out, ld_grad, float(grad_scale),
+            next_s.data_ptr(), next_ld_s, next_workspace.data_ptr(),
+            next_workspace.numel() * next_workspace.element_size(), st)
+    if rc:
+        raise GQError("gq_hessian_accumulate_ahead", rc)
+    return next_s
 
 
 def gq_hessian_finalize(H: torch.Tensor, stream=None) -> torch.Tensor:

@@ -24,8 +24,10 @@
 // Per CTA and k-step (1024 tensor-core clocks for two groups) this moves 32 KB from L2 (half of what a
 // per-group pass over pre-scaled operands needs) and 112 KB through shared memory.
 //
-// Warps: 0 TMA producer (one lane) | 1 MMA issuer (one lane, first CTA) | 2 TMEM allocation | 3 idle |
-//        4..15 scalers | 16..23 epilogue.
+// Warps: 0 TMA producer (one lane) | 1 MMA issuer (one lane, first CTA) | 2 TMEM allocation | 3 - |
+//        4..15 scalers | 16..23 epilogue.  Warps 2 and 3 have nothing to do in the Hessian step; on request
+//        (SaliencyAhead) they compute the saliency of the next token chunk meanwhile: 296 warps that stream the
+//        next gradient block at a small fraction of the memory bandwidth, hidden behind the tensor-core work.
 // Work units are (tile, pair of groups), plus (row block, pair of column tiles) for an odd last group; they are dealt to the CTA pairs as described in gq_pipeline.cuh
 // (round-robin rounds, then the incomplete last round cut along the token axis).  Because H is updated
 // by reduce-adds only, pieces of a cut unit need no special treatment.
@@ -58,6 +60,20 @@ constexpr int HS_STAGING_BYTES = HS_EPI_WARPS * 4096;          // one 32 x 32 fp
 constexpr int HS_THREADS = 32 * (4 + HS_SCALER_WARPS + HS_EPI_WARPS);
 constexpr int HS_SMEM_BYTES = HS_STAGES * HS_STAGE_BYTES + HS_STAGING_BYTES + 1024;
 
+// The saliency step of the NEXT token chunk, computed by the two warps per CTA that the Hessian step leaves idle
+// (Algorithm 1: the saliency of a chunk depends on nothing the Hessian step of the previous chunk writes).
+// grad == nullptr: nothing to do.
+struct SaliencyAhead {
+    const __nv_bfloat16 *grad;   // [n][ld_grad]
+    unsigned n;                  // tokens of the next chunk
+    int m;                       // d_out / g
+    long long ld_grad;
+    float coef;                  // grad_scale^2 / m
+    float *s;                    // [g][ld_s]
+    long long ld_s;
+    uint32_t *words;             // the next call's packed saliency: [ceil(g / 2)][n] pairs of words
+};
+
 struct HessianParams {
     const __nv_bfloat16 *X;  // [n][ld_x]
     long long ld_x;
@@ -72,6 +88,7 @@ struct HessianParams {
     Schedule sched;          // units = narrow_units + (g odd ? column-pair slots : 0), ksteps = ceil(n / 64)
     uint32_t *status;
     unsigned long long wait_budget_ns;
+    SaliencyAhead ahead;
 };
 
 // What a work unit computes.  A unit always fills (up to) two 256-column accumulators from one pass over
@@ -466,6 +483,68 @@ hessian_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__
             acc_ph ^= 1u;
         }
         if (lane == 0) bulk_wait_group_read0();       // shared memory must outlive the last reduce-add's read
+    } else if ((warp == 2 || warp == 3) && p.ahead.grad != nullptr) {
+        // ------------------------------------------------------------------ saliency of the next chunk
+        // Same lane-to-element assignment and the same order of additions as saliency_kernel, so the values are
+        // the same bits.  Segment = (token, group); the 2 * gridDim.x warps take segments round-robin, so at any
+        // time they read one contiguous window of the gradient block.  Short segments (at most four loads per
+        // lane) are taken two at a time, eight loads in flight per lane.
+        const SaliencyAhead &a = p.ahead;
+        const unsigned g_u = static_cast<unsigned>(p.g);
+        const unsigned total = a.n * g_u;
+        const unsigned stride = gridDim.x * 2u;
+        const int vecs = a.m >> 3;
+        unsigned seg = blockIdx.x * 2u + static_cast<unsigned>(warp - 2);
+        auto segment_src = [&](unsigned sg, unsigned &i, int &k) {
+            i = sg / g_u;
+            k = static_cast<int>(sg - i * g_u);
+            return reinterpret_cast<const uint4 *>(a.grad + static_cast<long long>(i) * a.ld_grad + static_cast<long long>(k) * a.m);
+        };
+        if (vecs <= 128) {
+            for (; seg < total; seg += 2u * stride) {
+                const bool two = seg + stride < total;
+                unsigned i0, i1 = 0u;
+                int k0, k1 = 0;
+                const uint4 *src0 = segment_src(seg, i0, k0);
+                const uint4 *src1 = two ? segment_src(seg + stride, i1, k1) : src0;
+                uint4 x[8];
+#pragma unroll
+                for (int t = 0; t < 4; ++t)
+                    x[t] = (lane + 32 * t < vecs) ? ld_once_16(src0 + lane + 32 * t) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                for (int t = 0; t < 4; ++t)
+                    x[4 + t] = (two && lane + 32 * t < vecs) ? ld_once_16(src1 + lane + 32 * t) : make_uint4(0u, 0u, 0u, 0u);
+                float acc[8];
+#pragma unroll
+                for (int t = 0; t < 8; ++t) acc[t] = sum_sq_bf16x8(x[t], 0.f);
+                const float sum0 = warp_sum_butterfly((acc[0] + acc[1]) + (acc[2] + acc[3]));
+                const float sum1 = warp_sum_butterfly((acc[4] + acc[5]) + (acc[6] + acc[7]));
+                if (lane == 0) {
+                    saliency_store(sum0 * a.coef, i0, k0, a.n, p.g, a.s, a.ld_s, a.words);
+                    if (two) saliency_store(sum1 * a.coef, i1, k1, a.n, p.g, a.s, a.ld_s, a.words);
+                }
+            }
+        } else {
+            // Long segments: eight loads in flight per lane from the first to the last (saliency_kernel takes
+            // the ends of a segment four at a time; element lane + 32 t of every group of eight goes to partial
+            // sum t & 3 in ascending order either way, so the sums are the same bits).
+            for (; seg < total; seg += stride) {
+                unsigned i;
+                int k;
+                const uint4 *src = segment_src(seg, i, k);
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int v = lane; v < vecs; v += 256) {
+                    uint4 x[8];
+#pragma unroll
+                    for (int t = 0; t < 8; ++t)
+                        x[t] = (v + 32 * t < vecs) ? ld_once_16(src + v + 32 * t) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) acc[t & 3] = sum_sq_bf16x8(x[t], acc[t & 3]);
+                }
+                const float sum = warp_sum_butterfly((acc[0] + acc[1]) + (acc[2] + acc[3]));
+                if (lane == 0) saliency_store(sum * a.coef, i, k, a.n, p.g, a.s, a.ld_s, a.words);
+            }
+        }
     }
 
     __syncwarp();

@@ -70,17 +70,9 @@ __device__ __forceinline__ float sum_sq_bf16x8(const uint4 &v, float acc)
 // If `words` is not null the value is also stored in the packed form of split_scale, laid out as the
 // guided-Hessian kernel reads it: [ceil(g / 2)][n] pairs of words, pair q of token i = groups 2q and 2q + 1
 // (the second word of an odd last group is 0).
-__global__ void __launch_bounds__(256)
-saliency_kernel(const __nv_bfloat16 *__restrict__ grad, unsigned n, int m, long long ld_grad, int g, float coef,
-                float *__restrict__ s, long long ld_s, uint32_t *__restrict__ words)
+// A lane's share of sum_j grad[j]^2 over one segment of `vecs` 16-byte vectors (before the butterfly).
+__device__ __forceinline__ float saliency_lane_sum(const uint4 *__restrict__ src, int vecs, int lane)
 {
-    const int lane = threadIdx.x & 31;
-    const unsigned seg = blockIdx.x * 8u + (threadIdx.x >> 5);
-    if (seg >= n * static_cast<unsigned>(g)) return;
-    const unsigned i = seg / static_cast<unsigned>(g);
-    const int k = static_cast<int>(seg - i * static_cast<unsigned>(g));
-    const int vecs = m >> 3;                             // 16-byte vectors per segment
-    const uint4 *src = reinterpret_cast<const uint4 *>(grad + static_cast<long long>(i) * ld_grad + static_cast<long long>(k) * m);
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     {
         uint4 x[4];
@@ -106,18 +98,40 @@ saliency_kernel(const __nv_bfloat16 *__restrict__ grad, unsigned n, int m, long 
 #pragma unroll
         for (int t = 0; t < 4; ++t) acc[t] = sum_sq_bf16x8(x[t], acc[t]);
     }
-    float sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    return (acc[0] + acc[1]) + (acc[2] + acc[3]);
+}
+
+__device__ __forceinline__ float warp_sum_butterfly(float sum)
+{
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-    if (lane == 0) {
-        const float val = sum * coef;
-        s[static_cast<long long>(k) * ld_s + i] = val;
-        if (words) {
-            uint32_t *w = words + (static_cast<long long>(k >> 1) * n + i) * 2;
-            w[k & 1] = split_scale(val);
-            if ((k & 1) == 0 && k + 1 == g) w[1] = 0u;
-        }
+    return sum;
+}
+
+// Stores s[k][i] and, if `words` is not null, its packed two-term form (one lane calls this).
+__device__ __forceinline__ void saliency_store(float val, unsigned i, int k, unsigned n, int g, float *__restrict__ s,
+                                               long long ld_s, uint32_t *__restrict__ words)
+{
+    s[static_cast<long long>(k) * ld_s + i] = val;
+    if (words) {
+        uint32_t *w = words + (static_cast<long long>(k >> 1) * n + i) * 2;
+        w[k & 1] = split_scale(val);
+        if ((k & 1) == 0 && k + 1 == g) w[1] = 0u;
     }
+}
+
+__global__ void __launch_bounds__(256)
+saliency_kernel(const __nv_bfloat16 *__restrict__ grad, unsigned n, int m, long long ld_grad, int g, float coef,
+                float *__restrict__ s, long long ld_s, uint32_t *__restrict__ words)
+{
+    const int lane = threadIdx.x & 31;
+    const unsigned seg = blockIdx.x * 8u + (threadIdx.x >> 5);
+    if (seg >= n * static_cast<unsigned>(g)) return;
+    const unsigned i = seg / static_cast<unsigned>(g);
+    const int k = static_cast<int>(seg - i * static_cast<unsigned>(g));
+    const uint4 *src = reinterpret_cast<const uint4 *>(grad + static_cast<long long>(i) * ld_grad + static_cast<long long>(k) * m);
+    const float sum = warp_sum_butterfly(saliency_lane_sum(src, m >> 3, lane));
+    if (lane == 0) saliency_store(sum * coef, i, k, n, g, s, ld_s, words);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -100,6 +100,25 @@ inline size_t span_bytes(int64_t rows, int64_t width, int64_t ld, size_t elem)
     if (rows <= 0 || width <= 0) return 0;
     return (static_cast<size_t>(rows - 1) * static_cast<size_t>(ld) + static_cast<size_t>(width)) * elem;
 }
+// True if two row sets of fp32 elements share an element: `rows` rows of width na at a (leading dimension ld_a)
+// and of width nb at b (leading dimension ld_b).  Exact when the leading dimensions are equal (two column
+// ranges of one [rows, ld] buffer interleave without touching); otherwise decided by the spans.
+inline bool rows_overlap_f32(const float *a, int64_t na, int64_t ld_a, const float *b, int64_t nb, int64_t ld_b, int64_t rows)
+{
+    if (!overlaps(a, span_bytes(rows, na, ld_a, 4), b, span_bytes(rows, nb, ld_b, 4))) return false;
+    const intptr_t diff = reinterpret_cast<intptr_t>(b) - reinterpret_cast<intptr_t>(a);
+    if (ld_a != ld_b || diff % 4 != 0) return true;
+    const int64_t D = diff / 4, ld = ld_a;
+    int64_t r = D % ld, q = D / ld;
+    if (r < 0) {
+        r += ld;
+        q -= 1;
+    }
+    // element (k, i) of a and (k', j) of b coincide iff (k - k') ld = D + j - i, i.e. r + j - i is 0 or ld
+    const bool same_row = r < na && q > -rows && q < rows;                 // r + j - i = 0, k - k' = q
+    const bool next_row = r + nb > ld && q + 1 > -rows && q + 1 < rows;    // r + j - i = ld, k - k' = q + 1
+    return same_row || next_row;
+}
 
 int32_t device_info(DeviceInfo **out)
 {
@@ -389,16 +408,22 @@ int32_t gq_last_cuda_error(void) { return tl_last_cuda_error; }
 
 uint64_t gq_launch_count(void) { return g_launches.load(); }
 
-static int32_t saliency_impl(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad, int32_t g, float grad_scale,
-                             float *s, int64_t ld_s, bool prepare, void *hessian_workspace, size_t workspace_bytes,
-                             void *stream)
+// Argument checks of the saliency step (gq_saliency, gq_saliency_prepared and the saliency half of
+// gq_hessian_accumulate_ahead).  GQ_OK with *empty = true means: nothing to do, pointers were not looked at.
+static int32_t check_saliency_args(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad, int32_t g, float grad_scale,
+                                   const float *s, int64_t ld_s, bool prepare, const void *hessian_workspace,
+                                   size_t workspace_bytes, bool *empty)
 {
+    *empty = false;
     if (n < 0 || g < 1 || d_out < 1 || d_out % g != 0 || ld_grad < d_out || ld_s < n ||
         !(grad_scale == grad_scale) || grad_scale - grad_scale != 0.0f)
         return GQ_ERR_INVALID_ARG;
     if ((d_out / g) % 8 != 0 || g > 1024 || d_out > (1ll << 24) || n * g >= (1ll << 31)) return GQ_ERR_UNSUPPORTED_SHAPE;
     if (ld_grad % 8 != 0) return GQ_ERR_ALIGNMENT;
-    if (n == 0) return GQ_OK;              // nothing to read or write: pointers are not looked at
+    if (n == 0) {                          // nothing to read or write: pointers are not looked at
+        *empty = true;
+        return GQ_OK;
+    }
     if (!grad || !s) return GQ_ERR_INVALID_ARG;
     if (!aligned(grad, 16) || !aligned(s, 4)) return GQ_ERR_ALIGNMENT;
     const size_t g_bytes = span_bytes(n, d_out, ld_grad, 2), s_bytes = span_bytes(g, n, ld_s, 4);
@@ -410,6 +435,18 @@ static int32_t saliency_impl(const void *grad, int64_t n, int64_t d_out, int64_t
         if (overlaps(hessian_workspace, ws_bytes, grad, g_bytes) || overlaps(hessian_workspace, ws_bytes, s, s_bytes))
             return GQ_ERR_INVALID_ARG;
     }
+    return GQ_OK;
+}
+
+static int32_t saliency_impl(const void *grad, int64_t n, int64_t d_out, int64_t ld_grad, int32_t g, float grad_scale,
+                             float *s, int64_t ld_s, bool prepare, void *hessian_workspace, size_t workspace_bytes,
+                             void *stream)
+{
+    bool empty;
+    if (int32_t rc = check_saliency_args(grad, n, d_out, ld_grad, g, grad_scale, s, ld_s, prepare, hessian_workspace,
+                                         workspace_bytes, &empty))
+        return rc;
+    if (empty) return GQ_OK;
     DeviceInfo *di;
     if (int32_t rc = device_info(&di)) return rc;
     const int m = static_cast<int>(d_out / g);
@@ -487,9 +524,9 @@ size_t gq_hessian_workspace_bytes(int64_t n_max, int64_t d_in, int32_t g, uint32
     return hessian_ws_bytes(n_max, d_in, g);
 }
 
-int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld_x, const float *s, int64_t ld_s,
-                              int32_t g, float *H, uint32_t flags, void *workspace, size_t workspace_bytes,
-                              void *stream)
+static int32_t hessian_accumulate_impl(const void *X, int64_t n, int64_t d_in, int64_t ld_x, const float *s, int64_t ld_s,
+                                       int32_t g, float *H, uint32_t flags, void *workspace, size_t workspace_bytes,
+                                       const gq::SaliencyAhead *ahead, void *stream)
 {
     if (n < 0 || ld_x < d_in || ld_s < n ||
         (flags & ~static_cast<uint32_t>(GQ_HESSIAN_DETERMINISTIC | GQ_HESSIAN_S_PREPARED)) != 0)
@@ -544,6 +581,7 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
     p.sched = gq::plan_schedule(units, ksteps, pairs, balanced);
     p.status = di->status_ptr;
     p.wait_budget_ns = wait_budget_ns();
+    if (ahead) p.ahead = *ahead;
     const int grid = 2 * ((p.sched.full_waves == 0 && p.sched.tail_pairs > 0) ? p.sched.tail_pairs : pairs);
     {
         LaunchScope scope(GQ_KERNEL_HESSIAN, st);
@@ -551,6 +589,81 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
     }
     GQ_CUDA(cudaGetLastError());
     return GQ_OK;
+}
+
+int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld_x, const float *s, int64_t ld_s,
+                              int32_t g, float *H, uint32_t flags, void *workspace, size_t workspace_bytes,
+                              void *stream)
+{
+    return hessian_accumulate_impl(X, n, d_in, ld_x, s, ld_s, g, H, flags, workspace, workspace_bytes, nullptr, stream);
+}
+
+int32_t gq_hessian_accumulate_ahead(const void *X, int64_t n, int64_t d_in, int64_t ld_x, const float *s, int64_t ld_s,
+                                    int32_t g, float *H, uint32_t flags, void *workspace, size_t workspace_bytes,
+                                    const void *next_grad, int64_t next_n, int64_t d_out, int64_t ld_grad, float grad_scale,
+                                    float *next_s, int64_t next_ld_s, void *next_workspace, size_t next_workspace_bytes,
+                                    void *stream)
+{
+    bool empty;
+    if (int32_t rc = check_saliency_args(next_grad, next_n, d_out, ld_grad, g, grad_scale, next_s, next_ld_s, true,
+                                         next_workspace, next_workspace_bytes, &empty))
+        return rc;
+    if (empty)
+        return hessian_accumulate_impl(X, n, d_in, ld_x, s, ld_s, g, H, flags, workspace, workspace_bytes, nullptr, stream);
+    if (n <= 0) {
+        // no Hessian work to hide behind: check the rest of the call as gq_hessian_accumulate would, then run the
+        // saliency step as a launch of its own
+        if (int32_t rc = hessian_accumulate_impl(X, n, d_in, ld_x, s, ld_s, g, H, flags, workspace, workspace_bytes, nullptr, stream))
+            return rc;
+        return saliency_impl(next_grad, next_n, d_out, ld_grad, g, grad_scale, next_s, next_ld_s, true, next_workspace,
+                             next_workspace_bytes, stream);
+    }
+    if (!X || !s || !H || !workspace || d_in < 1 || ld_x < d_in || ld_s < n) return GQ_ERR_INVALID_ARG;
+    {
+        // what the look-ahead writes must not share memory with anything the Hessian step reads or writes, and
+        // what it reads must not be written by the Hessian step
+        const size_t h_bytes = static_cast<size_t>(g) * d_in * d_in * 4, ws_bytes = hessian_ws_bytes(n, d_in, g);
+        const size_t x_bytes = span_bytes(n, d_in, ld_x, 2), s_bytes = span_bytes(g, n, ld_s, 4);
+        const size_t ng_bytes = span_bytes(next_n, d_out, ld_grad, 2), ns_bytes = span_bytes(g, next_n, next_ld_s, 4);
+        const size_t nws_bytes = hessian_ws_bytes(next_n, 8, g);
+        const void *outs[2] = {next_s, next_workspace};
+        const size_t out_bytes[2] = {ns_bytes, nws_bytes};
+        for (int o = 0; o < 2; ++o)
+            if (overlaps(outs[o], out_bytes[o], H, h_bytes) || overlaps(outs[o], out_bytes[o], X, x_bytes) ||
+                overlaps(outs[o], out_bytes[o], workspace, ws_bytes))
+                return GQ_ERR_INVALID_ARG;
+        // s and next_s may be two column ranges of one [g, ld] buffer that holds the saliency of all chunks
+        if (rows_overlap_f32(s, n, ld_s, next_s, next_n, next_ld_s, g) || overlaps(next_workspace, nws_bytes, s, s_bytes))
+            return GQ_ERR_INVALID_ARG;
+        if (overlaps(next_grad, ng_bytes, H, h_bytes) || overlaps(next_grad, ng_bytes, workspace, ws_bytes))
+            return GQ_ERR_INVALID_ARG;
+    }
+    {
+        // Does the saliency step fit behind the Hessian step?  Measured on B200: the two spare warps per CTA stream
+        // the gradient block at about 1.0e12 bytes/s while the tensor cores work through 1.25e15 issued flop/s.
+        // If the gradients would take longer than 85 % of the Hessian work (plus 5 us, about what a launch of its
+        // own costs), the launch would only get longer: run the saliency step as a kernel of its own instead.
+        const double nj = static_cast<double>((d_in + gq::TILE_N - 1) / gq::TILE_N);
+        const double tok = static_cast<double>((n + gq::TILE_K - 1) / gq::TILE_K * gq::TILE_K);
+        const double t_hessian = 2.0 * gq::TILE_M * gq::TILE_N * tok * (nj * (nj + 1.0) / 2.0) * g / 1.25e15;
+        const double t_saliency = static_cast<double>(next_n) * static_cast<double>(d_out) * 2.0 / 1.0e12;
+        if (t_saliency > 0.85 * t_hessian + 5e-6) {
+            if (int32_t rc = saliency_impl(next_grad, next_n, d_out, ld_grad, g, grad_scale, next_s, next_ld_s, true,
+                                           next_workspace, next_workspace_bytes, stream))
+                return rc;
+            return hessian_accumulate_impl(X, n, d_in, ld_x, s, ld_s, g, H, flags, workspace, workspace_bytes, nullptr, stream);
+        }
+    }
+    gq::SaliencyAhead a{};
+    a.grad = static_cast<const __nv_bfloat16 *>(next_grad);
+    a.n = static_cast<unsigned>(next_n);
+    a.m = static_cast<int>(d_out / g);
+    a.ld_grad = ld_grad;
+    a.coef = grad_scale * grad_scale / static_cast<float>(a.m);
+    a.s = next_s;
+    a.ld_s = next_ld_s;
+    a.words = static_cast<uint32_t *>(next_workspace);
+    return hessian_accumulate_impl(X, n, d_in, ld_x, s, ld_s, g, H, flags, workspace, workspace_bytes, &a, stream);
 }
 
 int32_t gq_hessian_finalize(float *H, int64_t d_in, int32_t g, void *stream)

@@ -118,6 +118,24 @@ def test_aliasing_between_outputs_and_inputs_is_rejected(L):
     assert L.gq_hessian_accumulate(X, 4, 64, 64, H + 64, 4, 2, H, 0, ws, 1024, None) == INVALID      # s inside H
     assert L.gq_hessian_accumulate(X, 4, 64, 64, s_, 4, 2, H, 0, H + 1024, 1024, None) == INVALID    # workspace inside H
     assert L.gq_hessian_accumulate(X, 4, 64, 64, s_, 4, 2, H, 0, X, 1024, None) == INVALID           # workspace over X
+    # hessian with the next chunk's saliency: next grad [4, 64] = 512 B, next s 32 B, second workspace 1 KiB
+    ng, ns, nws = base + 131072, base + 132096, base + 133120
+    ahead = lambda ng_, ns_, nws_, nws_bytes=1024: L.gq_hessian_accumulate_ahead(
+        X, 4, 64, 64, s_, 4, 2, H, 0, ws, 1024, ng_, 4, 64, 64, 1.0, ns_, 4, nws_, nws_bytes, None)
+    assert ahead(ng, ns, ws) == INVALID                       # the second scratch block is the first one
+    assert ahead(ng, s_, nws) == INVALID                      # next s over the s being read
+    assert ahead(ng, H + 128, nws) == INVALID                 # next s inside H
+    assert ahead(ng, ns, X) == INVALID                        # second scratch block over X
+    assert ahead(H, ns, nws) == INVALID                       # next grad inside H (written by the same launch)
+    assert ahead(ng, ng + 16, nws) == INVALID                 # next s inside next grad
+    assert ahead(ng, ns, nws, 16) == WS
+    # s and next_s as column ranges of one [2, 16] buffer (leading dimension 16): disjoint columns are fine
+    # although their spans interleave, shared columns are not
+    in_one = lambda col: L.gq_hessian_accumulate_ahead(X, 4, 64, 64, s_, 16, 2, H, 0, ws, 1024, ng, 4, 64, 64, 1.0,
+                                                       s_ + 4 * col, 16, nws, 1024, None)
+    assert in_one(4) not in (INVALID, WS, -2, -3) and in_one(12) not in (INVALID, WS, -2, -3)
+    assert in_one(3) == INVALID and in_one(0) == INVALID and in_one(13) == INVALID      # 13..16 wraps into the next row
+    assert ahead(ng, ns, nws) not in (INVALID, WS, -2, -3)    # a valid call gets as far as the device (none here)
     # objective: W, W_hat [64, 64] fp32 = 16 KiB each, H [2, 64, 64] = 32 KiB, loss 24 B
     need = L.gq_objective_workspace_bytes(64, 64, 2)
     W, Wh, Hh, loss, ows = base, base + 16384, base + 32768, base + 65536, base + 131072

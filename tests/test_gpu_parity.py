@@ -225,6 +225,110 @@ def test_prepared_saliency_gives_the_same_hessian(dev, n, d_in, d_out, g):
     assert "GQ_ERR_WORKSPACE" in str(e.value)
 
 
+@pytest.mark.parametrize("chunks,d_in,d_out,g", [
+    ([300, 257, 64, 1], 520, 512, 4),      # ragged chunks, short segments (two per round of the look-ahead warps)
+    ([200, 333], 264, 120, 3),             # odd g: the last group's second word is written as 0
+    ([96, 160, 31], 256, 4096, 1),         # segments of 512 vectors: two rounds of the long-segment loop
+    ([130, 70], 128, 2080, 2),             # 130 vectors per segment: just over the short-segment limit
+])
+def test_accumulate_ahead_matches_oracle_and_two_launch_path(dev, chunks, d_in, d_out, g):
+    """The chunk loop with the saliency of chunk c + 1 computed inside the Hessian launch of chunk c
+    (gq_hessian_accumulate_ahead): s of every chunk against the oracle and bit-equal to gq_saliency_prepared, H
+    against the oracle and (single-writer schedule) bit-equal to the two-launch loop."""
+    gen = torch.Generator(device=dev).manual_seed(sum(chunks) + d_in + g)
+    X = [torch.randn(n, d_in, generator=gen, device=dev).to(torch.bfloat16) for n in chunks]
+    G = [(torch.randn(n, d_out, generator=gen, device=dev) * torch.exp(torch.randn(n, 1, generator=gen, device=dev))
+          ).to(torch.bfloat16) for n in chunks]
+    flags = libgq.GQ_HESSIAN_DETERMINISTIC | libgq.GQ_HESSIAN_S_PREPARED
+    nb = libgq.gq_hessian_workspace_bytes(max(chunks), d_in, g, flags)
+    ws = [libgq.alloc_workspace(nb, dev) for _ in range(2)]
+    for w in ws:
+        w.fill_(0xFF)
+    n_all = sum(chunks)
+    s_all = torch.full((g, n_all + 3), -1.0, dtype=torch.float32, device=dev)      # one buffer for all chunks, padded
+    offs = np.concatenate([[0], np.cumsum(chunks)])
+    view = lambda c: s_all[:, offs[c]:offs[c + 1]]
+    H = torch.zeros((g, d_in, d_in), dtype=torch.float32, device=dev)
+    launches = libgq.gq_launch_count()
+    libgq.gq_saliency_prepared(G[0], g, ws[0], 1.0, view(0))
+    for c in range(len(chunks)):
+        if c + 1 < len(chunks):
+            libgq.gq_hessian_accumulate_ahead(X[c], view(c), H, ws[c & 1], G[c + 1], ws[(c + 1) & 1], 1.0, view(c + 1), flags)
+        else:
+            libgq.gq_hessian_accumulate(X[c], view(c), H, ws[c & 1], flags)
+    assert libgq.gq_launch_count() - launches == len(chunks) + 1      # small enough to be hidden: one launch per chunk
+    libgq.gq_check()
+    assert torch.all(s_all[:, n_all:] == -1.0)
+    # two launches per chunk, same flags
+    H2 = torch.zeros_like(H)
+    ws2 = libgq.alloc_workspace(nb, dev)
+    for c in range(len(chunks)):
+        s2 = libgq.gq_saliency_prepared(G[c], g, ws2)
+        assert torch.equal(s2, view(c))
+        used = (g + 1) // 2 * chunks[c] * 8
+        assert torch.equal(ws2[:used], ws[c & 1][:used]) or c + 2 < len(chunks)      # a later chunk reused the block
+        libgq.gq_hessian_accumulate(X[c], s2, H2, ws2, flags)
+    libgq.gq_check()
+    assert torch.equal(H, H2)
+    s_o = np.concatenate([orc.saliency(synth.bf16_bits(gr), g) for gr in G], axis=1)
+    check_s(s_all[:, :n_all], s_o)
+    H_o = orc.hessian(np.concatenate([synth.bf16_bits(x) for x in X]), s_o)
+    check_H(H, H_o, upper_only=True)
+
+
+def test_accumulate_ahead_runs_saliency_separately_when_it_cannot_hide(dev):
+    """Few groups and many output channels: the next chunk's gradients would take longer to stream than this chunk's
+    Hessian work, so the call launches the saliency kernel on its own.  Same results."""
+    g, d_in, d_out, n = 1, 64, 32768, 512
+    gen = torch.Generator(device=dev).manual_seed(5)
+    X = torch.randn(n, d_in, generator=gen, device=dev).to(torch.bfloat16)
+    G = torch.randn(n, d_out, generator=gen, device=dev).to(torch.bfloat16)
+    nb = libgq.gq_hessian_workspace_bytes(n, d_in, g)
+    ws, ws_next = libgq.alloc_workspace(nb, dev), libgq.alloc_workspace(nb, dev)
+    s = libgq.gq_saliency_prepared(G, g, ws)
+    H = torch.zeros((g, d_in, d_in), dtype=torch.float32, device=dev)
+    launches = libgq.gq_launch_count()
+    s_next = libgq.gq_hessian_accumulate_ahead(X, s, H, ws, G, ws_next,
+                                               flags=libgq.GQ_HESSIAN_S_PREPARED | libgq.GQ_HESSIAN_DETERMINISTIC)
+    assert libgq.gq_launch_count() - launches == 2
+    libgq.gq_check()
+    assert torch.equal(s_next, s) and torch.equal(ws_next[:n * 8], ws[:n * 8])
+    check_s(s_next, orc.saliency(synth.bf16_bits(G), g))
+    check_H(H, orc.hessian(synth.bf16_bits(X), s_next.cpu().numpy().astype(np.float64)), upper_only=True)
+
+
+def test_accumulate_ahead_degenerate_and_errors(dev):
+    g, d_in, d_out, n = 2, 64, 32, 48
+    X = torch.randn(n, d_in, device=dev).to(torch.bfloat16)
+    G = torch.randn(n, d_out, device=dev).to(torch.bfloat16)
+    nb = libgq.gq_hessian_workspace_bytes(n, d_in, g)
+    ws, ws_next = libgq.alloc_workspace(nb, dev), libgq.alloc_workspace(nb, dev)
+    s = libgq.gq_saliency_prepared(G, g, ws)
+    H = torch.zeros((g, d_in, d_in), dtype=torch.float32, device=dev)
+    # no next chunk: plain accumulate
+    libgq.gq_hessian_accumulate_ahead(X, s, H, ws, G[:0], ws_next, flags=libgq.GQ_HESSIAN_S_PREPARED)
+    H1 = torch.zeros_like(H)
+    libgq.gq_hessian_accumulate(X, s, H1, ws, libgq.GQ_HESSIAN_S_PREPARED)
+    assert torch.equal(torch.triu(H), torch.triu(H1))
+    # no current chunk: the saliency step alone, H untouched
+    s_next = libgq.gq_hessian_accumulate_ahead(X[:0], s[:, :0], H, ws, G, ws_next)
+    assert torch.equal(s_next, s) and torch.equal(torch.triu(H), torch.triu(H1))
+    used = g // 2 * n * 8
+    assert torch.equal(ws_next[:used], ws[:used])
+    # the second scratch block must be a different one; next_s must not be the s being read
+    for bad in (lambda: libgq.gq_hessian_accumulate_ahead(X, s, H, ws, G, ws, flags=libgq.GQ_HESSIAN_S_PREPARED),
+                lambda: libgq.gq_hessian_accumulate_ahead(X, s, H, ws, G, ws_next, next_s=s),
+                lambda: libgq.gq_hessian_accumulate_ahead(X, s, H, ws, G, ws_next, next_s=H.view(-1)[:g * n].view(g, n))):
+        with pytest.raises(libgq.GQError) as e:
+            bad()
+        assert "GQ_ERR_INVALID_ARG" in str(e.value)
+    with pytest.raises(libgq.GQError) as e:
+        libgq.gq_hessian_accumulate_ahead(X, s, H, ws, G, ws_next[:8])
+    assert "GQ_ERR_WORKSPACE" in str(e.value)
+    libgq.gq_check()
+    assert torch.equal(torch.triu(H), torch.triu(H1))    # nothing was written by the rejected calls
+
+
 def test_hessian_errors(dev):
     X = torch.zeros((16, 64), dtype=torch.bfloat16, device=dev)
     s = torch.zeros((2, 16), dtype=torch.float32, device=dev)

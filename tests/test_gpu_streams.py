@@ -76,3 +76,45 @@ def test_side_stream_and_graph_replay_match_the_default_stream(dev):
     torch.cuda.synchronize()
     libgq.gq_check()
     assert torch.equal(b2[0], ref[0]) and torch.equal(b2[4], ref[4])
+
+
+def run_path_ahead(cfg, xs, gs, W, What, bufs, extra):
+    """The same path with one launch per chunk: the saliency of chunk c + 1 is computed inside the Hessian launch
+    of chunk c (two saliency buffers and scratch blocks in turn)."""
+    H, s_buf, ws, ows, loss = bufs
+    sb, wb = (s_buf, extra[0]), (ws, extra[1])
+    g = cfg.g
+    flags = libgq.GQ_HESSIAN_DETERMINISTIC | libgq.GQ_HESSIAN_S_PREPARED
+    H.zero_()
+    libgq.gq_saliency_prepared(gs[0], g, wb[0], 1.0, s=sb[0][:, :gs[0].shape[0]])
+    for c, x in enumerate(xs):
+        nt = x.shape[0]
+        if c + 1 < len(xs):
+            libgq.gq_hessian_accumulate_ahead(x, sb[c & 1][:, :nt], H, wb[c & 1], gs[c + 1], wb[(c + 1) & 1], 1.0,
+                                              sb[(c + 1) & 1][:, :gs[c + 1].shape[0]], flags=flags)
+        else:
+            libgq.gq_hessian_accumulate(x, sb[c & 1][:, :nt], H, wb[c & 1], flags=flags)
+    libgq.gq_hessian_finalize(H)
+    libgq.gq_objective(W, What, H, ows, loss=loss)
+
+
+def test_one_launch_per_chunk_in_a_graph_gives_the_same_bits(dev):
+    cfg, xs, gs, W, What = make(dev)
+    assert cfg.n_chunks >= 3
+    ref = buffers(cfg, dev)
+    run_path(cfg, xs, gs, W, What, ref)
+    torch.cuda.synchronize()
+    b = buffers(cfg, dev)
+    extra = (torch.empty_like(b[1]), libgq.alloc_workspace(libgq.gq_hessian_workspace_bytes(cfg.chunk, cfg.d_in, cfg.g), dev))
+    graph = torch.cuda.CUDAGraph()
+    launches0 = libgq.gq_launch_count()
+    with torch.cuda.graph(graph):
+        run_path_ahead(cfg, xs, gs, W, What, b, extra)
+    assert libgq.gq_launch_count() - launches0 == cfg.n_chunks + 1 + 5
+    for _ in range(2):
+        b[0].fill_(7.0)
+        b[4].zero_()
+        graph.replay()
+    torch.cuda.synchronize()
+    libgq.gq_check()
+    assert torch.equal(b[0], ref[0]) and torch.equal(b[4], ref[4])
