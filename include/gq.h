@@ -157,9 +157,10 @@ int32_t gq_hessian_accumulate(const void *X, int64_t n, int64_t d_in, int64_t ld
  *               buffer that holds the saliency of all chunks: with equal leading dimensions the check is exact.)  The next call passes next_workspace as its workspace together
  *               with GQ_HESSIAN_S_PREPARED.
  * next_s and next_workspace receive the same bits as a gq_saliency_prepared call would write.
- * The spare warps stream about 1 TB/s.  Where the next chunk's gradients would take longer than this chunk's
- * Hessian work (few groups and d_out large against d_in: roughly 3000 * d_out * next_n > g * d_in^2 * n) the
- * call runs the saliency step as a kernel of its own before the Hessian kernel instead; results are the same.
+ * The spare warps of a full launch stream about 1 TB/s.  Where the next chunk's gradients would take longer than
+ * this chunk's Hessian work (few groups and d_out large against d_in: roughly 3000 * d_out * next_n > g * d_in^2 * n;
+ * or a small d_in, whose launch has few CTAs) the call runs the saliency step as a kernel of its own before the
+ * Hessian kernel instead; results are the same.
  * next_n == 0: the call is gq_hessian_accumulate.  n == 0: the call is gq_saliency_prepared for the next chunk
  * (after the arguments of this chunk have been checked).
  * The caller runs the saliency step of the very first chunk with gq_saliency_prepared.

@@ -581,8 +581,29 @@ static int32_t hessian_accumulate_impl(const void *X, int64_t n, int64_t d_in, i
     p.sched = gq::plan_schedule(units, ksteps, pairs, balanced);
     p.status = di->status_ptr;
     p.wait_budget_ns = wait_budget_ns();
-    if (ahead) p.ahead = *ahead;
     const int grid = 2 * ((p.sched.full_waves == 0 && p.sched.tail_pairs > 0) ? p.sched.tail_pairs : pairs);
+    if (ahead) {
+        // Does the saliency step fit behind the Hessian step?  Measured on B200 with all 148 CTAs: the two spare
+        // warps per CTA stream the gradient block at about 1.0e12 bytes/s while the tensor cores work through
+        // 1.25e15 issued flop/s; both rates shrink with the number of CTAs of a small launch.  If the gradients
+        // would take longer than 85 % of the Hessian work (plus 5 us, about what a launch of its own costs), the
+        // launch would only get longer: the saliency step then runs as a kernel of its own.
+        const double share = static_cast<double>(grid) / (2.0 * di->max_pairs);
+        const double tiles = 2.0 * units;              // every unit fills (up to) two 256 x 256 accumulators
+        const double t_hessian = 2.0 * gq::TILE_M * gq::TILE_N * (static_cast<double>(ksteps) * gq::TILE_K) * tiles / (1.25e15 * share);
+        const double t_saliency = static_cast<double>(ahead->n) * ahead->m * g * 2.0 / (1.0e12 * share);
+        if (t_saliency <= 0.85 * t_hessian + 5e-6) {
+            p.ahead = *ahead;
+        } else {
+            const unsigned grid_s = static_cast<unsigned>((static_cast<long long>(ahead->n) * g + 7) / 8);
+            {
+                LaunchScope scope(GQ_KERNEL_SALIENCY, st);
+                gq::saliency_kernel<<<grid_s, 256, 0, st>>>(ahead->grad, ahead->n, ahead->m, ahead->ld_grad, g, ahead->coef,
+                                                            ahead->s, ahead->ld_s, ahead->words);
+            }
+            GQ_CUDA(cudaGetLastError());
+        }
+    }
     {
         LaunchScope scope(GQ_KERNEL_HESSIAN, st);
         gq::hessian_kernel<<<grid, gq::HS_THREADS, gq::HS_SMEM_BYTES, st>>>(mapX, mapH, p);
@@ -637,22 +658,6 @@ int32_t gq_hessian_accumulate_ahead(const void *X, int64_t n, int64_t d_in, int6
             return GQ_ERR_INVALID_ARG;
         if (overlaps(next_grad, ng_bytes, H, h_bytes) || overlaps(next_grad, ng_bytes, workspace, ws_bytes))
             return GQ_ERR_INVALID_ARG;
-    }
-    {
-        // Does the saliency step fit behind the Hessian step?  Measured on B200: the two spare warps per CTA stream
-        // the gradient block at about 1.0e12 bytes/s while the tensor cores work through 1.25e15 issued flop/s.
-        // If the gradients would take longer than 85 % of the Hessian work (plus 5 us, about what a launch of its
-        // own costs), the launch would only get longer: run the saliency step as a kernel of its own instead.
-        const double nj = static_cast<double>((d_in + gq::TILE_N - 1) / gq::TILE_N);
-        const double tok = static_cast<double>((n + gq::TILE_K - 1) / gq::TILE_K * gq::TILE_K);
-        const double t_hessian = 2.0 * gq::TILE_M * gq::TILE_N * tok * (nj * (nj + 1.0) / 2.0) * g / 1.25e15;
-        const double t_saliency = static_cast<double>(next_n) * static_cast<double>(d_out) * 2.0 / 1.0e12;
-        if (t_saliency > 0.85 * t_hessian + 5e-6) {
-            if (int32_t rc = saliency_impl(next_grad, next_n, d_out, ld_grad, g, grad_scale, next_s, next_ld_s, true,
-                                           next_workspace, next_workspace_bytes, stream))
-                return rc;
-            return hessian_accumulate_impl(X, n, d_in, ld_x, s, ld_s, g, H, flags, workspace, workspace_bytes, nullptr, stream);
-        }
     }
     gq::SaliencyAhead a{};
     a.grad = static_cast<const __nv_bfloat16 *>(next_grad);
