@@ -524,6 +524,11 @@ size_t gq_hessian_workspace_bytes(int64_t n_max, int64_t d_in, int32_t g, uint32
     return hessian_ws_bytes(n_max, d_in, g);
 }
 
+// Rate at which the two spare warps per CTA of a full guided-Hessian launch stream gradients (measured on B200).
+#ifndef GQ_AHEAD_BYTES_PER_S
+#define GQ_AHEAD_BYTES_PER_S 1.0e12
+#endif
+
 static int32_t hessian_accumulate_impl(const void *X, int64_t n, int64_t d_in, int64_t ld_x, const float *s, int64_t ld_s,
                                        int32_t g, float *H, uint32_t flags, void *workspace, size_t workspace_bytes,
                                        const gq::SaliencyAhead *ahead, void *stream)
@@ -587,11 +592,12 @@ static int32_t hessian_accumulate_impl(const void *X, int64_t n, int64_t d_in, i
         // warps per CTA stream the gradient block at about 1.0e12 bytes/s while the tensor cores work through
         // 1.25e15 issued flop/s; both rates shrink with the number of CTAs of a small launch.  If the gradients
         // would take longer than 85 % of the Hessian work (plus 5 us, about what a launch of its own costs), the
-        // launch would only get longer: the saliency step then runs as a kernel of its own.
+        // launch would only get longer: the saliency step then runs as a kernel of its own.  (Leaving part of the
+        // block to the spare warps and the rest to a kernel was measured too: no better than the kernel alone.)
         const double share = static_cast<double>(grid) / (2.0 * di->max_pairs);
         const double tiles = 2.0 * units;              // every unit fills (up to) two 256 x 256 accumulators
         const double t_hessian = 2.0 * gq::TILE_M * gq::TILE_N * (static_cast<double>(ksteps) * gq::TILE_K) * tiles / (1.25e15 * share);
-        const double t_saliency = static_cast<double>(ahead->n) * ahead->m * g * 2.0 / (1.0e12 * share);
+        const double t_saliency = static_cast<double>(ahead->n) * ahead->m * g * 2.0 / (GQ_AHEAD_BYTES_PER_S * share);
         if (t_saliency <= 0.85 * t_hessian + 5e-6) {
             p.ahead = *ahead;
         } else {

@@ -277,15 +277,18 @@ def test_accumulate_ahead_matches_oracle_and_two_launch_path(dev, chunks, d_in, 
     check_H(H, H_o, upper_only=True)
 
 
-def test_accumulate_ahead_runs_saliency_separately_when_it_cannot_hide(dev):
-    """Few groups and many output channels: the next chunk's gradients would take longer to stream than this chunk's
+@pytest.mark.parametrize("d_in,d_out,n", [(64, 32768, 512),       # two CTAs
+                                         (1024, 8192, 4096)])    # fourteen CTAs, 67 MB of gradients
+def test_accumulate_ahead_runs_saliency_separately_when_it_cannot_hide(dev, d_in, d_out, n):
+    """One group and many output channels: the next chunk's gradients would take longer to stream than this chunk's
     Hessian work, so the call launches the saliency kernel on its own.  Same results."""
-    g, d_in, d_out, n = 1, 64, 32768, 512
+    g = 1
     gen = torch.Generator(device=dev).manual_seed(5)
     X = torch.randn(n, d_in, generator=gen, device=dev).to(torch.bfloat16)
     G = torch.randn(n, d_out, generator=gen, device=dev).to(torch.bfloat16)
     nb = libgq.gq_hessian_workspace_bytes(n, d_in, g)
     ws, ws_next = libgq.alloc_workspace(nb, dev), libgq.alloc_workspace(nb, dev)
+    ws_next.fill_(0xFF)
     s = libgq.gq_saliency_prepared(G, g, ws)
     H = torch.zeros((g, d_in, d_in), dtype=torch.float32, device=dev)
     launches = libgq.gq_launch_count()
