@@ -314,6 +314,13 @@ def test_accumulate_ahead_degenerate_and_errors(dev):
     H1 = torch.zeros_like(H)
     libgq.gq_hessian_accumulate(X, s, H1, ws, libgq.GQ_HESSIAN_S_PREPARED)
     assert torch.equal(torch.triu(H), torch.triu(H1))
+    # without GQ_HESSIAN_S_PREPARED the call prepares s itself (three kernels' work in two launches)
+    H2 = torch.zeros_like(H)
+    ws.fill_(0xFF)
+    ws_next.fill_(0xFF)
+    s_again = libgq.gq_hessian_accumulate_ahead(X, s, H2, ws, G, ws_next)
+    assert torch.equal(s_again, s) and torch.equal(torch.triu(H2), torch.triu(H1))
+    libgq.gq_saliency_prepared(G, g, ws)                 # restore the packed form of s for the checks below
     # no current chunk: the saliency step alone, H untouched
     s_next = libgq.gq_hessian_accumulate_ahead(X[:0], s[:, :0], H, ws, G, ws_next)
     assert torch.equal(s_next, s) and torch.equal(torch.triu(H), torch.triu(H1))
