@@ -51,18 +51,28 @@ def test_full_n_diagonal_and_probes(name, groups):
     V = rng.choice([-1.0, 1.0], size=(N_PROBES, d_in))                 # random signs
     V2 = V * V
     Hs = {g: torch.zeros((g, d_in, d_in), dtype=torch.float32, device=dev) for g in groups}
-    wss = {g: libgq.alloc_workspace(libgq.gq_hessian_workspace_bytes(cfg.chunk, d_in, g), dev) for g in groups}
+    wss = {g: [libgq.alloc_workspace(libgq.gq_hessian_workspace_bytes(cfg.chunk, d_in, g), dev) for _ in range(2)]
+           for g in groups}
     diag = {g: np.zeros((g, d_in)) for g in groups}
     hv = {g: np.zeros((g, N_PROBES, d_in)) for g in groups}
     var = {g: np.zeros((g * N_PROBES, d_in)) for g in groups}
     dvar = {g: np.zeros((g, d_in)) for g in groups}
     worst_s = 0.0
+    # bench.py's chunk loop: the first chunk's saliency as a launch of its own, then one call per chunk that adds the
+    # chunk to H and computes the next chunk's saliency (two scratch blocks in turn)
+    PREP = libgq.GQ_HESSIAN_S_PREPARED
+    grad_next = syn.grad_chunk(0)
+    s_gpu = {g: libgq.gq_saliency_prepared(grad_next, g, wss[g][0], 1.0) for g in groups}
     for c in range(cfg.n_chunks):
-        X, grad = syn.x_chunk(c), syn.grad_chunk(c)
-        s_gpu = {}
+        X, grad = syn.x_chunk(c), grad_next
+        grad_next = syn.grad_chunk(c + 1) if c + 1 < cfg.n_chunks else None
+        s_after = {}
         for g in groups:
-            s_gpu[g] = libgq.gq_saliency(grad, g, 1.0)
-            libgq.gq_hessian_accumulate(X, s_gpu[g], Hs[g], wss[g])
+            if grad_next is not None:
+                s_after[g] = libgq.gq_hessian_accumulate_ahead(X, s_gpu[g], Hs[g], wss[g][c & 1], grad_next,
+                                                               wss[g][(c + 1) & 1], 1.0, flags=PREP)
+            else:
+                libgq.gq_hessian_accumulate(X, s_gpu[g], Hs[g], wss[g][c & 1], flags=PREP)
         xb, gb = synth.bf16_bits(X), synth.bf16_bits(grad)
         del X, grad
         x = orc.bf16_bits_to_f64(xb)                                   # widened once per chunk, exactly
@@ -80,6 +90,7 @@ def test_full_n_diagonal_and_probes(name, groups):
             w = (s_ref[:, None, :] ** 2 * q.T[None, :, :]).reshape(g * N_PROBES, -1)     # s_k[i]^2 q_i per (k, probe)
             orc.hessian_diag(x, w, var[g], impl="numpy")
             orc.hessian_diag(x2, s_ref ** 2, dvar[g], impl="numpy")                      # sum_i s_i^2 x_ia^4
+        s_gpu = s_after
     libgq.gq_check()
     Vd = torch.from_numpy(V).to(dev)
     for g in groups:
