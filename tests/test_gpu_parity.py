@@ -416,17 +416,23 @@ def run_layer(cfg, dev, n_tokens=None, grad_scale=1.0, seed=0):
     g = cfg.g
     n = cfg.n if n_tokens is None else n_tokens
     H = torch.zeros((g, cfg.d_in, cfg.d_in), dtype=torch.float32, device=dev)
-    ws = libgq.alloc_workspace(libgq.gq_hessian_workspace_bytes(cfg.chunk, cfg.d_in, g), dev)
+    ws = [libgq.alloc_workspace(libgq.gq_hessian_workspace_bytes(cfg.chunk, cfg.d_in, g), dev) for _ in range(2)]
     xs, gs, ss = [], [], []
     done, c = 0, 0
     while done < n:
         nt = min(cfg.chunk, n - done)
-        X, grad = syn.x_chunk(c, nt), syn.grad_chunk(c, nt)
-        s = libgq.gq_saliency_prepared(grad, g, ws, grad_scale)          # the two launches per chunk bench.py makes
-        libgq.gq_hessian_accumulate(X, s, H, ws, flags=libgq.GQ_HESSIAN_S_PREPARED)
-        xs.append(X), gs.append(grad), ss.append(s)
+        xs.append(syn.x_chunk(c, nt)), gs.append(syn.grad_chunk(c, nt))
         done += nt
         c += 1
+    # the chunk loop bench.py times: saliency of the first chunk, then one launch per chunk that adds the chunk to H
+    # and computes the next chunk's saliency (two scratch blocks in turn)
+    ss.append(libgq.gq_saliency_prepared(gs[0], g, ws[0], grad_scale))
+    for c in range(len(xs)):
+        if c + 1 < len(xs):
+            ss.append(libgq.gq_hessian_accumulate_ahead(xs[c], ss[c], H, ws[c & 1], gs[c + 1], ws[(c + 1) & 1], grad_scale,
+                                                        flags=libgq.GQ_HESSIAN_S_PREPARED))
+        else:
+            libgq.gq_hessian_accumulate(xs[c], ss[c], H, ws[c & 1], flags=libgq.GQ_HESSIAN_S_PREPARED)
     libgq.gq_hessian_finalize(H)
     W, What = syn.weights()
     ows = libgq.alloc_workspace(libgq.gq_objective_workspace_bytes(cfg.d_in, cfg.d_out, g), dev)
