@@ -129,6 +129,15 @@ def test_aliasing_between_outputs_and_inputs_is_rejected(L):
     assert ahead(H, ns, nws) == INVALID                       # next grad inside H (written by the same launch)
     assert ahead(ng, ng + 16, nws) == INVALID                 # next s inside next grad
     assert ahead(ng, ns, nws, 16) == WS
+    # the next chunk's arguments are checked like gq_saliency_prepared's: (token, group) count below 2^31, d_out % g,
+    # 16-byte rows
+    big = L.gq_hessian_accumulate_ahead(X, 4, 64, 64, s_, 4, 2, H, 0, ws, 1024, ng, 1 << 30, 64, 64, 1.0, ns, 1 << 30,
+                                        nws, 1 << 34, None)
+    assert big == -3
+    assert L.gq_hessian_accumulate_ahead(X, 4, 64, 64, s_, 4, 2, H, 0, ws, 1024, ng, 4, 63, 64, 1.0, ns, 4, nws, 1024,
+                                         None) == INVALID
+    assert L.gq_hessian_accumulate_ahead(X, 4, 64, 64, s_, 4, 2, H, 0, ws, 1024, ng, 4, 64, 68, 1.0, ns, 4, nws, 1024,
+                                         None) == -2
     # s and next_s as column ranges of one [2, 16] buffer (leading dimension 16): disjoint columns are fine
     # although their spans interleave, shared columns are not
     in_one = lambda col: L.gq_hessian_accumulate_ahead(X, 4, 64, 64, s_, 16, 2, H, 0, ws, 1024, ng, 4, 64, 64, 1.0,
